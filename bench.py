@@ -1,0 +1,404 @@
+#!/usr/bin/env python
+"""Benchmark of the per-layer cache probe on the BERT-base-shaped workload.
+
+One step = one pass of the whole hot path over one batch at every layer: for each
+of the 12 per-layer banks, llmcache_probe (fingerprint, bank scan, threshold +
+compaction, gather of hits, metadata refresh) followed by llmcache_commit (victim
+selection, scatter of miss outputs, insertion).  Metric: probed sequences per
+second per layer = (sequences x layers) / time.
+
+    python bench.py --gpus 1 --steps 20 --warmup 5
+    python bench.py --impl reference ...       # the CPU oracle, timed as it stands
+
+Prints one JSON line on rank 0.
+"""
+import argparse
+import hashlib
+import json
+import os
+import subprocess
+import sys
+import threading
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+import numpy as np
+import torch
+
+METRIC = "probed sequences/sec per layer (fingerprint+scan+gather)"
+UNIT = "sequences/s"
+
+# BERT-base-shaped workload: 12 layers, d_model 768, batch 256 x seq_len 384, vocabulary 30,522,
+# 60% of the sequences are token-level edits (10% of positions) of 64 seed sequences, per-layer bank of
+# 2,048 entries (bf16 activations 384 x 768).
+CFG = dict(layers=12, d_model=768, seq_len=384, batch=256, vocab=30522, n_seeds=64, edit_fraction=0.60,
+           edit_positions=0.10, bank=2048, fp_dim=256, tau=0.90, pool_batches=24)
+
+# DRAM traffic per launch from an ncu capture of the named kernel on this workload, valid only while the
+# kernel's source file is unchanged (sha256 prefix of the file at capture time).
+NCU_TRAFFIC = {}
+
+
+def parse():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=20)
+    ap.add_argument("--warmup", type=int, default=5)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--e2e-steps", type=int, default=3)
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    return ap.parse_args()
+
+
+def measured_peaks():
+    p = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(p):
+        try:
+            return json.load(open(p)), "measured"
+        except Exception:
+            pass
+    return {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}, "fallback"
+
+
+class ClockSampler:
+    """Samples nvidia-smi clocks and throttle reasons while the timed region runs."""
+    Q = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,"
+         "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
+         "clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, index):
+        self.index, self.proc, self.lines = index, None, []
+
+    def start(self):
+        try:
+            self.proc = subprocess.Popen(["nvidia-smi", "-i", str(self.index), "--query-gpu=" + self.Q,
+                                          "--format=csv,noheader,nounits", "-lms", "100"],
+                                         stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+            self.th = threading.Thread(target=self._read, daemon=True)
+            self.th.start()
+        except Exception:
+            self.proc = None
+
+    def _read(self):
+        for ln in self.proc.stdout:
+            self.lines.append(ln.strip())
+
+    def stop(self):
+        if not self.proc:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=5)
+        except Exception:
+            self.proc.kill()
+        sm, mx, reasons = [], [], set()
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        for ln in self.lines:
+            f = [x.strip() for x in ln.split(",")]
+            if len(f) < 7:
+                continue
+            try:
+                sm.append(float(f[0])); mx.append(float(f[1]))
+            except ValueError:
+                continue
+            for nm, v in zip(names, f[3:7]):
+                if v.lower().startswith("active"):
+                    reasons.add(nm)
+        return {"sm_mhz": float(np.median(sm)) if sm else None, "sm_max_mhz": max(mx) if mx else None,
+                "samples": len(sm), "reasons": sorted(reasons)}
+
+
+# ------------------------------------------------------------------------------------------------
+def build_batches(wl, seeds_tok, count, seed, device):
+    """`count` batches of hidden states: 60% edits of the seeds, 40% fresh, shuffled."""
+    from paper_2512_16843_b200 import synth
+    B = CFG["batch"]
+    n_edit = int(round(B * CFG["edit_fraction"]))
+    out = []
+    for i in range(count):
+        ed, _ = wl.edited(seeds_tok, n_edit, CFG["edit_positions"], seed + 10 * i + 1)
+        fr = wl.tokens(B - n_edit, seed + 10 * i + 2)
+        tok = torch.cat([ed, fr])[synth.shuffled(B, seed + 10 * i + 3, device)]
+        out.append(wl.hidden(tok))
+    return out
+
+
+def run_ours(args):
+    from paper_2512_16843_b200 import binding as L
+    from paper_2512_16843_b200 import synth
+    L.lib()                                              # fail loudly if the CUDA library is missing
+    rank = int(os.environ.get("RANK", "0"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device (there is no CPU fallback)")
+    torch.cuda.set_device(local)
+    dev = torch.device("cuda", local)
+    dist = None
+    if world > 1:
+        import torch.distributed as dist
+        dist.init_process_group("nccl", device_id=dev)
+    Lyr, d, n, B, N, k = (CFG[x] for x in ("layers", "d_model", "seq_len", "batch", "bank", "fp_dim"))
+    seed = synth.BASE_SEED + 2000 + 100000 * rank
+    wl = synth.TokenWorkload(CFG["vocab"], n, d, seed, dev)
+    seeds_tok = wl.tokens(CFG["n_seeds"], seed + 5)
+    proj = synth.projection(d, k, seed + 6, dev)
+    banks = [L.Bank(device=local, capacity=N, seq_len=n, d_model=d, fp_dim=k, max_batch=B, hidden_dtype=L.BF16,
+                    proj=proj, tau=CFG["tau"], policy=L.LRU_STALENESS) for _ in range(Lyr)]
+    bufs = [L.ProbeBuffers(B, k, dev) for _ in range(Lyr)]
+    P = CFG["pool_batches"]
+    pool = build_batches(wl, seeds_tok, P, seed + 1000, dev)
+    miss_out = [synth.activations(B, n, d, seed + 50 + i, dev) for i in range(2)]
+    h_out = [torch.empty((B, n * d), dtype=torch.bfloat16, device=dev) for _ in range(3)]
+    # warm every bank to capacity through the library: the seeds, then fresh sequences
+    warm = [wl.hidden(torch.cat([seeds_tok, wl.tokens(B - CFG["n_seeds"], seed + 7)]))]
+    for i in range(1, N // B):
+        warm.append(wl.hidden(wl.tokens(B, seed + 20 + i)))
+    for l in range(Lyr):
+        for i, hb in enumerate(warm):
+            banks[l].probe(hb, bufs[l], h_out=h_out[0])
+            banks[l].commit(miss_out[i % 2], bufs[l], h_out=h_out[0])
+    del warm
+    torch.cuda.synchronize()
+
+    counter = [0]
+
+    def one_step(host_pool=None, stage=None, results=None):
+        s = counter[0]
+        counter[0] += 1
+        for l in range(Lyr):
+            i = (s + 2 * l) % P
+            if host_pool is None:
+                h = pool[i]
+            else:
+                stage[l % 2].copy_(host_pool[i], non_blocking=True)
+                h = stage[l % 2]
+            ho = h_out[(s + l) % 3]
+            banks[l].probe(h, bufs[l], h_out=ho)
+            banks[l].commit(miss_out[(s + l) % 2], bufs[l], h_out=ho)
+            if results is not None:
+                r = results[l]
+                r[0].copy_(bufs[l].hit, non_blocking=True)
+                r[1].copy_(bufs[l].slot, non_blocking=True)
+                r[2].copy_(bufs[l].score, non_blocking=True)
+
+    def barrier():
+        if dist is not None:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    for _ in range(args.warmup):
+        one_step()
+    barrier()
+    launches0 = sum(b.stats()["kernel_launches"] for b in banks)
+    hits0 = sum(b.stats()["hits"] for b in banks)
+    sampler = ClockSampler(local)
+    if rank == 0:
+        sampler.start()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    barrier()
+    e0.record()
+    for _ in range(args.steps):
+        one_step()
+    e1.record()
+    barrier()
+    ms = e0.elapsed_time(e1)
+    clocks = sampler.stop() if rank == 0 else None
+    if dist is not None:
+        t = torch.tensor([ms], device=dev)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        ms = float(t.item())
+    launches = sum(b.stats()["kernel_launches"] for b in banks) - launches0
+    hits = sum(b.stats()["hits"] for b in banks) - hits0
+    seqs = B * Lyr * args.steps
+    value = world * seqs / (ms * 1e-3)
+
+    # ---- per-kernel device time over the same loop (events around every launch) -------------------
+    for b in banks:
+        b.profile(True)
+    st0 = [b.stats() for b in banks]
+    for _ in range(args.steps):
+        one_step()
+    torch.cuda.synchronize()
+    prof = {}
+    for b in banks:
+        b.profile(False)
+        for name, (tms, cnt) in b.profile_read().items():
+            a = prof.setdefault(name, [0.0, 0])
+            a[0] += tms
+            a[1] += cnt
+    st1 = [b.stats() for b in banks]
+    H_avg = sum(s1["hits"] - s0["hits"] for s0, s1 in zip(st0, st1)) / float(Lyr * args.steps)
+    M_avg = B - H_avg
+    row = n * d * 2
+    algo_bytes = {                                       # algorithmic bytes per launch
+        "pool": B * n * d * 2 + B * k * 2,
+        "gather": H_avg * row * 2,
+        "scatter": M_avg * row * 3 + M_avg * k * 2,
+    }
+    total_ms = sum(v[0] for v in prof.values()) or 1.0
+    kernels = {name: {"ms_per_launch": v[0] / v[1], "launches": v[1], "share": v[0] / total_ms}
+               for name, v in prof.items() if v[1]}
+    dom = max((k_ for k_ in kernels if k_ in algo_bytes), key=lambda k_: kernels[k_]["share"])
+    peaks, peak_kind = measured_peaks()
+    achieved = algo_bytes[dom] / (kernels[dom]["ms_per_launch"] * 1e-3) / 1e9
+    roof = {"kernel": dom, "bound": "hbm", "achieved": achieved, "peak": peaks["hbm_gbs"], "unit": "GB/s",
+            "frac": achieved / peaks["hbm_gbs"], "peak_kind": "of " + peak_kind, "traffic": ncu_traffic(dom),
+            "algorithmic_bytes_per_launch": algo_bytes[dom], "all_kernels": {}}
+    for name in kernels:
+        ent = dict(kernels[name])
+        if name in algo_bytes:
+            ent["achieved_GBps"] = algo_bytes[name] / (ent["ms_per_launch"] * 1e-3) / 1e9
+            ent["frac_of_hbm_peak"] = ent["achieved_GBps"] / peaks["hbm_gbs"]
+        roof["all_kernels"][name] = ent
+
+    # ---- end to end: inputs come from pinned host memory, decisions go back to the host ------------
+    e2e = None
+    if args.e2e_steps > 0:
+        host_pool = [p.cpu().pin_memory() for p in pool]
+        stage = [torch.empty_like(pool[0]) for _ in range(2)]
+        results = [(torch.empty(B, dtype=torch.uint8).pin_memory(), torch.empty(B, dtype=torch.int32).pin_memory(),
+                    torch.empty(B, dtype=torch.float32).pin_memory()) for _ in range(Lyr)]
+        one_step(host_pool, stage, results)
+        barrier()
+        e0.record()
+        for _ in range(args.e2e_steps):
+            one_step(host_pool, stage, results)
+        e1.record()
+        barrier()
+        ems = e0.elapsed_time(e1)
+        if dist is not None:
+            t = torch.tensor([ems], device=dev)
+            dist.all_reduce(t, op=dist.ReduceOp.MAX)
+            ems = float(t.item())
+        e2e = {"value": world * B * Lyr * args.e2e_steps / (ems * 1e-3), "unit": UNIT,
+               "h2d_bytes_per_step": Lyr * B * n * d * 2, "d2h_bytes_per_step": Lyr * B * 9 + Lyr * 8,
+               "steps": args.e2e_steps}
+        del host_pool
+
+    cpu = None
+    if rank == 0 and world == 1 and not args.no_cpu_baseline:
+        cpu = cpu_baseline_from_gpu_state(banks, pool, proj, counter[0])
+
+    if rank == 0:
+        out = {"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
+               "warmup": args.warmup, "ms_per_step": ms / args.steps, "higher_is_better": True, "scaling": "weak",
+               "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
+               "config": {"workload": "BERT-base-shaped encoder: 12 per-layer banks x 2048 entries (bf16 384x768), "
+                                      "batch 256 x seq_len 384, d_model 768, fp_dim 256 (projected), tau 0.90, "
+                                      "60% token-level edits of 64 seeds",
+                          "step": "probe + commit on each of 12 layers", "hit_fraction": hits / float(seqs),
+                          "l2": "inputs larger than L2: every layer of a step reads a different 151 MB batch out "
+                                "of a pool of 24, plus 1.2 GB of bank rows per layer",
+                          "parallelism": "independent replicas per GPU, no collective" if world > 1 else "single GPU"},
+               "e2e": e2e, "gpu_launches": launches, "roofline": roof, "cpu_baseline": cpu, "clocks": clocks}
+        print(json.dumps(out))
+    for b in banks:
+        b.close()
+    if dist is not None:
+        dist.destroy_process_group()
+
+
+def ncu_traffic(kernel):
+    ent = NCU_TRAFFIC.get(kernel)
+    if not ent:
+        return None
+    path = os.path.join(ROOT, "paper_2512_16843_b200", "csrc", ent["file"])
+    sha = hashlib.sha256(open(path, "rb").read()).hexdigest()[:12]
+    return ent["bytes_per_launch"] if sha == ent["sha"] else None
+
+
+# ------------------------------------------------------------------------------------------------
+def blas_threads():
+    try:
+        from threadpoolctl import threadpool_info
+        return max([i.get("num_threads", 1) for i in threadpool_info()] + [1])
+    except Exception:
+        return 1
+
+
+def cpu_baseline_from_gpu_state(banks, pool, proj, step, budget_s=20.0, max_layers=4):
+    """The oracle, as it stands, on the same batches and the banks' current contents."""
+    from oracle import llmcache_oracle as O
+    from paper_2512_16843_b200 import binding as L
+    from paper_2512_16843_b200 import synth
+    from tests import parity_util as U
+    Lyr, B, P = CFG["layers"], CFG["batch"], CFG["pool_batches"]
+    done, t_total = 0, 0.0
+    for l in range(min(Lyr, max_layers)):
+        ob = U.oracle_bank_like(banks[l], proj, None)
+        U.pull_state(banks[l], ob, with_act=True)
+        h = synth.bf16_bits(pool[(step + 2 * l) % P])
+        mo = np.zeros((B, ob.seq_len * ob.d_model), dtype=np.uint16)
+        h_out = np.zeros((B, ob.seq_len * ob.d_model), dtype=np.uint16)
+        t0 = time.perf_counter()
+        pr = O.probe(ob, h, "bf16", h_out=h_out)
+        O.commit(ob, pr, mo[:len(pr.miss_idx)], h_out)
+        t_total += time.perf_counter() - t0
+        done += 1
+        del ob
+        if t_total > budget_s:
+            break
+    return {"value": done * B / t_total, "unit": UNIT, "cores": blas_threads(), "kind": "oracle",
+            "sample": f"{done} of {Lyr} layers x the full batch of {B} sequences (probe + commit), "
+                      f"{t_total:.1f} s of CPU time; numpy, float64"}
+
+
+def run_reference(args):
+    """Times the CPU oracle on the same workload shape; each step is one layer's batch (a bounded sample)."""
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    from oracle import llmcache_oracle as O
+    from paper_2512_16843_b200 import synth
+    d, n, B, N, k = (CFG[x] for x in ("d_model", "seq_len", "batch", "bank", "fp_dim"))
+    seed = synth.BASE_SEED + 2000
+    wl = synth.TokenWorkload(CFG["vocab"], n, d, seed, "cpu")
+    seeds_tok = wl.tokens(CFG["n_seeds"], seed + 5)
+    proj = synth.projection(d, k, seed + 6, "cpu")
+    ob = O.Bank(capacity=N, seq_len=n, d_model=d, fp_dim=k, tau=CFG["tau"], proj=synth.bf16_bits(proj))
+    acts = np.zeros((B, n * d), dtype=np.uint16)
+    h_out = np.zeros((B, n * d), dtype=np.uint16)
+    warm_tok = [torch.cat([seeds_tok, wl.tokens(B - CFG["n_seeds"], seed + 7)])]
+    warm_tok += [wl.tokens(B, seed + 20 + i) for i in range(1, N // B)]
+    for tok in warm_tok:
+        pr = O.probe(ob, synth.bf16_bits(wl.hidden(tok)), "bf16")
+        O.commit(ob, pr, acts[:len(pr.miss_idx)])
+    total = args.warmup + args.steps
+    batches = build_batches(wl, seeds_tok, total, seed + 1000, "cpu")
+    hits = 0
+    t_timed = 0.0
+    for i, hb in enumerate(batches):
+        h = synth.bf16_bits(hb)
+        t0 = time.perf_counter()
+        pr = O.probe(ob, h, "bf16", h_out=h_out)
+        O.commit(ob, pr, acts[:len(pr.miss_idx)], h_out)
+        dt = time.perf_counter() - t0
+        if i >= args.warmup:
+            t_timed += dt
+            hits += int(pr.hit.sum())
+    value = B * args.steps / t_timed
+    cores = blas_threads()
+    out = {"impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus,
+           "steps": args.steps, "warmup": args.warmup, "ms_per_step": 1e3 * t_timed / args.steps,
+           "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+           "config": {"workload": "BERT-base-shaped encoder: bank of 2048 entries (bf16 384x768), batch 256 x "
+                                  "seq_len 384, d_model 768, fp_dim 256 (projected), tau 0.90, 60% token-level edits "
+                                  "of 64 seeds", "step": "probe + commit of one layer's batch (bounded sample of the "
+                                  "12-layer step)", "hit_fraction": hits / float(B * args.steps)},
+           "cpu_baseline": {"value": value, "unit": UNIT, "cores": cores, "kind": "oracle",
+                            "sample": "one layer x the full batch of 256 sequences per step; numpy, float64"},
+           "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+           "gpu_launches": 0}
+    print(json.dumps(out))
+
+
+if __name__ == "__main__":
+    a = parse()
+    if a.impl == "reference":
+        run_reference(a)
+    else:
+        run_ours(a)

@@ -1,0 +1,217 @@
+/*
+ * llmcache.h -- C ABI of the per-layer cache probe of LLMCache
+ * ("Layer-Wise Caching Strategies for Accelerated Reuse in Transformer
+ * Inference"), implemented as hand-written CUDA for sm_100a.
+ *
+ * One bank object stands for the cache C_l of one transformer layer
+ * (Sec. III-B: an independent set of (fingerprint, layer output) tuples).
+ * Per batch of B sequences entering the layer the caller does
+ *
+ *     llmcache_probe(bank, h_in, ...)      lookup + reuse      (Algorithm 1, if-branch)
+ *     <run the layer on the M compacted misses>
+ *     llmcache_commit(bank, miss_out, ...) scatter + insert    (Algorithm 1, else-branch)
+ *
+ * and, whenever it wants to bound growth or drop outdated keys,
+ *     llmcache_evict(bank, mode, ...)      refresh controller  (Sec. III-E, IV-D).
+ *
+ * Conventions that hold for every function:
+ *  - Plain C types only.  "device" pointers are CUDA device addresses on the
+ *    bank's GPU; "host" pointers are ordinary process memory.  `stream` is a
+ *    cudaStream_t passed as void* (NULL = the legacy default stream).
+ *  - All GPU work is enqueued on `stream` and the call returns without
+ *    waiting unless stated otherwise.  A bank must be driven from one stream
+ *    at a time; probe and commit of one bank alternate.
+ *  - The caller owns every input/output buffer; the bank owns its storage
+ *    (or borrows `arena`) until llmcache_bank_destroy.
+ *  - Return value: LLMCACHE_OK (0) or a negative llmcache_status.  Argument
+ *    errors are detected on the host before anything is launched.  There is no
+ *    CPU fallback: without a usable CUDA device every call fails with
+ *    LLMCACHE_ERR_CUDA.
+ *  - Shapes: n = seq_len, d = d_model, k = fp_dim, N = capacity.
+ *    d must be a multiple of 8, k a multiple of 64, rows are row-major and
+ *    densely packed, every device pointer must be 16-byte aligned.
+ */
+#ifndef LLMCACHE_H
+#define LLMCACHE_H
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+#define LLMCACHE_ABI_VERSION 1u
+
+typedef struct llmcache_bank llmcache_bank_t;
+
+typedef enum {
+  LLMCACHE_OK = 0,
+  LLMCACHE_ERR_ARG = -1,          /* null pointer, bad enum, bad struct_size, misaligned pointer */
+  LLMCACHE_ERR_SHAPE = -2,        /* size outside what the bank was created for */
+  LLMCACHE_ERR_NOMEM = -3,        /* allocation failed or arena too small */
+  LLMCACHE_ERR_CUDA = -4,         /* a CUDA runtime/driver call failed (incl. no device) */
+  LLMCACHE_ERR_STATE = -5,        /* calls out of order (commit without matching probe, ...) */
+  LLMCACHE_ERR_TIMEOUT = -6,      /* a bounded device-side wait expired (sticky, see bank_status) */
+  LLMCACHE_ERR_UNSUPPORTED = -7   /* valid request this build does not serve */
+} llmcache_status;
+
+enum { LLMCACHE_F32 = 0, LLMCACHE_BF16 = 1 };                 /* dtype of probe inputs h_in */
+enum { LLMCACHE_GT = 0, LLMCACHE_GE = 1 };                    /* hit iff sim > tau  |  sim >= tau */
+enum { LLMCACHE_LRU = 0, LLMCACHE_LRU_STALENESS = 1 };        /* eviction policy */
+enum { LLMCACHE_EVICT_STALE = 0, LLMCACHE_EVICT_IDLE = 1, LLMCACHE_EVICT_ALL = 2, LLMCACHE_EVICT_SLOTS = 3 };
+enum {                                                        /* arrays addressable by export/import */
+  LLMCACHE_WHAT_FP = 0,          /* bf16  [N,k]   stored fingerprints (unit length, rounded)   */
+  LLMCACHE_WHAT_RB = 1,          /* f32   [N]     1/||stored fingerprint||                      */
+  LLMCACHE_WHAT_VALID = 2,       /* u8    [N]     1 = slot occupied                             */
+  LLMCACHE_WHAT_LAST_USE = 3,    /* u32   [N]     tick of last hit (or of insertion)            */
+  LLMCACHE_WHAT_INSERT_TICK = 4, /* u32   [N]                                                   */
+  LLMCACHE_WHAT_HITS = 5,        /* u32   [N]     matches since insertion (saturating)          */
+  LLMCACHE_WHAT_RATE = 6,        /* u32   [N]     decayed match rate, Q8, as of RATE_EPOCH      */
+  LLMCACHE_WHAT_RATE_EPOCH = 7,  /* u32   [N]     tick / half_life_ticks at the last update     */
+  LLMCACHE_WHAT_ACT = 8,         /* bf16  [act_rows, n*d]  cached layer outputs                 */
+  LLMCACHE_WHAT_TICK = 9         /* u64   [1]     number of probe calls so far                  */
+};
+
+/* Bank description (Sec. III-B; the knobs of Sec. IV-E/VI-D: threshold, cache
+ * size, eviction policy).  Zero-initialise, set struct_size = sizeof, fill in. */
+typedef struct llmcache_bank_desc {
+  uint32_t struct_size;
+  int32_t  device;            /* CUDA device ordinal */
+  uint32_t capacity;          /* N >= 1 slots */
+  uint32_t seq_len;           /* n >= 1 */
+  uint32_t d_model;           /* d, multiple of 8, <= 8192 */
+  uint32_t fp_dim;            /* k, multiple of 64, <= 2048; must equal d_model when proj == NULL */
+  uint32_t hidden_dtype;      /* LLMCACHE_F32 | LLMCACHE_BF16 */
+  uint32_t act_rows;          /* rows of the activation store; 0 => capacity.  slot j uses row j % act_rows.
+                                 A bank with act_rows < capacity can be probed but not committed to. */
+  uint32_t max_batch;         /* largest B any call will pass (sizes internal scratch) */
+  float    tau;               /* default similarity threshold */
+  uint32_t cmp;               /* LLMCACHE_GT (Sec. IV-A, Algorithm 1) | LLMCACHE_GE (Sec. III-C) */
+  uint32_t policy;            /* LLMCACHE_LRU | LLMCACHE_LRU_STALENESS (Sec. IV-D) */
+  uint32_t half_life_ticks;   /* decayed match rate halves every this many probe calls (0 => 8) */
+  uint32_t stale_floor_q8;    /* stale if rate (Q8) below this ...                       (0 => 64) */
+  uint32_t min_age_ticks;     /* ... and at least this old                              (0 => 4) */
+  uint32_t max_idle_ticks;    /* LLMCACHE_EVICT_IDLE drops entries unused for longer    (0 => 32) */
+  uint32_t store_act;         /* 1 = keep layer outputs (normal); 0 = keys only (scan benchmarks) */
+  const void*  proj;          /* device, bf16 [d,k] row-major projection (Sec. IV-B "Dimensionality
+                                 Reduction"), copied at create; NULL => identity (k == d) */
+  const float* center;        /* device, f32 [d] subtracted before projection, copied; NULL => 0 */
+  void*    arena;             /* device memory to build the bank in (256-byte aligned), or NULL to
+                                 let the library cudaMalloc it */
+  size_t   arena_bytes;       /* size of arena; llmcache_bank_bytes tells how much is needed */
+} llmcache_bank_desc;
+
+/* Per-call outputs of a probe, all caller-owned DEVICE buffers sized for the
+ * call's B (counts_host excepted).  commit reads the same struct back. */
+typedef struct llmcache_probe_io {
+  uint8_t*  hit;          /* [B]   1 = reuse                                                    */
+  int32_t*  slot;         /* [B]   matching slot, -1 on miss                                    */
+  float*    score;        /* [B]   best cosine (-inf: bank empty; 0: degenerate fingerprint)    */
+  int32_t*  hit_idx;      /* [B]   first H entries: indices of hits, ascending                  */
+  int32_t*  miss_idx;     /* [B]   first M entries: indices of misses, ascending                */
+  uint32_t* counts;       /* [2]   {H, M}                                                       */
+  uint32_t* counts_host;  /* optional pinned HOST [2]; filled by an async copy on the stream    */
+  void*     fp;           /* [B,k] bf16 query fingerprints (probe writes; probe_fp: caller's)   */
+  float*    rq;           /* [B]   1/||fp|| (0 marks a degenerate fingerprint)                  */
+  void*     h_miss;       /* optional [B,n,d] (dtype of h_in): rows of the misses, compacted    */
+  uint64_t  generation;   /* written by probe, checked by commit                                */
+} llmcache_probe_io;
+
+typedef struct llmcache_stats {
+  uint64_t probes, sequences, hits, misses, degenerate;
+  uint64_t inserts, evictions, dropped, flushed, resident;
+  uint64_t kernel_launches;   /* kernels this bank has enqueued so far */
+} llmcache_stats;
+
+/* Kernels of the path, for llmcache_bank_profile_read. */
+enum {
+  LLMCACHE_K_POOL = 0,      /* Sec. IV-B pooled reduction                          */
+  LLMCACHE_K_PROJECT = 1,   /* Sec. IV-B projection + unit length + rounding       */
+  LLMCACHE_K_ROWNORM = 2,   /* inverse norms of caller-supplied fingerprints       */
+  LLMCACHE_K_SCAN = 3,      /* Sec. III-C cosine scan + best slot                  */
+  LLMCACHE_K_DECIDE = 4,    /* Sec. IV-A threshold + hit/miss compaction           */
+  LLMCACHE_K_TOUCH = 5,     /* Sec. III-E metadata refresh of matched slots        */
+  LLMCACHE_K_GATHER = 6,    /* Algorithm 1 reuse: copy of cached outputs           */
+  LLMCACHE_K_SELECT = 7,    /* Sec. IV-D victim selection                          */
+  LLMCACHE_K_SCATTER = 8,   /* Algorithm 1 insert: write-back + store              */
+  LLMCACHE_K_EVICT = 9,     /* Sec. III-E flushes                                  */
+  LLMCACHE_K_COUNT = 10
+};
+
+uint32_t    llmcache_abi_version(void);
+const char* llmcache_strerror(int status);
+/* Text of the most recent CUDA error seen by this thread inside the library ("" if none). */
+const char* llmcache_last_cuda_error(void);
+
+/* Bytes of device memory a bank of this description needs (for `arena`). */
+int llmcache_bank_bytes(const llmcache_bank_desc* desc, size_t* bytes_out);
+
+/* Build an empty bank C_l (Sec. III-B).  Synchronous. */
+int llmcache_bank_create(const llmcache_bank_desc* desc, llmcache_bank_t** bank_out);
+
+/* Release the bank (frees its memory unless it lives in a caller arena).  Synchronises the device. */
+int llmcache_bank_destroy(llmcache_bank_t* bank);
+
+/* Fingerprint only (Sec. IV-B): mean over the n positions of h_in[b], minus
+ * center, times proj, scaled to unit length, rounded to bf16.
+ * h_in: device [B,n,d] of the bank's hidden_dtype.  fp: device bf16 [B,k].  rq: device f32 [B]. */
+int llmcache_fingerprint(llmcache_bank_t* bank, const void* h_in, uint32_t B,
+                         void* fp, float* rq, void* stream);
+
+/* Lookup and reuse for one batch (Sec. III-C, Sec. IV-A case equation,
+ * Algorithm 1 "if exists (f',h') with sim > tau then h_l <- h'").
+ * Advances the bank's tick.  For each sequence: fingerprint h_in[b], cosine
+ * against every occupied slot, best slot (ties: lowest), hit iff best > tau
+ * (>= under LLMCACHE_GE).  h_out[b] (device bf16 [B,n,d]) receives the stored
+ * layer output of each hit, byte for byte; rows of misses are left untouched.
+ * tau: NaN => the bank's default.  B == 0 is valid and does nothing but tick.
+ * All sequences see the bank as it was when the call began. */
+int llmcache_probe(llmcache_bank_t* bank, const void* h_in, uint32_t B, float tau,
+                   void* h_out, llmcache_probe_io* io, void* stream);
+
+/* Same with precomputed fingerprints (Algorithm 1 computes f_X once and reuses
+ * it at every layer): io->fp holds bf16 [B,k] on entry; io->rq is written.
+ * h_in may be NULL (then io->h_miss is not produced). */
+int llmcache_probe_fp(llmcache_bank_t* bank, const void* h_in, uint32_t B, float tau,
+                      void* h_out, llmcache_probe_io* io, void* stream);
+
+/* After the layer ran on the misses (Algorithm 1 else-branch, "C_l[f_X] <- h_l";
+ * victim choice per Sec. III-E / IV-D).  miss_out: device bf16 [M,n,d] in the
+ * order of io->miss_idx.  Writes miss_out[m] to h_out[miss_idx[m]] (skipped when
+ * h_out is NULL) and inserts it under the probe's fingerprint.  Victims: free
+ * slots ascending, then occupied slots by ascending (stale first, decayed rate,
+ * last use, slot).  Misses with rq == 0 and misses beyond capacity are dropped.
+ * new_slot: optional device i32 [B]; [m] = slot taken, -1 = dropped. */
+int llmcache_commit(llmcache_bank_t* bank, const void* miss_out, const llmcache_probe_io* io,
+                    void* h_out, int32_t* new_slot, void* stream);
+
+/* Refresh controller (Sec. III-E): drop every stale entry, every entry idle
+ * for more than max_idle_ticks, all entries, or the n listed slots (device
+ * i32).  n_evicted_dev: optional device u32 [1] receiving the count. */
+int llmcache_evict(llmcache_bank_t* bank, uint32_t mode, const int32_t* slots, uint32_t n,
+                   uint32_t* n_evicted_dev, void* stream);
+
+/* Copy one of the bank's arrays (LLMCACHE_WHAT_*) out to / in from `ptr`
+ * (host or device), `bytes` must equal the array's size.  Enqueued on stream;
+ * host memory must stay valid until the stream has run.  TICK is synchronous. */
+int llmcache_bank_export(llmcache_bank_t* bank, uint32_t what, void* ptr, size_t bytes, void* stream);
+int llmcache_bank_import(llmcache_bank_t* bank, uint32_t what, const void* ptr, size_t bytes, void* stream);
+
+/* Counters since creation.  Synchronises the device. */
+int llmcache_bank_stats(llmcache_bank_t* bank, llmcache_stats* host_out);
+
+/* Per-kernel device timing (the paper has no counterpart; this is instrumentation).  While
+ * enabled, every kernel launch of this bank is bracketed by CUDA events on its stream.
+ * profile_read synchronises the device, returns the summed duration and the number of launches
+ * of kernel `kernel_id` since the last read, and clears them. */
+int llmcache_bank_profile(llmcache_bank_t* bank, int enable);
+int llmcache_bank_profile_read(llmcache_bank_t* bank, uint32_t kernel_id, double* total_ms, uint64_t* launches);
+
+/* Sticky device-side status (LLMCACHE_OK or LLMCACHE_ERR_TIMEOUT).  Synchronises the device. */
+int llmcache_bank_status(llmcache_bank_t* bank);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* LLMCACHE_H */

@@ -1,0 +1,127 @@
+// Threshold decision, hit/miss compaction and metadata refresh.
+//   Sec. IV-A case equation / Algorithm 1: hit iff sim > tau (">=" selectable, Sec. III-C).
+//   Sec. III-E / IV-D: recency, match count and decayed match rate of matched slots.
+#include "llmcache_internal.cuh"
+
+namespace llmc {
+
+constexpr int DEC_THREADS = 1024;
+
+// Exclusive rank of `pred` among the threads of the block (in thread order) and
+// the block total.  warp_tot is a 32-word shared array.
+__device__ __forceinline__ uint32_t block_rank(bool pred, uint32_t* warp_tot, uint32_t& total) {
+  const uint32_t lane = threadIdx.x & 31, w = threadIdx.x >> 5;
+  const uint32_t bal = __ballot_sync(0xFFFFFFFFu, pred);
+  const uint32_t in_warp = __popc(bal & ((1u << lane) - 1u));
+  __syncthreads();
+  if (lane == 0) warp_tot[w] = __popc(bal);
+  __syncthreads();
+  uint32_t before = 0, tot = 0;
+  const uint32_t nw = blockDim.x >> 5;
+  for (uint32_t i = 0; i < nw; ++i) {
+    const uint32_t c = warp_tot[i];
+    if (i < w) before += c;
+    tot += c;
+  }
+  total = tot;
+  return before + in_warp;
+}
+
+// One block walks the batch in order, so hit_idx and miss_idx come out ascending.
+__global__ void __launch_bounds__(DEC_THREADS)
+k_decide_compact(unsigned long long* __restrict__ best, const float* __restrict__ rq,
+                 uint32_t B, float tau, int cmp_ge,
+                 uint8_t* __restrict__ hit, int32_t* __restrict__ slot, float* __restrict__ score,
+                 int32_t* __restrict__ hit_idx, int32_t* __restrict__ miss_idx,
+                 uint32_t* __restrict__ counts, uint32_t* __restrict__ hitcnt,
+                 unsigned long long* __restrict__ stats) {
+  __shared__ uint32_t warp_tot[32];
+  uint32_t hbase = 0, mbase = 0, ndegen = 0;
+  for (uint32_t base = 0; base < B; base += DEC_THREADS) {
+    const uint32_t b = base + threadIdx.x;
+    bool is_hit = false, in_range = b < B;
+    if (in_range) {
+      const unsigned long long pk = best[b];
+      best[b] = 0ull;                                   // ready for the next probe
+      const float r = rq[b];
+      float sc;
+      int32_t sl = -1;
+      if (!(r > 0.f)) {
+        sc = 0.f;                                       // degenerate fingerprint: never a hit
+        ++ndegen;
+      } else if (pk == 0ull) {
+        sc = -INFINITY;                                 // no occupied slot
+      } else {
+        sc = orderable_float((uint32_t)(pk >> 32)) * r;
+        sl = (int32_t)(0xFFFFFFFFu - (uint32_t)pk);
+        is_hit = cmp_ge ? (sc >= tau) : (sc > tau);
+      }
+      if (!is_hit) sl = -1;
+      hit[b] = is_hit ? 1 : 0;
+      slot[b] = sl;
+      score[b] = sc;
+      if (is_hit) atomicAdd(hitcnt + sl, 1u);
+    }
+    uint32_t nh;
+    const uint32_t r = block_rank(is_hit, warp_tot, nh);
+    if (in_range) {
+      if (is_hit) hit_idx[hbase + r] = (int32_t)b;
+      else        miss_idx[mbase + (threadIdx.x - r)] = (int32_t)b;
+    }
+    const uint32_t chunk = min((uint32_t)DEC_THREADS, B - base);
+    hbase += nh;
+    mbase += chunk - nh;
+  }
+  // degenerate count: block reduction by atomics on shared memory
+  __shared__ uint32_t sdeg;
+  if (threadIdx.x == 0) sdeg = 0;
+  __syncthreads();
+  if (ndegen) atomicAdd(&sdeg, ndegen);
+  __syncthreads();
+  if (threadIdx.x == 0) {
+    counts[0] = hbase;
+    counts[1] = mbase;
+    stats[ST_SEQ] += B;
+    stats[ST_HIT] += hbase;
+    stats[ST_MISS] += mbase;
+    stats[ST_DEGEN] += sdeg;
+  }
+}
+
+// Apply the matches of this probe to the slots' metadata; one thread per slot,
+// so the result does not depend on the order of the batch.
+__global__ void k_touch(uint32_t* __restrict__ hitcnt, uint32_t* __restrict__ last_use,
+                        uint32_t* __restrict__ hits, uint32_t* __restrict__ rate,
+                        uint32_t* __restrict__ rate_epoch, uint32_t N, uint32_t tick, uint32_t epoch) {
+  const uint32_t j = blockIdx.x * blockDim.x + threadIdx.x;
+  if (j >= N) return;
+  const uint32_t c = hitcnt[j];
+  if (c == 0) return;
+  hitcnt[j] = 0;
+  const unsigned long long m = (unsigned long long)rate_now(rate[j], rate_epoch[j], epoch) + (unsigned long long)HIT_Q8 * c;
+  rate[j] = m > M_CAP ? M_CAP : (uint32_t)m;
+  rate_epoch[j] = epoch;
+  last_use[j] = tick;
+  const unsigned long long h = (unsigned long long)hits[j] + c;
+  hits[j] = h > 0xFFFFFFFFull ? 0xFFFFFFFFu : (uint32_t)h;
+}
+
+cudaError_t launch_decide(llmcache_bank* bk, uint32_t B, float tau, const float* rq,
+                          const llmcache_probe_io* io, cudaStream_t st) {
+  ProfScope prof(bk, LLMCACHE_K_DECIDE, st);
+  k_decide_compact<<<1, DEC_THREADS, 0, st>>>(bk->a.best, rq, B, tau, bk->desc.cmp == LLMCACHE_GE,
+                                              io->hit, io->slot, io->score, io->hit_idx, io->miss_idx,
+                                              io->counts, bk->a.hitcnt, bk->a.stats);
+  return cudaGetLastError();
+}
+
+cudaError_t launch_touch(llmcache_bank* bk, cudaStream_t st) {
+  const uint32_t N = bk->desc.capacity;
+  const uint32_t epoch = (uint32_t)(bk->tick / bk->pol.half_life);
+  ProfScope prof(bk, LLMCACHE_K_TOUCH, st);
+  k_touch<<<(N + 255) / 256, 256, 0, st>>>(bk->a.hitcnt, bk->a.last_use, bk->a.hits, bk->a.rate,
+                                           bk->a.rate_epoch, N, (uint32_t)bk->tick, epoch);
+  return cudaGetLastError();
+}
+
+}  // namespace llmc

@@ -1,0 +1,247 @@
+// Replacement controller (Sec. III-E, Sec. IV-D): choice of the slots that
+// receive the inserted misses (free slots first, then least-recently-used with
+// stale entries ahead), and the explicit flushes.  Integer arithmetic only.
+#include "llmcache_internal.cuh"
+
+namespace llmc {
+
+constexpr int SEL_THREADS = 1024;
+constexpr uint32_t SEL_SMEM_SORT = 2048;      // sort in shared memory up to this many candidates
+
+__device__ __forceinline__ uint32_t sel_rank(bool pred, uint32_t* warp_tot, uint32_t& total) {
+  const uint32_t lane = threadIdx.x & 31, w = threadIdx.x >> 5;
+  const uint32_t bal = __ballot_sync(0xFFFFFFFFu, pred);
+  const uint32_t in_warp = __popc(bal & ((1u << lane) - 1u));
+  __syncthreads();
+  if (lane == 0) warp_tot[w] = __popc(bal);
+  __syncthreads();
+  uint32_t before = 0, tot = 0;
+  for (uint32_t i = 0; i < (SEL_THREADS >> 5); ++i) {
+    const uint32_t c = warp_tot[i];
+    if (i < w) before += c;
+    tot += c;
+  }
+  total = tot;
+  return before + in_warp;
+}
+
+struct MetaView {
+  const uint8_t* valid;
+  const uint32_t *last_use, *insert_tick, *rate, *rate_epoch;
+};
+
+__device__ __forceinline__ unsigned long long key_of(const MetaView& mv, const PolicyParams& p,
+                                                     uint32_t j, uint32_t tick, uint32_t epoch) {
+  return evict_key(p, tick, epoch, mv.rate[j], mv.rate_epoch[j], mv.insert_tick[j], mv.last_use[j]);
+}
+
+// In-place bitonic sort of (key, slot) pairs, ascending by key then slot.
+// len is a power of two; the arrays may live in shared or global memory.
+__device__ void bitonic_sort(unsigned long long* key, uint32_t* val, uint32_t len) {
+  for (uint32_t size = 2; size <= len; size <<= 1) {
+    for (uint32_t stride = size >> 1; stride > 0; stride >>= 1) {
+      __syncthreads();
+      for (uint32_t i = threadIdx.x; i < len; i += SEL_THREADS) {
+        const uint32_t l = i ^ stride;
+        if (l > i) {
+          const unsigned long long ka = key[i], kb = key[l];
+          const uint32_t va = val[i], vb = val[l];
+          const bool a_gt_b = (ka > kb) || (ka == kb && va > vb);
+          const bool ascending = (i & size) == 0;
+          if (a_gt_b == ascending) {
+            key[i] = kb; key[l] = ka;
+            val[i] = vb; val[l] = va;
+          }
+        }
+      }
+    }
+  }
+  __syncthreads();
+}
+
+// One block.  Output: new_slot[m] for every miss m (in miss order): the slot it
+// is stored in, or -1 when it is dropped.
+__global__ void __launch_bounds__(SEL_THREADS)
+k_select_victims(MetaView mv, PolicyParams pol, uint32_t N, uint32_t tick, uint32_t epoch,
+                 const int32_t* __restrict__ miss_idx, const float* __restrict__ rq,
+                 const uint32_t* __restrict__ counts, int32_t* __restrict__ new_slot,
+                 int32_t* __restrict__ victims, unsigned long long* __restrict__ g_key,
+                 uint32_t* __restrict__ g_val, uint32_t sort_cap,
+                 unsigned long long* __restrict__ stats) {
+  __shared__ uint32_t warp_tot[32];
+  __shared__ uint32_t hist[256];
+  __shared__ unsigned long long s_key[SEL_SMEM_SORT];
+  __shared__ uint32_t s_val[SEL_SMEM_SORT];
+  __shared__ unsigned long long s_prefix;
+  __shared__ uint32_t s_need;
+
+  const uint32_t M = counts[1];
+  // 1. how many misses can be inserted at all
+  uint32_t n_ins = 0;
+  for (uint32_t base = 0; base < M; base += SEL_THREADS) {
+    const uint32_t m = base + threadIdx.x;
+    const bool ok = m < M && rq[miss_idx[m]] > 0.f;
+    uint32_t tot;
+    sel_rank(ok, warp_tot, tot);
+    n_ins += tot;
+  }
+  const uint32_t take = min(n_ins, N);
+
+  // 2. free slots, ascending
+  uint32_t n_free_taken = 0, n_free = 0;
+  for (uint32_t base = 0; base < N; base += SEL_THREADS) {
+    const uint32_t j = base + threadIdx.x;
+    const bool fr = j < N && !mv.valid[j];
+    uint32_t tot;
+    const uint32_t r = sel_rank(fr, warp_tot, tot);
+    if (fr && n_free + r < take) victims[n_free + r] = (int32_t)j;
+    n_free += tot;
+  }
+  n_free_taken = min(n_free, take);
+  const uint32_t n_evict = take - n_free_taken;     // occupied slots that must give way
+
+  if (n_evict > 0) {
+    // 3. radix select: the n_evict-th smallest key among occupied slots
+    unsigned long long prefix = 0ull;
+    uint32_t need = n_evict;                        // rank still to locate inside the current bucket
+    for (int shift = 56; shift >= 0; shift -= 8) {
+      for (uint32_t i = threadIdx.x; i < 256; i += SEL_THREADS) hist[i] = 0;
+      __syncthreads();
+      const unsigned long long hi_mask = shift == 56 ? 0ull : (~0ull << (shift + 8));
+      for (uint32_t j = threadIdx.x; j < N; j += SEL_THREADS) {
+        if (!mv.valid[j]) continue;
+        const unsigned long long key = key_of(mv, pol, j, tick, epoch);
+        if ((key & hi_mask) == prefix) atomicAdd(&hist[(uint32_t)(key >> shift) & 255u], 1u);
+      }
+      __syncthreads();
+      if (threadIdx.x == 0) {
+        uint32_t acc = 0, digit = 0;
+        for (; digit < 256; ++digit) {
+          if (acc + hist[digit] >= need) break;
+          acc += hist[digit];
+        }
+        s_prefix = prefix | ((unsigned long long)digit << shift);
+        s_need = need - acc;
+      }
+      __syncthreads();
+      prefix = s_prefix;
+      need = s_need;
+      __syncthreads();
+    }
+    const unsigned long long T = prefix;            // threshold key; `need` entries equal to T are taken
+    // 4. collect the chosen slots in slot order, then sort them by (key, slot)
+    uint32_t pow2 = 1;
+    while (pow2 < n_evict) pow2 <<= 1;
+    const bool in_smem = pow2 <= SEL_SMEM_SORT;
+    unsigned long long* skey = in_smem ? s_key : g_key;
+    uint32_t* sval = in_smem ? s_val : g_val;
+    if (!in_smem && pow2 > sort_cap) pow2 = sort_cap;   // cannot happen: sort_cap >= pow2(min(B,N))
+    uint32_t n_eq_seen = 0, n_out = 0;
+    for (uint32_t base = 0; base < N; base += SEL_THREADS) {
+      const uint32_t j = base + threadIdx.x;
+      unsigned long long key = 0ull;
+      bool occ = j < N && mv.valid[j];
+      if (occ) key = key_of(mv, pol, j, tick, epoch);
+      const bool eq = occ && key == T;
+      uint32_t tot_eq;
+      const uint32_t r_eq = sel_rank(eq, warp_tot, tot_eq);
+      const bool chosen = occ && (key < T || (eq && n_eq_seen + r_eq < need));
+      uint32_t tot_ch;
+      const uint32_t r_ch = sel_rank(chosen, warp_tot, tot_ch);
+      if (chosen && n_out + r_ch < pow2) {
+        skey[n_out + r_ch] = key;
+        sval[n_out + r_ch] = j;
+      }
+      n_eq_seen += tot_eq;
+      n_out += tot_ch;
+    }
+    for (uint32_t i = n_evict + threadIdx.x; i < pow2; i += SEL_THREADS) {
+      skey[i] = ~0ull;
+      sval[i] = 0xFFFFFFFFu;
+    }
+    bitonic_sort(skey, sval, pow2);
+    for (uint32_t i = threadIdx.x; i < n_evict; i += SEL_THREADS) victims[n_free_taken + i] = (int32_t)sval[i];
+  }
+  __syncthreads();
+
+  // 5. hand the victims to the insertable misses in miss order
+  uint32_t given = 0;
+  for (uint32_t base = 0; base < M; base += SEL_THREADS) {
+    const uint32_t m = base + threadIdx.x;
+    const bool ok = m < M && rq[miss_idx[m]] > 0.f;
+    uint32_t tot;
+    const uint32_t r = sel_rank(ok, warp_tot, tot);
+    if (m < M) new_slot[m] = (ok && given + r < take) ? victims[given + r] : -1;
+    given += tot;
+  }
+  if (threadIdx.x == 0) {
+    stats[ST_INSERT] += take;
+    stats[ST_EVICT] += n_evict;
+    stats[ST_DROP] += M - take;
+  }
+}
+
+// Flushes.  mode STALE / IDLE / ALL: one thread per slot.  SLOTS: one thread per listed slot.
+__global__ void k_evict(uint8_t* __restrict__ valid, const uint32_t* __restrict__ last_use,
+                        const uint32_t* __restrict__ insert_tick, const uint32_t* __restrict__ rate,
+                        const uint32_t* __restrict__ rate_epoch, PolicyParams pol, uint32_t N,
+                        uint32_t tick, uint32_t epoch, uint32_t mode, const int32_t* __restrict__ slots,
+                        uint32_t n_slots, uint32_t* __restrict__ n_evicted, unsigned long long* __restrict__ stats) {
+  const uint32_t i = blockIdx.x * blockDim.x + threadIdx.x;
+  bool go = false;
+  if (mode == LLMCACHE_EVICT_SLOTS) {
+    if (i < n_slots) {
+      const int32_t j = slots[i];
+      if (j >= 0 && (uint32_t)j < N) {
+        // a slot listed twice is counted once: only the thread that flips the flag counts
+        const uint32_t word = (uint32_t)j & ~3u, sh = ((uint32_t)j & 3u) * 8;
+        const uint32_t old = atomicAnd(reinterpret_cast<uint32_t*>(valid + word), ~(0xFFu << sh));
+        go = ((old >> sh) & 0xFFu) != 0;
+      }
+    }
+  } else if (i < N && valid[i]) {
+    if (mode == LLMCACHE_EVICT_ALL) go = true;
+    else if (mode == LLMCACHE_EVICT_IDLE) go = (tick - last_use[i]) > pol.max_idle;
+    else if (mode == LLMCACHE_EVICT_STALE)
+      go = pol.policy == LLMCACHE_LRU_STALENESS &&
+           rate_now(rate[i], rate_epoch[i], epoch) < pol.stale_floor && (tick - insert_tick[i]) >= pol.min_age;
+    if (go) valid[i] = 0;
+  }
+  const uint32_t bal = __ballot_sync(0xFFFFFFFFu, go);
+  if ((threadIdx.x & 31) == 0 && bal) {
+    const uint32_t c = __popc(bal);
+    if (n_evicted) atomicAdd(n_evicted, c);
+    atomicAdd(stats + ST_FLUSH, (unsigned long long)c);
+  }
+}
+
+cudaError_t launch_select_victims(llmcache_bank* bk, const llmcache_probe_io* io, uint32_t B,
+                                  int32_t* new_slot, cudaStream_t st) {
+  if (B == 0) return cudaSuccess;
+  MetaView mv{bk->a.valid, bk->a.last_use, bk->a.insert_tick, bk->a.rate, bk->a.rate_epoch};
+  const uint32_t epoch = (uint32_t)(bk->tick / bk->pol.half_life);
+  ProfScope prof(bk, LLMCACHE_K_SELECT, st);
+  k_select_victims<<<1, SEL_THREADS, 0, st>>>(mv, bk->pol, bk->desc.capacity, (uint32_t)bk->tick, epoch,
+                                              io->miss_idx, io->rq, io->counts, new_slot, bk->a.victims,
+                                              bk->a.sort_key, bk->a.sort_slot, bk->sort_len, bk->a.stats);
+  return cudaGetLastError();
+}
+
+cudaError_t launch_evict(llmcache_bank* bk, uint32_t mode, const int32_t* slots, uint32_t n,
+                         uint32_t* n_evicted, cudaStream_t st) {
+  const uint32_t N = bk->desc.capacity;
+  const uint32_t epoch = (uint32_t)(bk->tick / bk->pol.half_life);
+  if (n_evicted) {
+    cudaError_t e = cudaMemsetAsync(n_evicted, 0, sizeof(uint32_t), st);
+    if (e != cudaSuccess) return e;
+  }
+  const uint32_t work = mode == LLMCACHE_EVICT_SLOTS ? n : N;
+  if (work == 0) return cudaSuccess;
+  ProfScope prof(bk, LLMCACHE_K_EVICT, st);
+  k_evict<<<(work + 255) / 256, 256, 0, st>>>(bk->a.valid, bk->a.last_use, bk->a.insert_tick, bk->a.rate,
+                                              bk->a.rate_epoch, bk->pol, N, (uint32_t)bk->tick, epoch, mode,
+                                              slots, n, n_evicted, bk->a.stats);
+  return cudaGetLastError();
+}
+
+}  // namespace llmc

@@ -1,0 +1,156 @@
+// Internal definitions shared by the translation units of libllmcache.
+#pragma once
+#include <cuda_runtime.h>
+#include <cuda_bf16.h>
+#include <stdint.h>
+#include <stddef.h>
+#include <vector>
+#include <utility>
+#include "llmcache.h"
+
+namespace llmc {
+
+constexpr uint32_t M_CAP = (1u << 30) - 1u;   // ceiling of the decayed match rate (Q8)
+constexpr uint32_t HIT_Q8 = 256u;             // one match in Q8
+constexpr uint32_t COPY_CHUNK = 32768u;       // bytes one CTA moves per work item in row copies
+constexpr int      POOL_MAX_SPLIT = 64;
+
+// Counters kept on the device (index into Bank::d_stats).
+enum { ST_SEQ = 0, ST_HIT, ST_MISS, ST_DEGEN, ST_INSERT, ST_EVICT, ST_DROP, ST_FLUSH, ST_COUNT };
+
+struct PolicyParams {
+  uint32_t policy, half_life, stale_floor, min_age, max_idle;
+};
+
+// Device arrays of one bank.  All sub-allocations are 256-byte aligned.
+struct BankArrays {
+  __nv_bfloat16* fp;        // [N,k]
+  float*    rb;             // [N]
+  uint8_t*  valid;          // [N]
+  uint32_t* last_use;       // [N]
+  uint32_t* insert_tick;    // [N]
+  uint32_t* hits;           // [N]
+  uint32_t* rate;           // [N]
+  uint32_t* rate_epoch;     // [N]
+  __nv_bfloat16* act;       // [act_rows, n*d]
+  __nv_bfloat16* proj;      // [d,k] or nullptr
+  float*    center;         // [d] or nullptr
+  // scratch
+  float*    pool_partial;   // [max_batch, POOL_MAX_SPLIT? no: split, d]
+  unsigned long long* best; // [max_batch] packed (orderable score << 32 | ~slot); 0 = none
+  uint32_t* hitcnt;         // [N] matches per slot within the current probe (zero between calls)
+  int32_t*  victims;        // [min(max_batch,N)]
+  unsigned long long* sort_key;   // [pow2 >= min(max_batch,N)]
+  uint32_t* sort_slot;      // same length
+  unsigned long long* stats;      // [ST_COUNT]
+  uint32_t* status;         // [1] sticky device status
+  uint32_t* misc;           // [8] small per-call words
+};
+
+}  // namespace llmc
+
+struct llmcache_bank {
+  llmcache_bank_desc desc{};
+  llmc::BankArrays a{};
+  llmc::PolicyParams pol{};
+  void*    base = nullptr;  // start of the bank's device memory
+  size_t   bytes = 0;
+  bool     owns_memory = false;
+  uint64_t tick = 0;        // probe calls so far
+  uint64_t generation = 0;  // bumped by every probe
+  bool     probe_open = false;   // a probe happened and was not yet committed
+  uint32_t last_B = 0;
+  uint64_t n_probes = 0;
+  uint32_t pool_split_max = 0;   // splits the scratch is sized for
+  int      sm_count = 0;
+  uint32_t sort_len = 0;    // length of sort_key / sort_slot
+  // TMA descriptor of the fingerprint matrix (opaque 128-byte blob)
+  alignas(64) unsigned char tmap_bank[128] = {};
+  bool     has_tmap = false;
+  // instrumentation
+  uint64_t n_launches = 0;
+  bool     prof_on = false;
+  std::vector<std::pair<cudaEvent_t, cudaEvent_t>> prof_used[LLMCACHE_K_COUNT];
+  std::vector<std::pair<cudaEvent_t, cudaEvent_t>> prof_free;
+};
+
+namespace llmc {
+
+// Counts a kernel launch and, while profiling is on, brackets it with events.
+struct ProfScope {
+  llmcache_bank* bk; int kid; cudaStream_t st; cudaEvent_t stop = nullptr;
+  ProfScope(llmcache_bank* b, int k, cudaStream_t s) : bk(b), kid(k), st(s) {
+    bk->n_launches += 1;
+    if (!bk->prof_on) return;
+    std::pair<cudaEvent_t, cudaEvent_t> ev;
+    if (!bk->prof_free.empty()) { ev = bk->prof_free.back(); bk->prof_free.pop_back(); }
+    else if (cudaEventCreate(&ev.first) != cudaSuccess || cudaEventCreate(&ev.second) != cudaSuccess) return;
+    cudaEventRecord(ev.first, st);
+    stop = ev.second;
+    bk->prof_used[kid].push_back(ev);
+  }
+  ~ProfScope() { if (stop) cudaEventRecord(stop, st); }
+};
+
+// ---- launch wrappers implemented in the kernel translation units ----------
+size_t project_smem_bytes(uint32_t d, uint32_t k, bool has_proj);
+cudaError_t setup_fingerprint_kernels();
+cudaError_t setup_scan_kernels();
+uint32_t pool_split_for(uint32_t B, uint32_t n, int sm_count, uint32_t R);
+cudaError_t launch_fingerprint(llmcache_bank* bk, const void* h_in, uint32_t B,
+                               __nv_bfloat16* fp, float* rq, cudaStream_t st);
+cudaError_t launch_rownorm(llmcache_bank* bk, const __nv_bfloat16* fp, uint32_t B, uint32_t k, float* rq, cudaStream_t st);
+cudaError_t launch_scan(llmcache_bank* bk, const __nv_bfloat16* q, uint32_t B, cudaStream_t st);
+cudaError_t launch_decide(llmcache_bank* bk, uint32_t B, float tau, const float* rq,
+                          const llmcache_probe_io* io, cudaStream_t st);
+cudaError_t launch_touch(llmcache_bank* bk, cudaStream_t st);
+cudaError_t launch_gather(llmcache_bank* bk, const void* h_in, void* h_out,
+                          const llmcache_probe_io* io, uint32_t B, cudaStream_t st);
+cudaError_t launch_select_victims(llmcache_bank* bk, const llmcache_probe_io* io, uint32_t B,
+                                  int32_t* new_slot, cudaStream_t st);
+cudaError_t launch_scatter_insert(llmcache_bank* bk, const void* miss_out, const llmcache_probe_io* io,
+                                  void* h_out, const int32_t* new_slot, uint32_t B, cudaStream_t st);
+cudaError_t launch_evict(llmcache_bank* bk, uint32_t mode, const int32_t* slots, uint32_t n,
+                         uint32_t* n_evicted, cudaStream_t st);
+
+// ---- small device helpers ---------------------------------------------------
+__device__ __forceinline__ uint32_t float_orderable(float f) {
+  uint32_t u = __float_as_uint(f);
+  return (u & 0x80000000u) ? ~u : (u | 0x80000000u);
+}
+__device__ __forceinline__ float orderable_float(uint32_t o) {
+  uint32_t u = (o & 0x80000000u) ? (o & 0x7FFFFFFFu) : ~o;
+  return __uint_as_float(u);
+}
+__device__ __forceinline__ unsigned long long pack_best(float s, uint32_t slot) {
+  return ((unsigned long long)float_orderable(s) << 32) | (unsigned long long)(0xFFFFFFFFu - slot);
+}
+
+__device__ __forceinline__ uint32_t rate_now(uint32_t rate, uint32_t rate_epoch, uint32_t epoch) {
+  uint32_t sh = epoch - rate_epoch;
+  return sh > 31u ? (rate >> 31) : (rate >> sh);
+}
+
+// Eviction key of an occupied slot; smaller goes first.  Ties are broken by slot.
+__device__ __forceinline__ unsigned long long evict_key(const PolicyParams& p, uint32_t tick, uint32_t epoch,
+                                                        uint32_t rate, uint32_t rate_epoch,
+                                                        uint32_t insert_tick, uint32_t last_use) {
+  if (p.policy == LLMCACHE_LRU) return (unsigned long long)last_use;
+  uint32_t r = rate_now(rate, rate_epoch, epoch);
+  bool stale = (r < p.stale_floor) && (tick - insert_tick >= p.min_age);
+  return ((unsigned long long)(stale ? 0u : 1u) << 62) | ((unsigned long long)r << 32) | (unsigned long long)last_use;
+}
+
+// 16-byte streaming load / store (data touched once: keep it out of L1).
+__device__ __forceinline__ uint4 ld_stream16(const void* p) {
+  uint4 v;
+  asm volatile("ld.global.nc.L1::no_allocate.v4.u32 {%0,%1,%2,%3}, [%4];"
+               : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "l"(p));
+  return v;
+}
+__device__ __forceinline__ void st_stream16(void* p, uint4 v) {
+  asm volatile("st.global.L1::no_allocate.v4.u32 [%0], {%1,%2,%3,%4};"
+               :: "l"(p), "r"(v.x), "r"(v.y), "r"(v.z), "r"(v.w) : "memory");
+}
+
+}  // namespace llmc

@@ -1,0 +1,247 @@
+"""GPU-vs-oracle parity through the C ABI (element by element, same seeded inputs)."""
+import numpy as np
+import pytest
+import torch
+
+from oracle import llmcache_oracle as O
+from paper_2512_16843_b200 import binding as L
+from paper_2512_16843_b200 import synth
+from tests import parity_util as U
+
+pytestmark = pytest.mark.gpu
+DEV = "cuda"
+
+
+def make_pair(N, n, d, k, B, dtype="bf16", proj=None, center=None, **kw):
+    gb = L.Bank(capacity=N, seq_len=n, d_model=d, fp_dim=k, max_batch=B,
+                hidden_dtype=L.BF16 if dtype == "bf16" else L.F32, proj=proj, center=center, **kw)
+    ob = U.oracle_bank_like(gb, proj, center)
+    return gb, ob
+
+
+def rand_h(B, n, d, seed, dtype):
+    return synth.randn((B, n, d), seed, DEV, torch.bfloat16 if dtype == "bf16" else torch.float32)
+
+
+@pytest.mark.parametrize("dtype", ["f32", "bf16"])
+@pytest.mark.parametrize("shape", [(1, 1, 64, 1), (3, 5, 64, 7), (100, 37, 128, 33), (257, 130, 192, 65)])
+def test_small_and_ragged_shapes_lockstep(shape, dtype):
+    N, n, d, B = shape
+    gb, ob = make_pair(N, n, d, d, B, dtype)
+    bufs = L.ProbeBuffers(B, d, DEV)
+    base = rand_h(B, n, d, 11, dtype)
+    for step in range(4):
+        h = base.clone()
+        if step >= 1:                                  # half repeats (hits), half new
+            h[B // 2:] = rand_h(B - B // 2, n, d, 100 + step, dtype)
+        mo = synth.activations(B, n, d, 500 + step, DEV)
+        r = U.lockstep_step(gb, ob, bufs, h, dtype, mo)
+        if step == 0:
+            assert r["H"] == 0
+        if step >= 1 and N >= B:
+            assert r["H"] >= B // 2
+    gb.close()
+
+
+@pytest.mark.parametrize("k,use_center", [(768, False), (256, False), (256, True)])
+def test_config1_single_layer_probe(k, use_center):
+    """d_model 768, seq_len 128, fp32 hidden states, 1024 entries from 16 centres, 64 queries, tau 0.9."""
+    N, n, d, B = 1024, 128, 768, 64
+    proj = synth.projection(d, k, 77, DEV) if k != d else None
+    center = synth.randn((d,), 78, DEV, scale=0.01) if use_center else None
+    gb, ob = make_pair(N, n, d, k, B, "f32", proj, center, tau=0.9)
+    wl = synth.ClusterWorkload(16, n, d, synth.BASE_SEED + 1000, DEV)
+    bufs = L.ProbeBuffers(B, k, DEV)
+    for first in range(0, N, B):                       # warm the bank through the library itself
+        h = wl.entries(first, B)
+        gb.probe(h, bufs)
+        gb.commit(synth.activations(B, n, d, 9000 + first, DEV), bufs)
+    torch.cuda.synchronize()
+    assert gb.stats()["resident"] > 0
+    h, src = wl.queries(B, N, synth.BASE_SEED + 1001)
+    r = U.lockstep_step(gb, ob, bufs, h, "f32", synth.activations(B, n, d, 4242, DEV))
+    # by construction the 32 near queries hit (cosine ~0.9987) and the 32 fresh ones miss
+    hit = bufs.hit[:B].cpu().numpy().astype(bool)
+    assert np.array_equal(hit, (src >= 0).cpu().numpy()), r
+    assert r["near_thr"] == 0
+    gb.close()
+
+
+@pytest.mark.parametrize("policy", [L.LRU, L.LRU_STALENESS])
+def test_churn_lockstep_many_batches(policy):
+    """Drifting centres, junk that never repeats, continuous eviction (small stand-in of the churn config)."""
+    N, n, d, B = 64, 16, 128, 48
+    gb, ob = make_pair(N, n, d, d, B, "bf16", policy=policy, half_life_ticks=2, min_age_ticks=2)
+    bufs = L.ProbeBuffers(B, d, DEV)
+    centres = synth.randn((16, n, d), 5, DEV)
+    tot = dict(near_thr=0, near_tie=0, H=0, inserted=0)
+    for step in range(24):
+        centres = centres + synth.randn(centres.shape, 600 + step, DEV, scale=0.02)
+        pick = torch.randint(0, 16, (36,), generator=torch.Generator().manual_seed(step)).to(DEV)
+        near = centres[pick] + synth.randn((36, n, d), 700 + step, DEV, scale=0.05)
+        junk = synth.randn((12, n, d), 800 + step, DEV)
+        h = torch.cat([near, junk])[synth.shuffled(B, 900 + step, DEV)].to(torch.bfloat16).contiguous()
+        r = U.lockstep_step(gb, ob, bufs, h, "bf16", synth.activations(B, n, d, 1000 + step, DEV))
+        for key in tot:
+            tot[key] += r[key]
+    assert tot["H"] > 200 and tot["inserted"] > 200
+    st = gb.stats()
+    assert st["evictions"] > 0 and st["resident"] <= N
+    gb.close()
+
+
+def test_probe_fp_path_and_act_rows_aliasing():
+    N, k, B = 5000, 256, 300
+    bank_fp, q, src = synth.scan_stress(N, B, k, n_clusters=128, seed=31, device=DEV)
+    gb = L.Bank(capacity=N, seq_len=4, d_model=k, fp_dim=k, max_batch=B, act_rows=1000)
+    ob = U.oracle_bank_like(gb)
+    gb.import_(L.WHAT_FP, bank_fp)
+    gb.import_(L.WHAT_RB, torch.from_numpy(O.inv_norm_of_stored(U.bits(bank_fp))))
+    valid = torch.ones(N, dtype=torch.uint8)
+    valid[::17] = 0
+    gb.import_(L.WHAT_VALID, valid)
+    gb.import_(L.WHAT_ACT, synth.activations(1000, 4, k, 3, DEV))
+    bufs = L.ProbeBuffers(B, k, DEV)
+    r = U.lockstep_step(gb, ob, bufs, q, "bf16", None, fp_only=True, do_commit=False)
+    assert r["H"] > 30
+    with pytest.raises(L.LLMCacheError) as e:
+        gb.commit(synth.activations(B, 4, k, 4, DEV), bufs)
+    assert e.value.status == L.ERR_UNSUPPORTED
+    gb.close()
+
+
+def test_empty_batch_degenerate_rows_and_miss_input_compaction():
+    N, n, d, B = 16, 8, 64, 12
+    gb, ob = make_pair(N, n, d, d, B, "f32")
+    h_miss = torch.zeros((B, n, d), dtype=torch.float32, device=DEV)
+    bufs = L.ProbeBuffers(B, d, DEV, h_miss=h_miss)
+    gb.probe(torch.zeros((0, n, d), device=DEV), bufs, B=0)
+    gb.commit(None, bufs)
+    torch.cuda.synchronize()
+    assert bufs.counts.tolist() == [0, 0] and int(gb.export(L.WHAT_TICK)[0]) == 1
+    h = rand_h(B, n, d, 21, "f32")
+    h[2] = 0.0
+    h[5, 3, 7] = float("nan")
+    h[7, 0, 0] = float("inf")
+    mo = synth.activations(B, n, d, 22, DEV)
+    r = U.lockstep_step(gb, ob, bufs, h, "f32", mo)
+    assert r["H"] == 0 and r["inserted"] == B - 3
+    assert torch.equal(h_miss.view(torch.int32), h.view(torch.int32))          # all miss: identity compaction
+    r = U.lockstep_step(gb, ob, bufs, h, "f32", mo)
+    assert r["H"] == B - 3
+    mi = bufs.miss_idx[:3].long()
+    assert mi.tolist() == [2, 5, 7]
+    assert torch.equal(h_miss[:3].view(torch.int32), h[mi].view(torch.int32))
+    st = gb.stats()
+    assert st["degenerate"] == 6 and st["hits"] == B - 3 and st["sequences"] == 2 * B
+    gb.close()
+
+
+def test_threshold_modes_and_tau_sweep_monotone():
+    N, n, d, B = 32, 4, 64, 32
+    onehot = torch.zeros((B, n, d), device=DEV)
+    for b in range(B):
+        onehot[b, :, b] = 1.0
+    for cmp, expect in ((L.GT, 0), (L.GE, B)):
+        gb, ob = make_pair(N, n, d, d, B, "f32", cmp=cmp)
+        bufs = L.ProbeBuffers(B, d, DEV)
+        U.lockstep_step(gb, ob, bufs, onehot, "f32", synth.activations(B, n, d, 1, DEV))
+        gb.probe(onehot, bufs, tau=1.0)                 # one-hot keys score exactly 1.0
+        torch.cuda.synchronize()
+        assert int(bufs.counts[0]) == expect
+        gb.commit(synth.activations(B, n, d, 1, DEV), bufs)
+        gb.close()
+    gb, ob = make_pair(256, 8, 128, 128, 64, "bf16")
+    bufs = L.ProbeBuffers(64, 128, DEV)
+    base = rand_h(64, 8, 128, 5, "bf16")
+    U.lockstep_step(gb, ob, bufs, base, "bf16", synth.activations(64, 8, 128, 2, DEV))
+    noisy = (base.float() + 0.45 * synth.randn(base.shape, 6, DEV)).to(torch.bfloat16)
+    prev = None
+    for tau in (0.5, 0.8, 0.85, 0.9, 0.95):
+        r = U.lockstep_step(gb, ob, bufs, noisy, "bf16", None, tau=tau, do_commit=False)
+        hit = bufs.hit[:64].cpu().numpy()
+        if prev is not None:
+            assert np.all(hit <= prev)
+        prev = hit
+    assert prev.sum() < 64
+    gb.close()
+
+
+def test_evict_modes_match_oracle():
+    import copy
+    N, n, d, B = 40, 4, 64, 10
+    gb, ob = make_pair(N, n, d, d, B, "f32", half_life_ticks=2, min_age_ticks=2, max_idle_ticks=6)
+    bufs = L.ProbeBuffers(B, d, DEV)
+    items = [rand_h(B, n, d, 40 + i, "f32") for i in range(4)]
+    for i in range(4):
+        U.lockstep_step(gb, ob, bufs, items[i], "f32", synth.activations(B, n, d, i, DEV))
+    for _ in range(8):
+        U.lockstep_step(gb, ob, bufs, items[1], "f32", synth.activations(B, n, d, 9, DEV))
+    count = torch.zeros(1, dtype=torch.int32, device=DEV)
+    U.pull_state(gb, ob)
+    for mode in (L.EVICT_STALE, L.EVICT_IDLE):
+        g2 = copy.deepcopy(ob)
+        want = O.evict(g2, mode)
+        saved = gb.export(L.WHAT_VALID)
+        gb.evict(mode, count=count)
+        torch.cuda.synchronize()
+        assert int(count) == want and want > 0
+        assert np.array_equal(gb.export(L.WHAT_VALID).numpy(), g2.valid)
+        gb.import_(L.WHAT_VALID, saved)
+    slots = torch.tensor([3, 3, 11, 39, -1, 400], dtype=torch.int32, device=DEV)
+    gb.evict(L.EVICT_SLOTS, slots=slots, count=count)
+    torch.cuda.synchronize()
+    want = O.evict(ob, O.EVICT_SLOTS, [3, 3, 11, 39, -1, 400])
+    assert int(count) == want and np.array_equal(gb.export(L.WHAT_VALID).numpy(), ob.valid)
+    gb.evict(L.EVICT_ALL, count=count)
+    torch.cuda.synchronize()
+    assert int(count) == O.evict(ob, O.EVICT_ALL) and gb.stats()["resident"] == 0
+    gb.close()
+
+
+def test_call_order_and_argument_errors():
+    gb, _ = make_pair(8, 4, 64, 64, 4, "f32")
+    bufs = L.ProbeBuffers(4, 64, DEV)
+    with pytest.raises(L.LLMCacheError) as e:
+        gb.commit(synth.activations(4, 4, 64, 1, DEV), bufs)          # no probe yet
+    assert e.value.status == L.ERR_STATE
+    h = rand_h(4, 4, 64, 1, "f32")
+    gb.probe(h, bufs)
+    gb.commit(synth.activations(4, 4, 64, 1, DEV), bufs)
+    with pytest.raises(L.LLMCacheError) as e:
+        gb.commit(synth.activations(4, 4, 64, 1, DEV), bufs)          # committed twice
+    assert e.value.status == L.ERR_STATE
+    with pytest.raises(L.LLMCacheError) as e:
+        gb.probe(rand_h(5, 4, 64, 1, "f32"), bufs)                     # B > max_batch
+    assert e.value.status == L.ERR_SHAPE
+    with pytest.raises(L.LLMCacheError) as e:
+        L.llmcache_probe(gb.handle, None, 4, None, None, bufs.io)       # null input
+    assert e.value.status == L.ERR_ARG
+    with pytest.raises(L.LLMCacheError) as e:
+        L.llmcache_probe(gb.handle, h.data_ptr() + 4, 4, None, None, bufs.io)   # misaligned
+    assert e.value.status == L.ERR_ARG
+    assert gb.status() == L.OK
+    gb.close()
+
+
+def test_arena_supplied_by_caller_and_repeatability():
+    desc = L.make_desc(capacity=64, seq_len=8, d_model=64, fp_dim=64, max_batch=16, hidden_dtype=L.BF16)
+    need = L.llmcache_bank_bytes(desc)
+    arena = torch.empty(need + 256, dtype=torch.uint8, device=DEV)
+    off = (-arena.data_ptr()) % 256
+    outs = []
+    for rep in range(2):
+        gb = L.Bank(capacity=64, seq_len=8, d_model=64, fp_dim=64, max_batch=16, hidden_dtype=L.BF16,
+                    arena=arena.data_ptr() + off, arena_bytes=need)
+        bufs = L.ProbeBuffers(16, 64, DEV)
+        h = rand_h(16, 8, 64, 3, "bf16")
+        gb.probe(h, bufs)
+        gb.commit(synth.activations(16, 8, 64, 4, DEV), bufs)
+        gb.probe(h, bufs)
+        torch.cuda.synchronize()
+        outs.append((bufs.score.clone(), bufs.slot.clone(), bufs.fp.clone()))
+        gb.close()
+    assert all(torch.equal(a, b) for a, b in zip(outs[0], outs[1]))      # same bits on every run
+    with pytest.raises(L.LLMCacheError) as e:
+        L.Bank(capacity=64, seq_len=8, d_model=64, fp_dim=64, max_batch=16, arena=arena.data_ptr() + off, arena_bytes=1024)
+    assert e.value.status == L.ERR_NOMEM
