@@ -50,6 +50,9 @@ def parse():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--e2e-steps", type=int, default=3)
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--workload", default="bert_base", choices=["bert_base", "scan_stress"])
+    ap.add_argument("--bank", type=int, default=65536, help="scan_stress: number of bank entries")
+    ap.add_argument("--queries", type=int, default=65536, help="scan_stress: queries per batch")
     return ap.parse_args()
 
 
@@ -302,6 +305,65 @@ def run_ours(args):
         dist.destroy_process_group()
 
 
+def run_scan_stress(args):
+    """Bank-scan stress: d_model = fp_dim = 1024, precomputed bf16 fingerprints, top-1 + threshold 0.9."""
+    from paper_2512_16843_b200 import binding as L
+    from paper_2512_16843_b200 import synth
+    L.lib()
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device (there is no CPU fallback)")
+    dev = torch.device("cuda", 0)
+    N, B, k = args.bank, args.queries, 1024
+    keys, q, src = synth.scan_stress(N, B, k, n_clusters=4096, spread=0.1, near_fraction=0.3, q_sigma=0.05,
+                                     seed=synth.BASE_SEED + 4000, device=dev)
+    bank = L.Bank(capacity=N, seq_len=1, d_model=k, fp_dim=k, max_batch=B, store_act=0, tau=0.9)
+    bufs = L.ProbeBuffers(B, k, dev)
+    for f in range(0, N, B):                             # fill through the library: tau 2 => every key inserts
+        c = min(B, N - f)
+        bufs.fp[:c].copy_(keys[f:f + c])
+        bank.probe_fp(bufs, c, tau=2.0)
+        bank.commit(None, bufs)
+    torch.cuda.synchronize()
+    assert bank.stats()["resident"] == N
+    bufs.fp.copy_(q)
+    for _ in range(args.warmup):
+        bank.probe_fp(bufs, B)
+    torch.cuda.synchronize()
+    sampler = ClockSampler(0)
+    sampler.start()
+    bank.profile(True)
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record()
+    for _ in range(args.steps):
+        bank.probe_fp(bufs, B)
+    e1.record()
+    torch.cuda.synchronize()
+    clocks = sampler.stop()
+    ms = e0.elapsed_time(e1)
+    prof = bank.profile_read()
+    scan_ms = prof["scan"][0] / prof["scan"][1]
+    peaks, kind = measured_peaks()
+    flops = 2.0 * B * N * k
+    ach = flops / (scan_ms * 1e-3) / 1e12
+    peak = peaks["bf16_tflops_sustained"] if scan_ms * args.steps > 500 else peaks["bf16_tflops"]
+    H = int(bufs.counts[0])
+    exp_hits = int((src >= 0).sum())
+    out = {"metric": METRIC, "value": B * args.steps / (ms * 1e-3), "unit": UNIT, "n_gpus": 1, "steps": args.steps,
+           "warmup": args.warmup, "ms_per_step": ms / args.steps, "higher_is_better": True, "scaling": "weak",
+           "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
+           "config": {"workload": f"bank-scan stress: {N} keys x {B} queries x fp_dim 1024 bf16, 4096 clusters "
+                                  f"(spread 0.1), 30% near-duplicate queries, top-1 + tau 0.9, keys only",
+                      "hits": H, "expected_hits": exp_hits, "l2": "key matrix %.0f MB per scan" % (N * k * 2 / 1e6)},
+           "gpu_launches": prof["scan"][1] + prof["rownorm"][1] + prof["decide"][1] + prof["touch"][1],
+           "roofline": {"kernel": "scan", "bound": "tensor", "achieved": ach, "peak": peak, "unit": "TFLOP/s",
+                        "frac": ach / peak, "peak_kind": "of " + kind, "traffic": None, "ms_per_launch": scan_ms,
+                        "flops_per_launch": flops,
+                        "all_kernels": {n_: {"ms_per_launch": v[0] / v[1], "launches": v[1]} for n_, v in prof.items() if v[1]}},
+           "clocks": clocks}
+    print(json.dumps(out))
+    bank.close()
+
+
 def ncu_traffic(kernel):
     ent = NCU_TRAFFIC.get(kernel)
     if not ent:
@@ -400,5 +462,7 @@ if __name__ == "__main__":
     a = parse()
     if a.impl == "reference":
         run_reference(a)
+    elif a.workload == "scan_stress":
+        run_scan_stress(a)
     else:
         run_ours(a)

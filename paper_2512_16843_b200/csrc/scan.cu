@@ -1,72 +1,337 @@
 // Bank scan (Sec. III-C, Sec. IV-A): cosine of every query fingerprint against
 // every occupied slot, reduced on the fly to the best slot per query.  The
 // B x N score matrix is never written to memory.
+//
+// The scan is the dense contraction  S[b, j] = sum_c q[b, c] * f[j, c]  over bf16
+// fingerprints, both stored with the fingerprint dimension contiguous.  It runs
+// on the 5th-generation tensor cores:
+//   - one warp streams 128 x 64 query tiles and 256 x 64 key tiles into shared
+//     memory with TMA (128-byte swizzle), four stages deep;
+//   - one thread issues tcgen05.mma (M = 128 queries, N = 256 slots, K = 16 per
+//     instruction) into one of two 256-column fp32 accumulators in tensor memory;
+//   - four warps drain the other accumulator with tcgen05.ld: each thread owns
+//     one query row, scales by the slot's inverse norm, masks free slots to -inf
+//     and keeps a running (best score, lowest slot) in registers.
+// A block walks a run of key tiles for one query tile and publishes its result
+// with one 64-bit atomicMax per query (score in orderable form above, inverted
+// slot below, so that equal scores resolve to the lowest slot).
+//
+// Every wait on an mbarrier is bounded: on expiry the block records
+// LLMCACHE_ERR_TIMEOUT in the bank's status word, drains what it has in flight,
+// frees its tensor memory and returns.
+#include <cuda.h>
 #include "llmcache_internal.cuh"
 
 namespace llmc {
 
-// Straightforward CUDA-core version: a block holds QT queries in shared memory
-// (as fp32) and each thread walks one bank row.
-constexpr int SCAN_QT = 16;
-constexpr int SCAN_THREADS = 128;
+constexpr int BM = 128;            // queries per tile (MMA M)
+constexpr int BN = 256;            // slots per tile   (MMA N)
+constexpr int BK = 64;             // fingerprint elements per stage (128 bytes: one swizzle span)
+constexpr int STAGES = 4;
+constexpr int UMMA_K = 16;
+constexpr int SCAN_THREADS = 192;  // warp 0: TMA, warp 1: MMA + TMEM owner, warps 2..5: epilogue
+constexpr uint32_t A_BYTES = BM * BK * 2;   // 16 KB
+constexpr uint32_t B_BYTES = BN * BK * 2;   // 32 KB
+constexpr uint32_t TMEM_COLS = 512;         // two accumulators of 256 columns
+constexpr unsigned long long WAIT_LIMIT_NS = 2000000000ull;
 
-__global__ void __launch_bounds__(SCAN_THREADS)
-k_scan_simt(const __nv_bfloat16* __restrict__ q, const __nv_bfloat16* __restrict__ bank_fp,
-            const float* __restrict__ rb, const uint8_t* __restrict__ valid,
-            unsigned long long* __restrict__ best, uint32_t B, uint32_t N, uint32_t k) {
-  extern __shared__ float sq[];                       // [QT][k]
-  const uint32_t b0 = blockIdx.y * SCAN_QT;
-  for (uint32_t idx = threadIdx.x; idx < SCAN_QT * k; idx += blockDim.x) {
-    const uint32_t qi = idx / k, c = idx - qi * k;
-    sq[idx] = (b0 + qi < B) ? __bfloat162float(q[(size_t)(b0 + qi) * k + c]) : 0.f;
+struct ScanSmem {
+  // offsets from the 1024-byte aligned base of dynamic shared memory
+  static constexpr uint32_t A = 0;
+  static constexpr uint32_t B = A + STAGES * A_BYTES;
+  static constexpr uint32_t SB = B + STAGES * B_BYTES;          // float2 [2][BN]
+  static constexpr uint32_t BAR = SB + 2 * BN * 8;              // full[4] empty[4] tfull[2] tempty[2]
+  static constexpr uint32_t MISC = BAR + 16 * 8;                // tmem base, abort flag, epilogue go flags
+  static constexpr uint32_t TOTAL = MISC + 64;
+};
+constexpr uint32_t SCAN_SMEM_BYTES = ScanSmem::TOTAL + 1024;    // slack for manual alignment
+
+// ---- PTX wrappers -----------------------------------------------------------
+__device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
+
+__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
+  asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive(uint32_t bar) {
+  asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes) {
+  asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ unsigned long long global_ns() {
+  unsigned long long t;
+  asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
+  return t;
+}
+// Bounded wait for the phase with the given parity.  Returns false on expiry or abort.
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile uint32_t* abort_flag,
+                                          unsigned long long limit_ns = WAIT_LIMIT_NS) {
+  unsigned long long t0 = 0;
+  for (uint32_t spin = 0;; ++spin) {
+    uint32_t done;
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+        "selp.u32 %0, 1, 0, p;\n\t}"
+        : "=r"(done) : "r"(bar), "r"(parity) : "memory");
+    if (done) return true;
+    if ((spin & 255u) == 255u) {
+      if (*abort_flag) return false;
+      const unsigned long long now = global_ns();
+      if (t0 == 0) t0 = now;
+      else if (now - t0 > limit_ns) return false;
+    }
   }
+}
+__device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* map, int c0, int c1, uint32_t bar) {
+  asm volatile(
+      "cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];"
+      ::"r"(dst), "l"(map), "r"(c0), "r"(c1), "r"(bar) : "memory");
+}
+__device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void tc_commit(uint32_t bar) {
+  asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
+}
+// D[tmem] (+)= A[smem] * B[smem]^T, bf16 inputs, fp32 accumulate
+__device__ __forceinline__ void tc_mma_bf16(uint32_t d_tmem, uint64_t a_desc, uint64_t b_desc, uint32_t idesc,
+                                            uint32_t accumulate) {
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "setp.ne.b32 p, %4, 0;\n\t"
+      "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
+      ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate) : "memory");
+}
+// 32 lanes x 32 consecutive fp32 columns: thread i of the warp receives lane (base + i)
+__device__ __forceinline__ void tc_ld_32x32(uint32_t taddr, uint32_t (&v)[32]) {
+  asm volatile(
+      "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
+      "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "
+      "%16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31}, [%32];"
+      : "=r"(v[0]), "=r"(v[1]), "=r"(v[2]), "=r"(v[3]), "=r"(v[4]), "=r"(v[5]), "=r"(v[6]), "=r"(v[7]),
+        "=r"(v[8]), "=r"(v[9]), "=r"(v[10]), "=r"(v[11]), "=r"(v[12]), "=r"(v[13]), "=r"(v[14]), "=r"(v[15]),
+        "=r"(v[16]), "=r"(v[17]), "=r"(v[18]), "=r"(v[19]), "=r"(v[20]), "=r"(v[21]), "=r"(v[22]), "=r"(v[23]),
+        "=r"(v[24]), "=r"(v[25]), "=r"(v[26]), "=r"(v[27]), "=r"(v[28]), "=r"(v[29]), "=r"(v[30]), "=r"(v[31])
+      : "r"(taddr) : "memory");
+}
+__device__ __forceinline__ void tc_wait_ld() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
+
+// Shared-memory matrix descriptor of a K-major tile written by TMA with the 128-byte swizzle:
+// rows are 128 bytes apart, groups of 8 rows (1024 bytes) repeat with the stride byte offset.
+__device__ __forceinline__ uint64_t smem_desc_sw128(uint32_t saddr) {
+  return (uint64_t)((saddr & 0x3FFFFu) >> 4)      // start address, 16-byte units
+         | (1ull << 16)                           // leading byte offset (unused with swizzled K-major)
+         | ((uint64_t)(1024 >> 4) << 32)          // stride byte offset between 8-row groups
+         | (1ull << 46)                           // descriptor version of this architecture
+         | (2ull << 61);                          // 128-byte swizzle
+}
+// kind::f16 instruction descriptor: fp32 accumulator, bf16 A and B, both K-major, M = 128, N = 256.
+constexpr uint32_t IDESC = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(BN >> 3) << 17) | ((uint32_t)(BM >> 4) << 24);
+
+// ---------------------------------------------------------------------------
+__global__ void __launch_bounds__(SCAN_THREADS, 1)
+k_scan_tc(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CUtensorMap map_bank,
+          const float* __restrict__ rb, const uint8_t* __restrict__ valid,
+          unsigned long long* __restrict__ best, uint32_t* __restrict__ status,
+          uint32_t B, uint32_t N, uint32_t KB, uint32_t MB, uint32_t NB, uint32_t chunk_len, uint32_t n_units) {
+  extern __shared__ uint8_t smem_raw[];
+  const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;
+  uint8_t* gbase = smem_raw + (base - smem_u32(smem_raw));
+  const uint32_t sA = base + ScanSmem::A, sB = base + ScanSmem::B;
+  float2* sb = reinterpret_cast<float2*>(gbase + ScanSmem::SB);
+  const uint32_t bar0 = base + ScanSmem::BAR;
+  auto full_bar = [&](uint32_t s) { return bar0 + 8 * s; };
+  auto empty_bar = [&](uint32_t s) { return bar0 + 8 * (STAGES + s); };
+  auto tfull_bar = [&](uint32_t b) { return bar0 + 8 * (2 * STAGES + b); };
+  auto tempty_bar = [&](uint32_t b) { return bar0 + 8 * (2 * STAGES + 2 + b); };
+  volatile uint32_t* misc = reinterpret_cast<volatile uint32_t*>(gbase + ScanSmem::MISC);
+  volatile uint32_t* tmem_slot = misc + 0;
+  volatile uint32_t* abort_flag = misc + 1;
+  volatile uint32_t* epi_go = misc + 2;          // [2]
+
+  const uint32_t warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+
+  if (threadIdx.x == 0) {
+    for (uint32_t s = 0; s < STAGES; ++s) { mbar_init(full_bar(s), 1); mbar_init(empty_bar(s), 1); }
+    for (uint32_t b = 0; b < 2; ++b) { mbar_init(tfull_bar(b), 1); mbar_init(tempty_bar(b), 128); }
+    misc[1] = 0; misc[2] = 0; misc[3] = 0;
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+  }
+  if (warp == 1) {
+    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;"
+                 ::"r"(smem_u32((const void*)tmem_slot)), "r"(TMEM_COLS) : "memory");
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+  }
+  tc_fence_before();
   __syncthreads();
-  const uint32_t j = blockIdx.x * SCAN_THREADS + threadIdx.x;
-  float acc[SCAN_QT];
-#pragma unroll
-  for (int i = 0; i < SCAN_QT; ++i) acc[i] = 0.f;
-  const bool live = (j < N) && valid[j];
-  if (live) {
-    const uint4* row = reinterpret_cast<const uint4*>(bank_fp + (size_t)j * k);
-    for (uint32_t c8 = 0; c8 < k / 8; ++c8) {
-      const uint4 v = __ldg(row + c8);
-      const uint32_t w[4] = {v.x, v.y, v.z, v.w};
-#pragma unroll
-      for (int u = 0; u < 4; ++u) {
-        const float f0 = __uint_as_float(w[u] << 16), f1 = __uint_as_float(w[u] & 0xFFFF0000u);
-        const uint32_t c = c8 * 8 + 2 * u;
-#pragma unroll
-        for (int i = 0; i < SCAN_QT; ++i) {
-          acc[i] = fmaf(sq[i * k + c], f0, acc[i]);
-          acc[i] = fmaf(sq[i * k + c + 1], f1, acc[i]);
+  tc_fence_after();
+  const uint32_t tmem_base = *tmem_slot;
+
+  uint32_t issued = 0;                            // producer: stages armed so far
+  if (warp == 0) {
+    // ------------------------------------------------------------ TMA producer
+    if (lane == 0) {
+      bool ok = true;
+      for (uint32_t u = blockIdx.x; u < n_units && ok; u += gridDim.x) {
+        const uint32_t mb = u % MB, ch = u / MB;
+        const uint32_t nb0 = ch * chunk_len, nb1 = min(NB, nb0 + chunk_len);
+        for (uint32_t nb = nb0; nb < nb1 && ok; ++nb) {
+          for (uint32_t kb = 0; kb < KB; ++kb) {
+            const uint32_t s = issued % STAGES, ph = (issued / STAGES) & 1u;
+            if (!mbar_wait(empty_bar(s), ph ^ 1u, abort_flag)) { ok = false; break; }
+            mbar_expect_tx(full_bar(s), A_BYTES + B_BYTES);
+            tma_load_2d(sA + s * A_BYTES, &map_q, (int)(kb * BK), (int)(mb * BM), full_bar(s));
+            tma_load_2d(sB + s * B_BYTES, &map_bank, (int)(kb * BK), (int)(nb * BN), full_bar(s));
+            ++issued;
+          }
         }
       }
+      if (!ok) { *abort_flag = 1; atomicExch(status, 1u); }
+    }
+  } else if (warp == 1) {
+    // ------------------------------------------------------------ MMA issuer
+    if (lane == 0) {
+      bool ok = true;
+      uint32_t it = 0, tile = 0;
+      for (uint32_t u = blockIdx.x; u < n_units && ok; u += gridDim.x) {
+        const uint32_t ch = u / MB;
+        const uint32_t nb0 = ch * chunk_len, nb1 = min(NB, nb0 + chunk_len);
+        for (uint32_t nb = nb0; nb < nb1 && ok; ++nb, ++tile) {
+          const uint32_t buf = tile & 1u, bph = (tile >> 1) & 1u;
+          if (!mbar_wait(tempty_bar(buf), bph ^ 1u, abort_flag)) { ok = false; break; }
+          tc_fence_after();
+          const uint32_t d_tmem = tmem_base + buf * BN;
+          for (uint32_t kb = 0; kb < KB; ++kb, ++it) {
+            const uint32_t s = it % STAGES, ph = (it / STAGES) & 1u;
+            if (!mbar_wait(full_bar(s), ph, abort_flag)) { ok = false; break; }
+            tc_fence_after();
+            const uint64_t da = smem_desc_sw128(sA + s * A_BYTES), db = smem_desc_sw128(sB + s * B_BYTES);
+#pragma unroll
+            for (uint32_t kk = 0; kk < BK / UMMA_K; ++kk)
+              tc_mma_bf16(d_tmem, da + kk * (UMMA_K * 2 / 16), db + kk * (UMMA_K * 2 / 16), IDESC, (kb | kk) != 0u);
+            tc_commit(empty_bar(s));              // stage reusable once these MMAs have read it
+          }
+          if (ok) tc_commit(tfull_bar(buf));      // accumulator complete
+        }
+      }
+      if (!ok) { *abort_flag = 1; atomicExch(status, 1u); }
+    }
+  } else {
+    // ------------------------------------------------------------ epilogue (128 threads)
+    const uint32_t et = threadIdx.x - 64;         // 0..127
+    const uint32_t quarter = warp & 3u;           // TMEM lanes this warp may read
+    const uint32_t row_in_tile = quarter * 32 + lane;
+    uint32_t tile = 0;
+    bool stop = false;
+    for (uint32_t u = blockIdx.x; u < n_units && !stop; u += gridDim.x) {
+      const uint32_t mb = u % MB, ch = u / MB;
+      const uint32_t nb0 = ch * chunk_len, nb1 = min(NB, nb0 + chunk_len);
+      float best_s = -INFINITY;
+      uint32_t best_j = 0xFFFFFFFFu;
+      for (uint32_t nb = nb0; nb < nb1; ++nb, ++tile) {
+        const uint32_t buf = tile & 1u, bph = (tile >> 1) & 1u;
+        float2* sbt = sb + buf * BN;
+#pragma unroll
+        for (uint32_t x = et; x < BN; x += 128) {
+          const uint32_t j = nb * BN + x;
+          const bool live = j < N && valid[j];
+          sbt[x] = live ? make_float2(rb[j], 0.f) : make_float2(0.f, -INFINITY);
+        }
+        if (et == 0) epi_go[buf] = *abort_flag;
+        asm volatile("bar.sync 1, 128;" ::: "memory");
+        if (epi_go[buf]) { stop = true; break; }  // uniform over the 128 threads
+        if (!mbar_wait(tfull_bar(buf), bph, abort_flag)) { *abort_flag = 1; atomicExch(status, 1u); }
+        tc_fence_after();
+        const uint32_t taddr = tmem_base + buf * BN + ((quarter * 32u) << 16);
+#pragma unroll 1
+        for (uint32_t c = 0; c < BN; c += 32) {
+          uint32_t v[32];
+          tc_ld_32x32(taddr + c, v);
+          tc_wait_ld();
+          const uint32_t j0 = nb * BN + c;
+#pragma unroll
+          for (uint32_t i = 0; i < 32; ++i) {
+            const float2 w = sbt[c + i];
+            const float s = fmaf(__uint_as_float(v[i]), w.x, w.y);
+            if (s > best_s) { best_s = s; best_j = j0 + i; }
+          }
+        }
+        tc_fence_before();
+        mbar_arrive(tempty_bar(buf));
+      }
+      const uint32_t b = mb * BM + row_in_tile;
+      if (!stop && b < B && best_j != 0xFFFFFFFFu) atomicMax(best + b, pack_best(best_s, best_j));
     }
   }
-  const float scale = live ? rb[j] : 0.f;
-#pragma unroll
-  for (int i = 0; i < SCAN_QT; ++i) {
-    unsigned long long pk = live ? pack_best(acc[i] * scale, j) : 0ull;
-#pragma unroll
-    for (int o = 16; o > 0; o >>= 1) {
-      const unsigned long long other = __shfl_xor_sync(0xFFFFFFFFu, pk, o);
-      pk = other > pk ? other : pk;
+
+  // ---------------------------------------------------------------- teardown
+  tc_fence_before();
+  __syncthreads();
+  if (threadIdx.x == 0 && *abort_flag) {
+    // loads that were armed but never consumed must land before the block's shared memory is released
+    const uint32_t back = issued < (uint32_t)STAGES ? issued : (uint32_t)STAGES;
+    volatile uint32_t never = 0;
+    for (uint32_t i = 0; i < back; ++i) {
+      const uint32_t itx = issued - 1 - i;
+      mbar_wait(full_bar(itx % STAGES), (itx / STAGES) & 1u, &never, 200000000ull);
     }
-    if ((threadIdx.x & 31) == 0 && pk != 0ull && b0 + i < B) atomicMax(best + b0 + i, pk);
+  }
+  __syncthreads();
+  if (warp == 1) {
+    tc_fence_after();
+    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(TMEM_COLS) : "memory");
   }
 }
 
+// ---------------------------------------------------------------------------
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                                  const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
+                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+static EncodeTiledFn g_encode = nullptr;
+
 cudaError_t setup_scan_kernels() {
-  return cudaFuncSetAttribute(k_scan_simt, cudaFuncAttributeMaxDynamicSharedMemorySize, SCAN_QT * 2048 * 4);
+  if (!g_encode) {
+    void* fn = nullptr;
+    cudaDriverEntryPointQueryResult q;
+    cudaError_t e = cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &fn, cudaEnableDefault, &q);
+    if (e != cudaSuccess) return e;
+    if (!fn || q != cudaDriverEntryPointSuccess) return cudaErrorNotSupported;
+    g_encode = (EncodeTiledFn)fn;
+  }
+  return cudaFuncSetAttribute(k_scan_tc, cudaFuncAttributeMaxDynamicSharedMemorySize, SCAN_SMEM_BYTES);
+}
+
+// bf16 [rows, k] row-major matrix, tiles of box_rows x 64 elements, 128-byte swizzle, zero fill outside.
+static bool make_map(CUtensorMap* map, const void* ptr, uint64_t rows, uint64_t k, uint32_t box_rows) {
+  const cuuint64_t dims[2] = {k, rows};
+  const cuuint64_t strides[1] = {k * 2};
+  const cuuint32_t box[2] = {(cuuint32_t)BK, box_rows};
+  const cuuint32_t estr[2] = {1, 1};
+  return g_encode(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(ptr), dims, strides, box, estr,
+                  CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                  CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
 cudaError_t launch_scan(llmcache_bank* bk, const __nv_bfloat16* q, uint32_t B, cudaStream_t st) {
   if (B == 0) return cudaSuccess;
   const uint32_t N = bk->desc.capacity, k = bk->desc.fp_dim;
-  dim3 grid((N + SCAN_THREADS - 1) / SCAN_THREADS, (B + SCAN_QT - 1) / SCAN_QT);
+  alignas(64) CUtensorMap map_q, map_bank;
+  if (!g_encode || !make_map(&map_q, q, B, k, BM) || !make_map(&map_bank, bk->a.fp, N, k, BN))
+    return cudaErrorInvalidValue;
+  const uint32_t MB = (B + BM - 1) / BM, NB = (N + BN - 1) / BN, KB = k / BK;
+  // split the key tiles into runs so that there are a few units of work per SM when the problem allows
+  const uint32_t target = 4u * (uint32_t)bk->sm_count;
+  uint32_t chunks = (target + MB - 1) / MB;
+  if (chunks < 1) chunks = 1;
+  if (chunks > NB) chunks = NB;
+  const uint32_t chunk_len = (NB + chunks - 1) / chunks;
+  chunks = (NB + chunk_len - 1) / chunk_len;
+  const uint32_t n_units = MB * chunks;
+  const uint32_t grid = n_units < (uint32_t)bk->sm_count ? n_units : (uint32_t)bk->sm_count;
   ProfScope prof(bk, LLMCACHE_K_SCAN, st);
-  k_scan_simt<<<grid, SCAN_THREADS, (size_t)SCAN_QT * k * sizeof(float), st>>>(
-      q, bk->a.fp, bk->a.rb, bk->a.valid, bk->a.best, B, N, k);
+  k_scan_tc<<<grid, SCAN_THREADS, SCAN_SMEM_BYTES, st>>>(map_q, map_bank, bk->a.rb, bk->a.valid, bk->a.best,
+                                                        bk->a.status, B, N, KB, MB, NB, chunk_len, n_units);
   return cudaGetLastError();
 }
 

@@ -110,6 +110,33 @@ def test_probe_fp_path_and_act_rows_aliasing():
     gb.close()
 
 
+@pytest.mark.parametrize("N,k,B", [(20000, 1024, 1000), (3000, 64, 130), (70000, 128, 40), (513, 512, 257)])
+def test_scan_many_tiles_and_runs(N, k, B):
+    """Key counts and batch sizes that span many tensor-core tiles, several runs per block and ragged tails."""
+    bank_fp, q, src = synth.scan_stress(N, B, k, n_clusters=64, seed=41 + k, device=DEV)
+    gb = L.Bank(capacity=N, seq_len=2, d_model=k, fp_dim=k, max_batch=B, act_rows=512)
+    ob = U.oracle_bank_like(gb)
+    gb.import_(L.WHAT_FP, bank_fp)
+    gb.import_(L.WHAT_RB, torch.from_numpy(O.inv_norm_of_stored(U.bits(bank_fp))))
+    valid = (synth.randn((N,), 5, "cpu") > -1.0).to(torch.uint8)
+    gb.import_(L.WHAT_VALID, valid)
+    gb.import_(L.WHAT_ACT, synth.activations(512, 2, k, 3, DEV))
+    bufs = L.ProbeBuffers(B, k, DEV)
+    r = U.lockstep_step(gb, ob, bufs, q, "bf16", None, fp_only=True, do_commit=False)
+    assert r["H"] > 0 and r["M"] > 0
+    # duplicate keys: an exact tie must resolve to the lowest slot
+    dup = bank_fp.clone()
+    dup[N // 2:] = bank_fp[: N - N // 2]
+    gb.import_(L.WHAT_FP, dup)
+    gb.import_(L.WHAT_RB, torch.from_numpy(O.inv_norm_of_stored(U.bits(dup))))
+    gb.import_(L.WHAT_VALID, torch.ones(N, dtype=torch.uint8))
+    r = U.lockstep_step(gb, ob, bufs, dup[N // 2: N // 2 + B].contiguous(), "bf16", None, fp_only=True, do_commit=False)
+    assert r["near_tie"] == 0 and r["H"] == B
+    half = min(B, N // 2)
+    assert bufs.slot[:half].cpu().tolist() == list(range(half))
+    gb.close()
+
+
 def test_empty_batch_degenerate_rows_and_miss_input_compaction():
     N, n, d, B = 16, 8, 64, 12
     gb, ob = make_pair(N, n, d, d, B, "f32")
