@@ -159,6 +159,37 @@ int llmcache_bank_destroy(llmcache_bank_t* bank);
 int llmcache_fingerprint(llmcache_bank_t* bank, const void* h_in, uint32_t B,
                          void* fp, float* rq, void* stream);
 
+/* Fingerprint for callers that must not allocate device memory.  (The paper has no counterpart:
+ * this is a packaging variant of llmcache_fingerprint, same kernels, same result.)
+ *
+ * Who needs it: code that runs after its host application has handed all device memory to its own
+ * pool (an inference server that reserves the GPU at start-up, say), or inside a latency-critical
+ * loop where the device-wide stall of cudaMalloc / cudaFree is not acceptable.  Such a caller has no
+ * bank arena to spare for scratch and cannot let the library allocate one.
+ *
+ * It takes no bank.  The call runs on the CURRENT device and performs no cudaMalloc, cudaFree or other
+ * allocating call; the partial sums of the pooling pass live in one fixed array inside the library
+ * image (LLMCACHE_FINGERPRINT_STATIC_MAX_FLOATS floats = 8 MiB, held by every GPU that loads the
+ * library until the process exits).
+ *   h_in   device [B, seq_len, d_model] of hidden_dtype (LLMCACHE_F32 | LLMCACHE_BF16)
+ *   proj   device bf16 [d_model, fp_dim] or NULL (then fp_dim == d_model);  center  device f32 [d_model] or NULL
+ *   fp     device bf16 [B, fp_dim] out;  rq  device f32 [B] out
+ * Limits: same shape rules as a bank, and B * splits * d_model <= LLMCACHE_FINGERPRINT_STATIC_MAX_FLOATS,
+ * where splits <= ceil(4 * SM count / B) (<= 64) is how many slices each sequence is pooled in.  A larger
+ * call is refused with LLMCACHE_ERR_SHAPE before anything is launched; llmcache_fingerprint_static_error()
+ * then holds the sizes.
+ * The first call on each device looks up the array's device address and sets a kernel attribute; make
+ * that first call outside any stream capture.  All calls share the one array and it keeps whatever
+ * the previous call left there (nothing in it needs to start at zero: each call overwrites what it
+ * reads).  Two calls that may overlap on the GPU -- different streams, or different threads -- race
+ * on it: serialise them. */
+#define LLMCACHE_FINGERPRINT_STATIC_MAX_FLOATS (2u * 1024u * 1024u)
+int llmcache_fingerprint_static(const void* h_in, uint32_t hidden_dtype, uint32_t B, uint32_t seq_len,
+                                uint32_t d_model, uint32_t fp_dim, const void* proj, const float* center,
+                                void* fp, float* rq, void* stream);
+/* Text describing why the last llmcache_fingerprint_static call of this thread failed ("" if it did not). */
+const char* llmcache_fingerprint_static_error(void);
+
 /* Lookup and reuse for one batch (Sec. III-C, Sec. IV-A case equation,
  * Algorithm 1 "if exists (f',h') with sim > tau then h_l <- h'").
  * Advances the bank's tick.  For each sequence: fingerprint h_in[b], cosine

@@ -31,7 +31,9 @@ EXPORTS = [
     "llmcache_bank_destroy", "llmcache_fingerprint", "llmcache_probe", "llmcache_probe_fp",
     "llmcache_commit", "llmcache_evict", "llmcache_bank_export", "llmcache_bank_import",
     "llmcache_bank_stats", "llmcache_bank_status", "llmcache_bank_profile", "llmcache_bank_profile_read",
+    "llmcache_fingerprint_static", "llmcache_fingerprint_static_error",
 ]
+FINGERPRINT_STATIC_MAX_FLOATS = 2 * 1024 * 1024
 KERNEL_NAMES = ["pool", "project", "rownorm", "scan", "decide", "touch", "gather", "select", "scatter", "evict"]
 
 
@@ -99,8 +101,12 @@ def lib():
         L.llmcache_bank_status.argtypes = [vp]
         L.llmcache_bank_profile.argtypes = [vp, C.c_int]
         L.llmcache_bank_profile_read.argtypes = [vp, u32, C.POINTER(C.c_double), C.POINTER(C.c_uint64)]
+        L.llmcache_fingerprint_static.argtypes = [vp, u32, u32, u32, u32, u32, vp, vp, vp, vp, vp]
+        L.llmcache_fingerprint_static_error.restype = C.c_char_p
+        L.llmcache_fingerprint_static_error.argtypes = []
         for name in EXPORTS:
-            if name not in ("llmcache_abi_version", "llmcache_strerror", "llmcache_last_cuda_error"):
+            if name not in ("llmcache_abi_version", "llmcache_strerror", "llmcache_last_cuda_error",
+                            "llmcache_fingerprint_static_error"):
                 getattr(L, name).restype = C.c_int
         _lib = L
     return _lib
@@ -171,6 +177,19 @@ def llmcache_bank_destroy(bank: int) -> None:
 def llmcache_fingerprint(bank, h_in, B, fp, rq, stream=None) -> None:
     _check(lib().llmcache_fingerprint(bank, _ptr(h_in), B, _ptr(fp), _ptr(rq), _stream(stream)),
            "llmcache_fingerprint")
+
+
+def llmcache_fingerprint_static(h_in, hidden_dtype, B, seq_len, d_model, fp_dim, proj, center, fp, rq,
+                                stream=None) -> None:
+    """Fingerprint on the current device without a bank and without any allocation by the library
+    (for callers whose device memory is all spoken for).  Raises LLMCacheError with the library's
+    explanation when the call is refused, e.g. because the batch exceeds the fixed scratch."""
+    rc = lib().llmcache_fingerprint_static(_ptr(h_in), hidden_dtype, B, seq_len, d_model, fp_dim, _ptr(proj),
+                                           _ptr(center), _ptr(fp), _ptr(rq), _stream(stream))
+    if rc != OK:
+        err = LLMCacheError(rc, "llmcache_fingerprint_static")
+        err.args = (err.args[0] + " " + lib().llmcache_fingerprint_static_error().decode(),)
+        raise err
 
 
 def llmcache_probe(bank, h_in, B, tau, h_out, io: ProbeIO, stream=None) -> None:

@@ -255,3 +255,105 @@ cudaError_t launch_rownorm(llmcache_bank* bk, const __nv_bfloat16* fp, uint32_t 
 }
 
 }  // namespace llmc
+
+// ---------------------------------------------------------------------------
+// Fingerprint without any allocation: the pooled partial sums go to a fixed
+// array that is part of the loaded library image instead of a bank's scratch.
+// ---------------------------------------------------------------------------
+#include <mutex>
+#include <cstdio>
+
+namespace {
+
+// Partial sums of the pooling pass, [B, splits, d] floats.  8 MiB per GPU that loads the library.
+static __device__ __align__(256) float g_fp_static_scratch[LLMCACHE_FINGERPRINT_STATIC_MAX_FLOATS];
+
+constexpr int STATIC_MAX_DEVICES = 64;
+struct StaticDev { bool ready = false; float* scratch = nullptr; int sm_count = 0; };
+StaticDev g_static_dev[STATIC_MAX_DEVICES];
+std::mutex g_static_mu;
+thread_local char g_static_err[192] = "";
+
+// Once per device, with that device current: resolve the device address of the array (its name is
+// only a host-side handle) and raise the projection kernel's shared-memory limit.
+cudaError_t static_setup(int dev, StaticDev** out) {
+  std::lock_guard<std::mutex> lock(g_static_mu);
+  StaticDev& sd = g_static_dev[dev];
+  if (!sd.ready) {
+    float* ptr = nullptr;
+    cudaError_t e = cudaGetSymbolAddress((void**)&ptr, g_fp_static_scratch);
+    if (e != cudaSuccess) return e;
+    if (!ptr) return cudaErrorInvalidSymbol;
+    int sms = 0;
+    e = cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
+    if (e != cudaSuccess) return e;
+    e = llmc::setup_fingerprint_kernels();
+    if (e != cudaSuccess) return e;
+    sd.scratch = ptr;
+    sd.sm_count = sms;
+    sd.ready = true;
+  }
+  *out = &sd;
+  return cudaSuccess;
+}
+
+}  // namespace
+
+extern "C" const char* llmcache_fingerprint_static_error(void) { return g_static_err; }
+
+extern "C" int llmcache_fingerprint_static(const void* h_in, uint32_t hidden_dtype, uint32_t B, uint32_t seq_len,
+                                           uint32_t d_model, uint32_t fp_dim, const void* proj,
+                                           const float* center, void* fp, float* rq, void* stream) {
+  using namespace llmc;
+  g_static_err[0] = 0;
+  auto fail = [&](int rc, const char* msg) { std::snprintf(g_static_err, sizeof(g_static_err), "%s", msg); return rc; };
+  if (hidden_dtype != LLMCACHE_F32 && hidden_dtype != LLMCACHE_BF16) return fail(LLMCACHE_ERR_ARG, "unknown hidden_dtype");
+  if (B && (!h_in || !fp || !rq)) return fail(LLMCACHE_ERR_ARG, "null input or output pointer");
+  if (((uintptr_t)h_in | (uintptr_t)fp | (uintptr_t)proj | (uintptr_t)center) & 15u)
+    return fail(LLMCACHE_ERR_ARG, "pointers must be 16-byte aligned");
+  const bool bf16 = hidden_dtype == LLMCACHE_BF16;
+  const uint32_t d = d_model, n = seq_len, k = fp_dim;
+  if (n == 0 || d == 0 || d % 8 != 0 || d > (bf16 ? 8192u : 4096u)) return fail(LLMCACHE_ERR_SHAPE, "d_model not supported");
+  if (k == 0 || k % 64 != 0 || k > 2048 || (!proj && k != d)) return fail(LLMCACHE_ERR_SHAPE, "fp_dim not supported");
+  if (project_smem_bytes(d, k, proj != nullptr) > 200 * 1024) return fail(LLMCACHE_ERR_UNSUPPORTED, "d_model + fp_dim too large");
+  if (B == 0) return LLMCACHE_OK;
+
+  int dev = -1;
+  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= STATIC_MAX_DEVICES) {
+    cudaGetLastError();
+    return fail(LLMCACHE_ERR_CUDA, "no current CUDA device");
+  }
+  StaticDev* sd = nullptr;
+  cudaError_t e = static_setup(dev, &sd);
+  if (e != cudaSuccess) { cudaGetLastError(); return fail(LLMCACHE_ERR_CUDA, cudaGetErrorString(e)); }
+
+  const uint32_t V = bf16 ? d / 8 : d / 4;
+  uint32_t R = 512 / V; if (R < 1) R = 1;
+  if (R > n) R = n;
+  const uint32_t S = pool_split_for(B, n, sd->sm_count, R);
+  const uint32_t rows_per_slice = (n + S - 1) / S;
+  const uint32_t S_eff = (n + rows_per_slice - 1) / rows_per_slice;
+  if ((unsigned long long)B * S_eff * d > (unsigned long long)LLMCACHE_FINGERPRINT_STATIC_MAX_FLOATS) {
+    std::snprintf(g_static_err, sizeof(g_static_err),
+                  "batch too large for the fixed scratch: B * splits * d_model = %llu floats, limit %llu",
+                  (unsigned long long)B * S_eff * d, (unsigned long long)LLMCACHE_FINGERPRINT_STATIC_MAX_FLOATS);
+    return LLMCACHE_ERR_SHAPE;
+  }
+  cudaStream_t st = (cudaStream_t)stream;
+  // every partial sum that the second kernel reads is written by the first one in this call, so
+  // nothing in the shared array has to start at zero
+  dim3 grid(S_eff, B);
+  const size_t smem = (size_t)R * d * sizeof(float);
+  if (bf16)
+    k_pool<true><<<grid, V * R, smem, st>>>((const uint4*)h_in, sd->scratch, n, d, V, R, S_eff, rows_per_slice);
+  else
+    k_pool<false><<<grid, V * R, smem, st>>>((const uint4*)h_in, sd->scratch, n, d, V, R, S_eff, rows_per_slice);
+  e = cudaGetLastError();
+  if (e == cudaSuccess) {
+    k_project<<<(B + PROJ_G - 1) / PROJ_G, PROJ_THREADS, project_smem_bytes(d, k, proj != nullptr), st>>>(
+        sd->scratch, (const __nv_bfloat16*)proj, center, (__nv_bfloat16*)fp, rq, B, n, d, k, S_eff);
+    e = cudaGetLastError();
+  }
+  if (e != cudaSuccess) return fail(LLMCACHE_ERR_CUDA, cudaGetErrorString(e));
+  return LLMCACHE_OK;
+}
