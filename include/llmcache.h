@@ -131,7 +131,7 @@ enum {
   LLMCACHE_K_ROWNORM = 2,   /* inverse norms of caller-supplied fingerprints       */
   LLMCACHE_K_SCAN = 3,      /* Sec. III-C cosine scan + best slot                  */
   LLMCACHE_K_DECIDE = 4,    /* Sec. IV-A threshold + hit/miss compaction           */
-  LLMCACHE_K_TOUCH = 5,     /* Sec. III-E metadata refresh of matched slots        */
+  LLMCACHE_K_TOUCH = 5,     /* (unused: the metadata refresh runs inside DECIDE)  */
   LLMCACHE_K_GATHER = 6,    /* Algorithm 1 reuse: copy of cached outputs           */
   LLMCACHE_K_SELECT = 7,    /* Sec. IV-D victim selection                          */
   LLMCACHE_K_SCATTER = 8,   /* Algorithm 1 insert: write-back + store              */
@@ -174,10 +174,10 @@ int llmcache_fingerprint(llmcache_bank_t* bank, const void* h_in, uint32_t B,
  *   h_in   device [B, seq_len, d_model] of hidden_dtype (LLMCACHE_F32 | LLMCACHE_BF16)
  *   proj   device bf16 [d_model, fp_dim] or NULL (then fp_dim == d_model);  center  device f32 [d_model] or NULL
  *   fp     device bf16 [B, fp_dim] out;  rq  device f32 [B] out
- * Limits: same shape rules as a bank, and B * splits * d_model <= LLMCACHE_FINGERPRINT_STATIC_MAX_FLOATS,
- * where splits <= ceil(4 * SM count / B) (<= 64) is how many slices each sequence is pooled in.  A larger
- * call is refused with LLMCACHE_ERR_SHAPE before anything is launched; llmcache_fingerprint_static_error()
- * then holds the sizes.
+ * Limits: same shape rules as a bank, and the partial sums must fit: (B + 3 * G) * d_model <=
+ * LLMCACHE_FINGERPRINT_STATIC_MAX_FLOATS is always enough, where G <= min(4 * SM count, 640) is the number
+ * of blocks of the pooling pass.  A larger call is refused with LLMCACHE_ERR_SHAPE before anything is
+ * launched; llmcache_fingerprint_static_error() then holds the sizes.
  * The first call on each device looks up the array's device address and sets a kernel attribute; make
  * that first call outside any stream capture.  All calls share the one array and it keeps whatever
  * the previous call left there (nothing in it needs to start at zero: each call overwrites what it

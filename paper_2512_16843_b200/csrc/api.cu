@@ -18,7 +18,7 @@ inline uint32_t pow2_ceil(uint32_t x) { uint32_t p = 1; while (p < x) p <<= 1; r
 struct Layout {
   size_t fp, rb, valid, last_use, insert_tick, hits, rate, rate_epoch, act, proj, center;
   size_t pool_partial, best, hitcnt, victims, sort_key, sort_slot, stats, status, misc, total;
-  uint32_t split_max, sort_len;
+  uint32_t sort_len;
 };
 
 // Device guard: make the bank's device current for the duration of a call.
@@ -70,11 +70,8 @@ Layout make_layout(const llmcache_bank_desc& d) {
   L.act = take(act_rows * n * dm * 2);
   L.proj = take(d.proj ? dm * k * 2 : 0);
   L.center = take(d.center ? dm * 4 : 0);
-  // scratch: the pooled partial sums take (splits x d) floats per sequence.  The split count is
-  // ceil(4 * SMs / B) at most, so splits * B < 4 * SMs + B; 512 SMs bounds any device.
-  const size_t worst = (size_t)4 * 512 + d.max_batch;
-  L.split_max = POOL_MAX_SPLIT;
-  L.pool_partial = take(worst * dm * 4);
+  // scratch: one vector of partial sums per (pool block, sequence it touches)
+  L.pool_partial = take(((size_t)d.max_batch + 3 * POOL_MAX_GRID) * dm * 4);
   L.best = take((size_t)d.max_batch * 8);
   L.hitcnt = take(N * 4);
   const uint32_t vmax = d.max_batch < d.capacity ? d.max_batch : d.capacity;
@@ -219,7 +216,6 @@ int llmcache_bank_create(const llmcache_bank_desc* desc, llmcache_bank_t** bank_
   a.status = (uint32_t*)(base + L.status);
   a.misc = (uint32_t*)(base + L.misc);
   bk->sort_len = L.sort_len;
-  bk->pool_split_max = L.split_max;
 
   cudaError_t e = cudaSuccess;
   e = cudaMemset(base, 0, L.total);
@@ -293,7 +289,6 @@ static int probe_common(llmcache_bank_t* bk, const void* h_in, bool compute_fp, 
     else            e = launch_rownorm(bk, (const __nv_bfloat16*)io->fp, B, bk->desc.fp_dim, io->rq, st);
     if (e == cudaSuccess) e = launch_scan(bk, (const __nv_bfloat16*)io->fp, B, st);
     if (e == cudaSuccess) e = launch_decide(bk, B, tau, io->rq, io, st);
-    if (e == cudaSuccess) e = launch_touch(bk, st);
     if (e == cudaSuccess) e = launch_gather(bk, h_in, h_out, io, B, st);
   }
   if (e == cudaSuccess && io->counts_host && io->counts)

@@ -1,4 +1,4 @@
-// Threshold decision, hit/miss compaction and metadata refresh.
+// Threshold decision, hit/miss compaction and metadata refresh (one kernel).
 //   Sec. IV-A case equation / Algorithm 1: hit iff sim > tau (">=" selectable, Sec. III-C).
 //   Sec. III-E / IV-D: recency, match count and decayed match rate of matched slots.
 #include "llmcache_internal.cuh"
@@ -34,7 +34,9 @@ k_decide_compact(unsigned long long* __restrict__ best, const float* __restrict_
                  uint8_t* __restrict__ hit, int32_t* __restrict__ slot, float* __restrict__ score,
                  int32_t* __restrict__ hit_idx, int32_t* __restrict__ miss_idx,
                  uint32_t* __restrict__ counts, uint32_t* __restrict__ hitcnt,
-                 unsigned long long* __restrict__ stats) {
+                 unsigned long long* __restrict__ stats,
+                 uint32_t* __restrict__ last_use, uint32_t* __restrict__ hits_total, uint32_t* __restrict__ rate,
+                 uint32_t* __restrict__ rate_epoch, uint32_t tick, uint32_t epoch) {
   __shared__ uint32_t warp_tot[32];
   uint32_t hbase = 0, mbase = 0, ndegen = 0;
   for (uint32_t base = 0; base < B; base += DEC_THREADS) {
@@ -72,6 +74,25 @@ k_decide_compact(unsigned long long* __restrict__ best, const float* __restrict_
     hbase += nh;
     mbase += chunk - nh;
   }
+  // Metadata refresh of matched slots (Sec. III-E / IV-D).  All matches of the batch are counted by
+  // now; for each matched slot exactly one thread (the one whose exchange returns the count) applies
+  // "one decay step, + 256 per match", so the result does not depend on the order of the batch, and
+  // the counter is back at zero for the next probe.
+  __syncthreads();
+  for (uint32_t base = 0; base < B; base += DEC_THREADS) {
+    const uint32_t b = base + threadIdx.x;
+    if (b >= B) continue;
+    const int32_t j = slot[b];
+    if (j < 0) continue;
+    const uint32_t c = atomicExch(hitcnt + j, 0u);
+    if (c == 0) continue;
+    const unsigned long long m = (unsigned long long)rate_now(rate[j], rate_epoch[j], epoch) + (unsigned long long)HIT_Q8 * c;
+    rate[j] = m > M_CAP ? M_CAP : (uint32_t)m;
+    rate_epoch[j] = epoch;
+    last_use[j] = tick;
+    const unsigned long long h = (unsigned long long)hits_total[j] + c;
+    hits_total[j] = h > 0xFFFFFFFFull ? 0xFFFFFFFFu : (uint32_t)h;
+  }
   // degenerate count: block reduction by atomics on shared memory
   __shared__ uint32_t sdeg;
   if (threadIdx.x == 0) sdeg = 0;
@@ -88,39 +109,14 @@ k_decide_compact(unsigned long long* __restrict__ best, const float* __restrict_
   }
 }
 
-// Apply the matches of this probe to the slots' metadata; one thread per slot,
-// so the result does not depend on the order of the batch.
-__global__ void k_touch(uint32_t* __restrict__ hitcnt, uint32_t* __restrict__ last_use,
-                        uint32_t* __restrict__ hits, uint32_t* __restrict__ rate,
-                        uint32_t* __restrict__ rate_epoch, uint32_t N, uint32_t tick, uint32_t epoch) {
-  const uint32_t j = blockIdx.x * blockDim.x + threadIdx.x;
-  if (j >= N) return;
-  const uint32_t c = hitcnt[j];
-  if (c == 0) return;
-  hitcnt[j] = 0;
-  const unsigned long long m = (unsigned long long)rate_now(rate[j], rate_epoch[j], epoch) + (unsigned long long)HIT_Q8 * c;
-  rate[j] = m > M_CAP ? M_CAP : (uint32_t)m;
-  rate_epoch[j] = epoch;
-  last_use[j] = tick;
-  const unsigned long long h = (unsigned long long)hits[j] + c;
-  hits[j] = h > 0xFFFFFFFFull ? 0xFFFFFFFFu : (uint32_t)h;
-}
-
 cudaError_t launch_decide(llmcache_bank* bk, uint32_t B, float tau, const float* rq,
                           const llmcache_probe_io* io, cudaStream_t st) {
   ProfScope prof(bk, LLMCACHE_K_DECIDE, st);
   k_decide_compact<<<1, DEC_THREADS, 0, st>>>(bk->a.best, rq, B, tau, bk->desc.cmp == LLMCACHE_GE,
                                               io->hit, io->slot, io->score, io->hit_idx, io->miss_idx,
-                                              io->counts, bk->a.hitcnt, bk->a.stats);
-  return cudaGetLastError();
-}
-
-cudaError_t launch_touch(llmcache_bank* bk, cudaStream_t st) {
-  const uint32_t N = bk->desc.capacity;
-  const uint32_t epoch = (uint32_t)(bk->tick / bk->pol.half_life);
-  ProfScope prof(bk, LLMCACHE_K_TOUCH, st);
-  k_touch<<<(N + 255) / 256, 256, 0, st>>>(bk->a.hitcnt, bk->a.last_use, bk->a.hits, bk->a.rate,
-                                           bk->a.rate_epoch, N, (uint32_t)bk->tick, epoch);
+                                              io->counts, bk->a.hitcnt, bk->a.stats,
+                                              bk->a.last_use, bk->a.hits, bk->a.rate, bk->a.rate_epoch,
+                                              (uint32_t)bk->tick, (uint32_t)(bk->tick / bk->pol.half_life));
   return cudaGetLastError();
 }
 

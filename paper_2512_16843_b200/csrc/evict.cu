@@ -5,9 +5,10 @@
 
 namespace llmc {
 
-constexpr int SEL_THREADS = 1024;
-constexpr uint32_t SEL_SMEM_SORT = 2048;      // sort in shared memory up to this many candidates
+constexpr int SEL_THREADS = 512;
+constexpr uint32_t SEL_SMEM = 2048;            // candidates / cached keys kept in shared memory
 
+// Exclusive rank of `pred` among the threads of the block (in thread order) and the block total.
 __device__ __forceinline__ uint32_t sel_rank(bool pred, uint32_t* warp_tot, uint32_t& total) {
   const uint32_t lane = threadIdx.x & 31, w = threadIdx.x >> 5;
   const uint32_t bal = __ballot_sync(0xFFFFFFFFu, pred);
@@ -16,6 +17,7 @@ __device__ __forceinline__ uint32_t sel_rank(bool pred, uint32_t* warp_tot, uint
   if (lane == 0) warp_tot[w] = __popc(bal);
   __syncthreads();
   uint32_t before = 0, tot = 0;
+#pragma unroll
   for (uint32_t i = 0; i < (SEL_THREADS >> 5); ++i) {
     const uint32_t c = warp_tot[i];
     if (i < w) before += c;
@@ -30,37 +32,49 @@ struct MetaView {
   const uint32_t *last_use, *insert_tick, *rate, *rate_epoch;
 };
 
-__device__ __forceinline__ unsigned long long key_of(const MetaView& mv, const PolicyParams& p,
-                                                     uint32_t j, uint32_t tick, uint32_t epoch) {
-  return evict_key(p, tick, epoch, mv.rate[j], mv.rate_epoch[j], mv.insert_tick[j], mv.last_use[j]);
+// Order in which slots are taken: free slots first (key 0), then occupied slots by ascending eviction
+// key (bit 63 set, which no eviction key has); ties go to the lower slot.  All loads are issued
+// unconditionally so that they overlap.
+__device__ __forceinline__ unsigned long long take_key(const MetaView& mv, const PolicyParams& p,
+                                                       uint32_t j, uint32_t tick, uint32_t epoch) {
+  const uint8_t v = mv.valid[j];
+  const uint32_t r = mv.rate[j], re = mv.rate_epoch[j], it = mv.insert_tick[j], lu = mv.last_use[j];
+  return v ? (evict_key(p, tick, epoch, r, re, it, lu) | (1ull << 63)) : 0ull;
 }
 
-// In-place bitonic sort of (key, slot) pairs, ascending by key then slot.
-// len is a power of two; the arrays may live in shared or global memory.
+// In-place bitonic sort of (key, slot) pairs, ascending by key then slot.  len is a power of two;
+// the arrays may live in shared or global memory.  Thread t handles the pair (i, i + stride) with
+// i = (t / stride) * 2 * stride + t % stride, so for stride <= 32 a warp only touches elements that
+// no other warp touches in that step and a warp-level sync is enough.
 __device__ void bitonic_sort(unsigned long long* key, uint32_t* val, uint32_t len) {
+  __syncthreads();
   for (uint32_t size = 2; size <= len; size <<= 1) {
-    for (uint32_t stride = size >> 1; stride > 0; stride >>= 1) {
-      __syncthreads();
-      for (uint32_t i = threadIdx.x; i < len; i += SEL_THREADS) {
-        const uint32_t l = i ^ stride;
-        if (l > i) {
-          const unsigned long long ka = key[i], kb = key[l];
-          const uint32_t va = val[i], vb = val[l];
-          const bool a_gt_b = (ka > kb) || (ka == kb && va > vb);
-          const bool ascending = (i & size) == 0;
-          if (a_gt_b == ascending) {
-            key[i] = kb; key[l] = ka;
-            val[i] = vb; val[l] = va;
-          }
+    for (uint32_t stride = size >> 1, lg = 31 - __clz(stride);; stride >>= 1, --lg) {
+      for (uint32_t t = threadIdx.x; t < (len >> 1); t += SEL_THREADS) {
+        const uint32_t i = ((t >> lg) << (lg + 1)) | (t & (stride - 1)), l = i + stride;
+        const unsigned long long ka = key[i], kb = key[l];
+        const uint32_t va = val[i], vb = val[l];
+        const bool a_gt_b = (ka > kb) || (ka == kb && va > vb);
+        const bool ascending = (i & size) == 0;
+        if (a_gt_b == ascending) {
+          key[i] = kb; key[l] = ka;
+          val[i] = vb; val[l] = va;
         }
       }
+      // a step with stride <= 32 stays inside the warp's own 64 elements; a block-level sync is only
+      // needed when this step or the next one reaches further
+      const uint32_t next = stride > 1 ? (stride >> 1) : size;
+      if (stride > 32 || next > 32) __syncthreads(); else __syncwarp();
+      if (stride == 1) break;
     }
   }
   __syncthreads();
 }
 
-// One block.  Output: new_slot[m] for every miss m (in miss order): the slot it
-// is stored in, or -1 when it is dropped.
+// One block.  Output: new_slot[m] for every miss m (in miss order): the slot it is stored in, or -1
+// when it is dropped.  The `take` slots that come first in the taking order are found with a radix
+// select over the 64-bit keys (bytes on which all keys agree are skipped), gathered in slot order,
+// sorted, and handed to the insertable misses in miss order.
 __global__ void __launch_bounds__(SEL_THREADS)
 k_select_victims(MetaView mv, PolicyParams pol, uint32_t N, uint32_t tick, uint32_t epoch,
                  const int32_t* __restrict__ miss_idx, const float* __restrict__ rq,
@@ -70,101 +84,128 @@ k_select_victims(MetaView mv, PolicyParams pol, uint32_t N, uint32_t tick, uint3
                  unsigned long long* __restrict__ stats) {
   __shared__ uint32_t warp_tot[32];
   __shared__ uint32_t hist[256];
-  __shared__ unsigned long long s_key[SEL_SMEM_SORT];
-  __shared__ uint32_t s_val[SEL_SMEM_SORT];
-  __shared__ unsigned long long s_prefix;
-  __shared__ uint32_t s_need;
+  __shared__ unsigned long long s_cache[SEL_SMEM];   // keys of all slots when N <= SEL_SMEM
+  __shared__ unsigned long long s_key[SEL_SMEM];     // chosen candidates
+  __shared__ uint32_t s_val[SEL_SMEM];
+  __shared__ unsigned long long s_and, s_or, s_prefix;
+  __shared__ uint32_t s_need, s_evict;
 
   const uint32_t M = counts[1];
-  // 1. how many misses can be inserted at all
+  const bool cached = N <= SEL_SMEM;
+  auto key_at = [&](uint32_t j) -> unsigned long long {
+    return cached ? s_cache[j] : take_key(mv, pol, j, tick, epoch);
+  };
+  if (threadIdx.x == 0) { s_and = ~0ull; s_or = 0ull; s_evict = 0; }
+  __syncthreads();
+
+  // keys of all slots; bitwise AND / OR over them tells which bytes differ at all
+  {
+    unsigned long long a = ~0ull, o = 0ull;
+    for (uint32_t j = threadIdx.x; j < N; j += SEL_THREADS) {
+      const unsigned long long key = take_key(mv, pol, j, tick, epoch);
+      if (cached) s_cache[j] = key;
+      a &= key; o |= key;
+    }
+#pragma unroll
+    for (int off = 16; off > 0; off >>= 1) {
+      a &= __shfl_xor_sync(0xFFFFFFFFu, a, off);
+      o |= __shfl_xor_sync(0xFFFFFFFFu, o, off);
+    }
+    if ((threadIdx.x & 31) == 0) { atomicAnd(&s_and, a); atomicOr(&s_or, o); }
+  }
+  // how many misses can be inserted at all
   uint32_t n_ins = 0;
   for (uint32_t base = 0; base < M; base += SEL_THREADS) {
     const uint32_t m = base + threadIdx.x;
     const bool ok = m < M && rq[miss_idx[m]] > 0.f;
-    uint32_t tot;
-    sel_rank(ok, warp_tot, tot);
-    n_ins += tot;
+    n_ins += (uint32_t)__syncthreads_count(ok);
   }
+  __syncthreads();
   const uint32_t take = min(n_ins, N);
+  const unsigned long long differ = s_and ^ s_or;
 
-  // 2. free slots, ascending
-  uint32_t n_free_taken = 0, n_free = 0;
-  for (uint32_t base = 0; base < N; base += SEL_THREADS) {
-    const uint32_t j = base + threadIdx.x;
-    const bool fr = j < N && !mv.valid[j];
-    uint32_t tot;
-    const uint32_t r = sel_rank(fr, warp_tot, tot);
-    if (fr && n_free + r < take) victims[n_free + r] = (int32_t)j;
-    n_free += tot;
-  }
-  n_free_taken = min(n_free, take);
-  const uint32_t n_evict = take - n_free_taken;     // occupied slots that must give way
-
-  if (n_evict > 0) {
-    // 3. radix select: the n_evict-th smallest key among occupied slots
+  if (take > 0) {
+    // radix select, most significant byte first: the take-th key in taking order
     unsigned long long prefix = 0ull;
-    uint32_t need = n_evict;                        // rank still to locate inside the current bucket
+    uint32_t need = take;                            // rank still to locate inside the current bucket
     for (int shift = 56; shift >= 0; shift -= 8) {
+      if (((differ >> shift) & 0xFFull) == 0ull) {   // every key has the same byte here
+        prefix |= s_and & (0xFFull << shift);
+        continue;
+      }
       for (uint32_t i = threadIdx.x; i < 256; i += SEL_THREADS) hist[i] = 0;
       __syncthreads();
       const unsigned long long hi_mask = shift == 56 ? 0ull : (~0ull << (shift + 8));
       for (uint32_t j = threadIdx.x; j < N; j += SEL_THREADS) {
-        if (!mv.valid[j]) continue;
-        const unsigned long long key = key_of(mv, pol, j, tick, epoch);
+        const unsigned long long key = key_at(j);
         if ((key & hi_mask) == prefix) atomicAdd(&hist[(uint32_t)(key >> shift) & 255u], 1u);
       }
       __syncthreads();
-      if (threadIdx.x == 0) {
-        uint32_t acc = 0, digit = 0;
-        for (; digit < 256; ++digit) {
-          if (acc + hist[digit] >= need) break;
-          acc += hist[digit];
+      if (threadIdx.x < 32) {
+        // warp 0 finds the bin that holds the need-th candidate: each lane sums 8 bins, an inclusive
+        // scan over the lanes locates the lane, the lane walks its 8 bins
+        const uint32_t lane = threadIdx.x;
+        uint32_t mine = 0;
+#pragma unroll
+        for (int i = 0; i < 8; ++i) mine += hist[lane * 8 + i];
+        uint32_t incl = mine;
+#pragma unroll
+        for (int o = 1; o < 32; o <<= 1) {
+          const uint32_t t = __shfl_up_sync(0xFFFFFFFFu, incl, o);
+          if (lane >= (uint32_t)o) incl += t;
         }
-        s_prefix = prefix | ((unsigned long long)digit << shift);
-        s_need = need - acc;
+        const uint32_t excl = incl - mine;
+        if (excl < need && need <= incl) {           // exactly one lane
+          uint32_t acc = excl, digit = lane * 8;
+          for (int i = 0; i < 8; ++i, ++digit) {
+            if (acc + hist[digit] >= need) break;
+            acc += hist[digit];
+          }
+          s_prefix = prefix | ((unsigned long long)digit << shift);
+          s_need = need - acc;
+        }
       }
       __syncthreads();
       prefix = s_prefix;
       need = s_need;
-      __syncthreads();
     }
-    const unsigned long long T = prefix;            // threshold key; `need` entries equal to T are taken
-    // 4. collect the chosen slots in slot order, then sort them by (key, slot)
+    const unsigned long long T = prefix;             // threshold key; `need` slots equal to T are taken
+    // collect the chosen slots in slot order, then sort them by (key, slot)
     uint32_t pow2 = 1;
-    while (pow2 < n_evict) pow2 <<= 1;
-    const bool in_smem = pow2 <= SEL_SMEM_SORT;
+    while (pow2 < take) pow2 <<= 1;
+    const bool in_smem = pow2 <= SEL_SMEM;
     unsigned long long* skey = in_smem ? s_key : g_key;
     uint32_t* sval = in_smem ? s_val : g_val;
-    if (!in_smem && pow2 > sort_cap) pow2 = sort_cap;   // cannot happen: sort_cap >= pow2(min(B,N))
-    uint32_t n_eq_seen = 0, n_out = 0;
+    if (!in_smem && pow2 > sort_cap) pow2 = sort_cap;   // cannot happen: sort_cap >= pow2(min(B, N))
+    uint32_t n_eq_seen = 0, n_out = 0, n_occ = 0;
     for (uint32_t base = 0; base < N; base += SEL_THREADS) {
       const uint32_t j = base + threadIdx.x;
-      unsigned long long key = 0ull;
-      bool occ = j < N && mv.valid[j];
-      if (occ) key = key_of(mv, pol, j, tick, epoch);
-      const bool eq = occ && key == T;
+      const unsigned long long key = j < N ? key_at(j) : ~0ull;
+      const bool eq = j < N && key == T;
       uint32_t tot_eq;
       const uint32_t r_eq = sel_rank(eq, warp_tot, tot_eq);
-      const bool chosen = occ && (key < T || (eq && n_eq_seen + r_eq < need));
+      const bool chosen = j < N && (key < T || (eq && n_eq_seen + r_eq < need));
       uint32_t tot_ch;
       const uint32_t r_ch = sel_rank(chosen, warp_tot, tot_ch);
       if (chosen && n_out + r_ch < pow2) {
         skey[n_out + r_ch] = key;
         sval[n_out + r_ch] = j;
+        if (key >> 63) ++n_occ;
       }
       n_eq_seen += tot_eq;
       n_out += tot_ch;
     }
-    for (uint32_t i = n_evict + threadIdx.x; i < pow2; i += SEL_THREADS) {
+    if (n_occ) atomicAdd(&s_evict, n_occ);
+    for (uint32_t i = take + threadIdx.x; i < pow2; i += SEL_THREADS) {
       skey[i] = ~0ull;
       sval[i] = 0xFFFFFFFFu;
     }
     bitonic_sort(skey, sval, pow2);
-    for (uint32_t i = threadIdx.x; i < n_evict; i += SEL_THREADS) victims[n_free_taken + i] = (int32_t)sval[i];
+    for (uint32_t i = threadIdx.x; i < take; i += SEL_THREADS) victims[i] = (int32_t)sval[i];
   }
   __syncthreads();
 
-  // 5. hand the victims to the insertable misses in miss order
+  // hand the victims to the insertable misses in miss order
   uint32_t given = 0;
   for (uint32_t base = 0; base < M; base += SEL_THREADS) {
     const uint32_t m = base + threadIdx.x;
@@ -176,7 +217,7 @@ k_select_victims(MetaView mv, PolicyParams pol, uint32_t N, uint32_t tick, uint3
   }
   if (threadIdx.x == 0) {
     stats[ST_INSERT] += take;
-    stats[ST_EVICT] += n_evict;
+    stats[ST_EVICT] += s_evict;
     stats[ST_DROP] += M - take;
   }
 }

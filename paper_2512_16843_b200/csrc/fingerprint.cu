@@ -5,28 +5,32 @@
 namespace llmc {
 
 // ---------------------------------------------------------------------------
-// Pool: partial[b, s, :] = sum over the s-th slice of positions of h[b, t, :].
-// grid (S, B).  A block is V x R threads: V = 16-byte vectors per row, R = rows
-// taken per pass.  Every thread always owns the same E columns, so the running
-// sums live in registers; the R row groups are combined through shared memory
-// in a fixed order (deterministic).
+// Pool.  The B*n rows of the batch are one flat list that is cut into equal
+// spans, one per block, so that every block streams the same number of bytes
+// and the grid is a single wave.  A span may cross sequence boundaries: a block
+// writes one vector of partial sums per sequence it touches,
+//     partial[(block * Jmax + j), :] = sum of its rows of the j-th sequence it touches.
+// A block is V x R threads (rounded up to whole warps): V = 16-byte vectors per
+// row, R = rows taken per pass.  Every thread always owns the same E columns, so
+// the running sums live in registers; the R row groups are combined through
+// shared memory in a fixed order (deterministic).
 // ---------------------------------------------------------------------------
 template <bool BF16>
-__global__ void __launch_bounds__(1024)
+__global__ void __launch_bounds__(1024, 1)
 k_pool(const uint4* __restrict__ h, float* __restrict__ partial,
-       uint32_t n, uint32_t d, uint32_t V, uint32_t R, uint32_t S, uint32_t rows_per_slice) {
+       uint32_t B, uint32_t n, uint32_t d, uint32_t V, uint32_t R, uint32_t L, uint32_t Jmax) {
   constexpr int E = BF16 ? 8 : 4;
   extern __shared__ float sm_pool[];           // [R][d]
-  const uint32_t b = blockIdx.y, s = blockIdx.x;
+  const bool active = threadIdx.x < V * R;
   const uint32_t col = threadIdx.x % V, rg = threadIdx.x / V;
-  const uint32_t t0 = s * rows_per_slice;
-  const uint32_t t1 = min(n, t0 + rows_per_slice);
-  float acc[E];
-#pragma unroll
-  for (int e = 0; e < E; ++e) acc[e] = 0.f;
+  const unsigned long long total = (unsigned long long)B * n;
+  unsigned long long r0 = (unsigned long long)blockIdx.x * L;
+  unsigned long long r1 = r0 + L;
+  if (r1 > total) r1 = total;
+  uint32_t b = (uint32_t)(r0 / n);
+  float* out = partial + (size_t)blockIdx.x * Jmax * d;
 
-  const uint4* base = h + (size_t)b * n * V + col;
-  auto add = [&](const uint4& v) {
+  auto add = [](float (&acc)[E], const uint4& v) {
     if (BF16) {
       const uint32_t w[4] = {v.x, v.y, v.z, v.w};
 #pragma unroll
@@ -39,38 +43,55 @@ k_pool(const uint4* __restrict__ h, float* __restrict__ partial,
       acc[2] += __uint_as_float(v.z); acc[3] += __uint_as_float(v.w);
     }
   };
-  uint32_t t = t0 + rg;
-  // four rows in flight per thread
-  for (; t + 3 * R < t1; t += 4 * R) {
-    uint4 v0 = ld_stream16(base + (size_t)t * V);
-    uint4 v1 = ld_stream16(base + (size_t)(t + R) * V);
-    uint4 v2 = ld_stream16(base + (size_t)(t + 2 * R) * V);
-    uint4 v3 = ld_stream16(base + (size_t)(t + 3 * R) * V);
-    add(v0); add(v1); add(v2); add(v3);
-  }
-  for (; t < t1; t += R) add(ld_stream16(base + (size_t)t * V));
 
+  while (r0 < r1) {
+    unsigned long long seg_end = (unsigned long long)(b + 1) * n;
+    if (seg_end > r1) seg_end = r1;
+    float acc[E];
 #pragma unroll
-  for (int e = 0; e < E; ++e) sm_pool[(size_t)rg * d + col * E + e] = acc[e];
-  __syncthreads();
-  float* out = partial + ((size_t)b * S + s) * d;
-  for (uint32_t i = threadIdx.x; i < d; i += blockDim.x) {
-    float sum = 0.f;
-    for (uint32_t r = 0; r < R; ++r) sum += sm_pool[(size_t)r * d + i];
-    out[i] = sum;
+    for (int e = 0; e < E; ++e) acc[e] = 0.f;
+    if (active) {
+      const uint4* base = h + col;
+      unsigned long long t = r0 + rg;
+      for (; t + 3ull * R < seg_end; t += 4ull * R) {        // four rows in flight per thread
+        const uint4 v0 = ld_stream16(base + t * V);
+        const uint4 v1 = ld_stream16(base + (t + R) * V);
+        const uint4 v2 = ld_stream16(base + (t + 2ull * R) * V);
+        const uint4 v3 = ld_stream16(base + (t + 3ull * R) * V);
+        add(acc, v0); add(acc, v1); add(acc, v2); add(acc, v3);
+      }
+      for (; t < seg_end; t += R) add(acc, ld_stream16(base + t * V));
+#pragma unroll
+      for (int e = 0; e < E; ++e) sm_pool[(size_t)rg * d + col * E + e] = acc[e];
+    }
+    __syncthreads();
+    for (uint32_t i = threadIdx.x; i < d; i += blockDim.x) {
+      float sum = 0.f;
+      for (uint32_t r = 0; r < R; ++r) sum += sm_pool[(size_t)r * d + i];
+      out[i] = sum;
+    }
+    __syncthreads();
+    out += d;
+    r0 = seg_end;
+    ++b;
   }
 }
 
 // ---------------------------------------------------------------------------
-// Project + normalise: G sequences per block.
-//   p = (sum_s partial) / n - mu ;  g = p . P  (or p when no projection)
+// Project + normalise: G sequences per block, 128 threads per sequence in the
+// element-wise phases.
+//   p = (sum of the sequence's partial vectors) / n - mu ;  g = p . P  (or p when no projection)
 //   q = bf16(g / ||g||) ; rq = 1 / ||q||
+// P is read with 16-byte loads: a thread owns 8 adjacent output columns and
+// every `slices`-th row; the row slices are combined through shared memory in a
+// fixed order.
 // ---------------------------------------------------------------------------
-constexpr int PROJ_G = 4;
-constexpr int PROJ_THREADS = 512;
+constexpr int PROJ_G = 2;
+constexpr int PROJ_THREADS = 1024;
+constexpr int PROJ_TPS = PROJ_THREADS / PROJ_G;      // threads per sequence
 
-__device__ __forceinline__ float block_sum(float v, float* red /*[32]*/) {
-  // fixed-order tree: lanes by shuffle, then warps serially by thread 0
+// Sum over the TPS threads that serve one sequence (fixed order).  red: [PROJ_THREADS / 32] floats.
+__device__ __forceinline__ float group_sum(float v, float* red, int group) {
 #pragma unroll
   for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xFFFFFFFFu, v, o);
   const int w = threadIdx.x >> 5, l = threadIdx.x & 31;
@@ -78,67 +99,90 @@ __device__ __forceinline__ float block_sum(float v, float* red /*[32]*/) {
   if (l == 0) red[w] = v;
   __syncthreads();
   float tot = 0.f;
-  const int nw = (blockDim.x + 31) >> 5;
-  for (int i = 0; i < nw; ++i) tot += red[i];
+  constexpr int WPG = PROJ_TPS / 32;
+#pragma unroll
+  for (int i = 0; i < WPG; ++i) tot += red[group * WPG + i];
   return tot;
 }
 
 __global__ void __launch_bounds__(PROJ_THREADS)
 k_project(const float* __restrict__ partial, const __nv_bfloat16* __restrict__ proj,
           const float* __restrict__ center, __nv_bfloat16* __restrict__ fp, float* __restrict__ rq,
-          uint32_t B, uint32_t n, uint32_t d, uint32_t k, uint32_t S) {
+          uint32_t B, uint32_t n, uint32_t d, uint32_t k, uint32_t L, uint32_t Jmax) {
   extern __shared__ float sm[];
   float* p = sm;                               // [G][d]
-  float* g = p + (size_t)PROJ_G * d;           // [G][k]
-  float* part = g + (size_t)PROJ_G * k;        // [slices][G][k]  (only with projection)
-  __shared__ float red[32];
+  float* g = p + (size_t)PROJ_G * d;           // [G][k]            (only with projection)
+  float* part = g + (size_t)PROJ_G * k;        // [slices][G][k]    (only with projection)
+  __shared__ float red[PROJ_THREADS / 32];
   const uint32_t b0 = blockIdx.x * PROJ_G;
   const float fn = (float)n;
+  const int grp = threadIdx.x / PROJ_TPS;      // sequence served in the element-wise phases
+  const uint32_t gt = threadIdx.x % PROJ_TPS;
+  const uint32_t bq = b0 + grp;
 
-  for (uint32_t idx = threadIdx.x; idx < PROJ_G * d; idx += blockDim.x) {
-    const uint32_t gi = idx / d, i = idx - gi * d;
-    const uint32_t b = b0 + gi;
-    float v = 0.f;
-    if (b < B) {
-      const float* src = partial + (size_t)b * S * d + i;
-      for (uint32_t s = 0; s < S; ++s) v += src[(size_t)s * d];
-      v = v / fn;
-      if (center) v -= center[i];
+  {
+    // pool blocks whose span overlaps rows [b*n, (b+1)*n), in block order
+    float* pg = p + (size_t)grp * d;
+    if (bq < B) {
+      const unsigned long long first = (unsigned long long)bq * n, last = first + n - 1;
+      const uint32_t c_lo = (uint32_t)(first / L), c_hi = (uint32_t)(last / L);
+      const uint32_t j_lo = bq - (uint32_t)(((unsigned long long)c_lo * L) / n);
+      for (uint32_t i = gt; i < d; i += PROJ_TPS) {
+        // the first block may have touched earlier sequences (index j_lo); later blocks start inside bq
+        float v = partial[((size_t)c_lo * Jmax + j_lo) * d + i];
+        for (uint32_t c = c_lo + 1; c <= c_hi; ++c) v += partial[(size_t)c * Jmax * d + i];
+        v = v / fn;
+        if (center) v -= center[i];
+        pg[i] = v;
+      }
+    } else {
+      for (uint32_t i = gt; i < d; i += PROJ_TPS) pg[i] = 0.f;
     }
-    p[idx] = v;
   }
   __syncthreads();
 
   if (proj) {
-    const uint32_t ncol2 = k >> 1;
-    const uint32_t slices = ncol2 >= blockDim.x ? 1u : blockDim.x / ncol2;
-    const uint32_t active = ncol2 >= blockDim.x ? blockDim.x : slices * ncol2;
-    if (threadIdx.x < active) {
-      const uint32_t sl = ncol2 >= blockDim.x ? 0u : threadIdx.x / ncol2;
-      const uint32_t c2_0 = ncol2 >= blockDim.x ? threadIdx.x : threadIdx.x % ncol2;
-      const uint32_t dper = (d + slices - 1) / slices;
-      const uint32_t i0 = sl * dper, i1 = min(d, i0 + dper);
-      for (uint32_t c2 = c2_0; c2 < ncol2; c2 += (ncol2 >= blockDim.x ? blockDim.x : ncol2)) {
-        float a0[PROJ_G], a1[PROJ_G];
+    const uint32_t ncg = k >> 3;                                   // groups of 8 columns
+    const uint32_t slices = ncg >= blockDim.x ? 1u : blockDim.x / ncg;
+    const uint4* P4 = reinterpret_cast<const uint4*>(proj);
+    for (uint32_t cg0 = 0; cg0 < ncg; cg0 += blockDim.x) {         // one trip unless k > 8 * threads
+      const uint32_t cg = cg0 + (ncg >= blockDim.x ? threadIdx.x : threadIdx.x % ncg);
+      const uint32_t sl = ncg >= blockDim.x ? 0u : threadIdx.x / ncg;
+      if (cg < ncg && sl < slices) {
+        float acc[PROJ_G][8];
 #pragma unroll
-        for (int gi = 0; gi < PROJ_G; ++gi) { a0[gi] = 0.f; a1[gi] = 0.f; }
-        const uint32_t* col = reinterpret_cast<const uint32_t*>(proj) + c2;
-#pragma unroll 8
-        for (uint32_t i = i0; i < i1; ++i) {
-          const uint32_t w = __ldg(col + (size_t)i * ncol2);
-          const float w0 = __uint_as_float(w << 16), w1 = __uint_as_float(w & 0xFFFF0000u);
+        for (int gi = 0; gi < PROJ_G; ++gi)
 #pragma unroll
-          for (int gi = 0; gi < PROJ_G; ++gi) {
-            const float x = p[gi * d + i];
-            a0[gi] = fmaf(x, w0, a0[gi]);
-            a1[gi] = fmaf(x, w1, a1[gi]);
+          for (int e = 0; e < 8; ++e) acc[gi][e] = 0.f;
+        auto fma_row = [&](const uint4& w, uint32_t i) {
+          const uint32_t ww[4] = {w.x, w.y, w.z, w.w};
+          float x[PROJ_G];
+#pragma unroll
+          for (int gi = 0; gi < PROJ_G; ++gi) x[gi] = p[gi * d + i];
+#pragma unroll
+          for (int u = 0; u < 4; ++u) {
+            const float w0 = __uint_as_float(ww[u] << 16), w1 = __uint_as_float(ww[u] & 0xFFFF0000u);
+#pragma unroll
+            for (int gi = 0; gi < PROJ_G; ++gi) {
+              acc[gi][2 * u]     = fmaf(x[gi], w0, acc[gi][2 * u]);
+              acc[gi][2 * u + 1] = fmaf(x[gi], w1, acc[gi][2 * u + 1]);
+            }
           }
-        }
+        };
+        constexpr int INFL = 8;                                    // rows in flight
+        uint32_t i = sl;
+        for (; i + (INFL - 1) * slices < d; i += INFL * slices) {
+          uint4 w[INFL];
 #pragma unroll
-        for (int gi = 0; gi < PROJ_G; ++gi) {
-          part[((size_t)sl * PROJ_G + gi) * k + 2 * c2]     = a0[gi];
-          part[((size_t)sl * PROJ_G + gi) * k + 2 * c2 + 1] = a1[gi];
+          for (int u = 0; u < INFL; ++u) w[u] = ld_nc16(P4 + (size_t)(i + u * slices) * ncg + cg);
+#pragma unroll
+          for (int u = 0; u < INFL; ++u) fma_row(w[u], i + u * slices);
         }
+        for (; i < d; i += slices) fma_row(ld_nc16(P4 + (size_t)i * ncg + cg), i);
+#pragma unroll
+        for (int gi = 0; gi < PROJ_G; ++gi)
+#pragma unroll
+          for (int e = 0; e < 8; ++e) part[((size_t)sl * PROJ_G + gi) * k + cg * 8 + e] = acc[gi][e];
       }
     }
     __syncthreads();
@@ -152,26 +196,25 @@ k_project(const float* __restrict__ partial, const __nv_bfloat16* __restrict__ p
     g = p;                                      // identity: k == d
   }
 
-  for (int gi = 0; gi < PROJ_G; ++gi) {
-    const uint32_t b = b0 + gi;
-    if (b >= B) break;                          // uniform across the block
-    const float* gv = g + (size_t)gi * k;
-    float ss = 0.f;
-    for (uint32_t c = threadIdx.x; c < k; c += blockDim.x) ss = fmaf(gv[c], gv[c], ss);
-    ss = block_sum(ss, red);
-    const float nrm = sqrtf(ss);
-    const bool ok = isfinite(ss) && nrm >= 1e-20f;
-    float qs = 0.f;
-    __nv_bfloat16* dst = fp + (size_t)b * k;
-    for (uint32_t c = threadIdx.x; c < k; c += blockDim.x) {
+  // unit length + rounding: the G sequences side by side, 128 threads each
+  const float* gv = g + (size_t)grp * k;
+  float ss = 0.f;
+  for (uint32_t c = gt; c < k; c += PROJ_TPS) ss = fmaf(gv[c], gv[c], ss);
+  ss = group_sum(ss, red, grp);
+  const float nrm = sqrtf(ss);
+  const bool ok = isfinite(ss) && nrm >= 1e-20f;
+  float qs = 0.f;
+  if (bq < B) {
+    __nv_bfloat16* dst = fp + (size_t)bq * k;
+    for (uint32_t c = gt; c < k; c += PROJ_TPS) {
       __nv_bfloat16 q = __float2bfloat16_rn(ok ? gv[c] / nrm : 0.f);
       dst[c] = q;
       const float qf = __bfloat162float(q);
       qs = fmaf(qf, qf, qs);
     }
-    qs = block_sum(qs, red);
-    if (threadIdx.x == 0) rq[b] = (ok && qs > 0.f) ? 1.0f / sqrtf(qs) : 0.f;
   }
+  qs = group_sum(qs, red, grp);
+  if (gt == 0 && bq < B) rq[bq] = (ok && qs > 0.f) ? 1.0f / sqrtf(qs) : 0.f;
 }
 
 // rq[b] = 1/||fp[b]|| for fingerprints supplied by the caller; one warp per row.
@@ -197,8 +240,8 @@ __global__ void k_rownorm(const __nv_bfloat16* __restrict__ fp, uint32_t B, uint
 
 // ---------------------------------------------------------------------------
 size_t project_smem_bytes(uint32_t d, uint32_t k, bool has_proj) {
-  uint32_t slices = 1;
-  if (has_proj && (k / 2) < (uint32_t)PROJ_THREADS) slices = PROJ_THREADS / (k / 2);
+  const uint32_t ncg = k / 8;
+  const uint32_t slices = (has_proj && ncg < (uint32_t)PROJ_THREADS) ? PROJ_THREADS / ncg : 1;
   return ((size_t)PROJ_G * d + (has_proj ? (size_t)PROJ_G * k + (size_t)slices * PROJ_G * k : 0)) * sizeof(float);
 }
 
@@ -206,14 +249,42 @@ cudaError_t setup_fingerprint_kernels() {
   return cudaFuncSetAttribute(k_project, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024);
 }
 
-uint32_t pool_split_for(uint32_t B, uint32_t n, int sm_count, uint32_t R) {
-  // aim for >= 4 blocks per SM, never slices shorter than 4 passes of R rows
-  uint32_t want = (uint32_t)((4 * sm_count + B - 1) / (B ? B : 1));
-  uint32_t max_by_len = n / (4 * R) ? n / (4 * R) : 1;
-  uint32_t S = want < 1 ? 1 : want;
-  if (S > max_by_len) S = max_by_len;
-  if (S > (uint32_t)POOL_MAX_SPLIT) S = POOL_MAX_SPLIT;
-  return S;
+// Launch shape of the pooling pass.  The scratch it needs is grid * Jmax * d floats, which never exceeds
+// (B + 3 * POOL_MAX_GRID) * d.
+PoolPlan pool_plan(uint32_t B, uint32_t n, uint32_t d, bool bf16, int sm_count) {
+  PoolPlan P;
+  P.V = bf16 ? d / 8 : d / 4;
+  P.R = 512 / P.V; if (P.R < 1) P.R = 1;
+  if (P.R > n) P.R = n;
+  P.threads = (P.V * P.R + 31) / 32 * 32;
+  const unsigned long long rows = (unsigned long long)B * n;
+  unsigned long long grid = 4ull * (unsigned long long)sm_count;     // four blocks per SM: one wave
+  if (grid > POOL_MAX_GRID) grid = POOL_MAX_GRID;
+  const unsigned long long min_rows = 8ull * P.R;                    // keep spans long enough to pipeline
+  if (grid * min_rows > rows) grid = (rows + min_rows - 1) / min_rows;
+  if (grid < 1) grid = 1;
+  P.L = (uint32_t)((rows + grid - 1) / grid);
+  P.grid = (uint32_t)((rows + P.L - 1) / P.L);
+  P.Jmax = (P.L + n - 1) / n + 1;
+  P.smem = (size_t)P.R * d * sizeof(float);
+  return P;
+}
+
+static cudaError_t launch_pool(const PoolPlan& P, bool bf16, const void* h_in, float* partial,
+                               uint32_t B, uint32_t n, uint32_t d, cudaStream_t st) {
+  if (bf16)
+    k_pool<true><<<P.grid, P.threads, P.smem, st>>>((const uint4*)h_in, partial, B, n, d, P.V, P.R, P.L, P.Jmax);
+  else
+    k_pool<false><<<P.grid, P.threads, P.smem, st>>>((const uint4*)h_in, partial, B, n, d, P.V, P.R, P.L, P.Jmax);
+  return cudaGetLastError();
+}
+
+static cudaError_t launch_project(const PoolPlan& P, const float* partial, const __nv_bfloat16* proj,
+                                  const float* center, __nv_bfloat16* fp, float* rq,
+                                  uint32_t B, uint32_t n, uint32_t d, uint32_t k, cudaStream_t st) {
+  k_project<<<(B + PROJ_G - 1) / PROJ_G, PROJ_THREADS, project_smem_bytes(d, k, proj != nullptr), st>>>(
+      partial, proj, center, fp, rq, B, n, d, k, P.L, P.Jmax);
+  return cudaGetLastError();
 }
 
 cudaError_t launch_fingerprint(llmcache_bank* bk, const void* h_in, uint32_t B,
@@ -221,30 +292,15 @@ cudaError_t launch_fingerprint(llmcache_bank* bk, const void* h_in, uint32_t B,
   if (B == 0) return cudaSuccess;
   const llmcache_bank_desc& D = bk->desc;
   const bool bf16 = D.hidden_dtype == LLMCACHE_BF16;
-  const uint32_t d = D.d_model, n = D.seq_len, k = D.fp_dim;
-  const uint32_t V = bf16 ? d / 8 : d / 4;
-  uint32_t R = 512 / V; if (R < 1) R = 1;
-  if (R > n) R = n;
-  const uint32_t S = pool_split_for(B, n, bk->sm_count, R);
-  const uint32_t rows_per_slice = (n + S - 1) / S;
-  const uint32_t S_eff = (n + rows_per_slice - 1) / rows_per_slice;
-  dim3 grid(S_eff, B);
-  const size_t smem = (size_t)R * d * sizeof(float);
+  const PoolPlan P = pool_plan(B, D.seq_len, D.d_model, bf16, bk->sm_count);
+  cudaError_t e;
   {
-  ProfScope prof(bk, LLMCACHE_K_POOL, st);
-  if (bf16)
-    k_pool<true><<<grid, V * R, smem, st>>>((const uint4*)h_in, bk->a.pool_partial, n, d, V, R, S_eff, rows_per_slice);
-  else
-    k_pool<false><<<grid, V * R, smem, st>>>((const uint4*)h_in, bk->a.pool_partial, n, d, V, R, S_eff, rows_per_slice);
+    ProfScope prof(bk, LLMCACHE_K_POOL, st);
+    e = launch_pool(P, bf16, h_in, bk->a.pool_partial, B, D.seq_len, D.d_model, st);
   }
-  cudaError_t e = cudaGetLastError();
   if (e != cudaSuccess) return e;
-
-  const size_t smem2 = project_smem_bytes(d, k, bk->a.proj != nullptr);
   ProfScope prof(bk, LLMCACHE_K_PROJECT, st);
-  k_project<<<(B + PROJ_G - 1) / PROJ_G, PROJ_THREADS, smem2, st>>>(
-      bk->a.pool_partial, bk->a.proj, bk->a.center, fp, rq, B, n, d, k, S_eff);
-  return cudaGetLastError();
+  return launch_project(P, bk->a.pool_partial, bk->a.proj, bk->a.center, fp, rq, B, D.seq_len, D.d_model, D.fp_dim, st);
 }
 
 cudaError_t launch_rownorm(llmcache_bank* bk, const __nv_bfloat16* fp, uint32_t B, uint32_t k, float* rq, cudaStream_t st) {
@@ -327,33 +383,20 @@ extern "C" int llmcache_fingerprint_static(const void* h_in, uint32_t hidden_dty
   cudaError_t e = static_setup(dev, &sd);
   if (e != cudaSuccess) { cudaGetLastError(); return fail(LLMCACHE_ERR_CUDA, cudaGetErrorString(e)); }
 
-  const uint32_t V = bf16 ? d / 8 : d / 4;
-  uint32_t R = 512 / V; if (R < 1) R = 1;
-  if (R > n) R = n;
-  const uint32_t S = pool_split_for(B, n, sd->sm_count, R);
-  const uint32_t rows_per_slice = (n + S - 1) / S;
-  const uint32_t S_eff = (n + rows_per_slice - 1) / rows_per_slice;
-  if ((unsigned long long)B * S_eff * d > (unsigned long long)LLMCACHE_FINGERPRINT_STATIC_MAX_FLOATS) {
+  const PoolPlan P = pool_plan(B, n, d, bf16, sd->sm_count);
+  const unsigned long long need = (unsigned long long)P.grid * P.Jmax * d;
+  if (need > (unsigned long long)LLMCACHE_FINGERPRINT_STATIC_MAX_FLOATS) {
     std::snprintf(g_static_err, sizeof(g_static_err),
-                  "batch too large for the fixed scratch: B * splits * d_model = %llu floats, limit %llu",
-                  (unsigned long long)B * S_eff * d, (unsigned long long)LLMCACHE_FINGERPRINT_STATIC_MAX_FLOATS);
+                  "batch too large for the fixed scratch: %llu floats of partial sums needed, limit %llu",
+                  need, (unsigned long long)LLMCACHE_FINGERPRINT_STATIC_MAX_FLOATS);
     return LLMCACHE_ERR_SHAPE;
   }
   cudaStream_t st = (cudaStream_t)stream;
   // every partial sum that the second kernel reads is written by the first one in this call, so
   // nothing in the shared array has to start at zero
-  dim3 grid(S_eff, B);
-  const size_t smem = (size_t)R * d * sizeof(float);
-  if (bf16)
-    k_pool<true><<<grid, V * R, smem, st>>>((const uint4*)h_in, sd->scratch, n, d, V, R, S_eff, rows_per_slice);
-  else
-    k_pool<false><<<grid, V * R, smem, st>>>((const uint4*)h_in, sd->scratch, n, d, V, R, S_eff, rows_per_slice);
-  e = cudaGetLastError();
-  if (e == cudaSuccess) {
-    k_project<<<(B + PROJ_G - 1) / PROJ_G, PROJ_THREADS, project_smem_bytes(d, k, proj != nullptr), st>>>(
-        sd->scratch, (const __nv_bfloat16*)proj, center, (__nv_bfloat16*)fp, rq, B, n, d, k, S_eff);
-    e = cudaGetLastError();
-  }
+  e = launch_pool(P, bf16, h_in, sd->scratch, B, n, d, st);
+  if (e == cudaSuccess)
+    e = launch_project(P, sd->scratch, (const __nv_bfloat16*)proj, center, (__nv_bfloat16*)fp, rq, B, n, d, k, st);
   if (e != cudaSuccess) return fail(LLMCACHE_ERR_CUDA, cudaGetErrorString(e));
   return LLMCACHE_OK;
 }

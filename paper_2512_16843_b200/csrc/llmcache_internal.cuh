@@ -12,8 +12,7 @@ namespace llmc {
 
 constexpr uint32_t M_CAP = (1u << 30) - 1u;   // ceiling of the decayed match rate (Q8)
 constexpr uint32_t HIT_Q8 = 256u;             // one match in Q8
-constexpr uint32_t COPY_CHUNK = 32768u;       // bytes one CTA moves per work item in row copies
-constexpr int      POOL_MAX_SPLIT = 64;
+constexpr uint32_t POOL_MAX_GRID = 640;       // most blocks the pooling pass ever launches
 
 // Counters kept on the device (index into Bank::d_stats).
 enum { ST_SEQ = 0, ST_HIT, ST_MISS, ST_DEGEN, ST_INSERT, ST_EVICT, ST_DROP, ST_FLUSH, ST_COUNT };
@@ -36,7 +35,7 @@ struct BankArrays {
   __nv_bfloat16* proj;      // [d,k] or nullptr
   float*    center;         // [d] or nullptr
   // scratch
-  float*    pool_partial;   // [max_batch, POOL_MAX_SPLIT? no: split, d]
+  float*    pool_partial;   // [(max_batch + 3 * POOL_MAX_GRID), d] partial sums of the pooling pass
   unsigned long long* best; // [max_batch] packed (orderable score << 32 | ~slot); 0 = none
   uint32_t* hitcnt;         // [N] matches per slot within the current probe (zero between calls)
   int32_t*  victims;        // [min(max_batch,N)]
@@ -61,7 +60,6 @@ struct llmcache_bank {
   bool     probe_open = false;   // a probe happened and was not yet committed
   uint32_t last_B = 0;
   uint64_t n_probes = 0;
-  uint32_t pool_split_max = 0;   // splits the scratch is sized for
   int      sm_count = 0;
   uint32_t sort_len = 0;    // length of sort_key / sort_slot
   // TMA descriptor of the fingerprint matrix (opaque 128-byte blob)
@@ -96,14 +94,14 @@ struct ProfScope {
 size_t project_smem_bytes(uint32_t d, uint32_t k, bool has_proj);
 cudaError_t setup_fingerprint_kernels();
 cudaError_t setup_scan_kernels();
-uint32_t pool_split_for(uint32_t B, uint32_t n, int sm_count, uint32_t R);
+struct PoolPlan { uint32_t V, R, threads, grid, L, Jmax; size_t smem; };
+PoolPlan pool_plan(uint32_t B, uint32_t n, uint32_t d, bool bf16, int sm_count);
 cudaError_t launch_fingerprint(llmcache_bank* bk, const void* h_in, uint32_t B,
                                __nv_bfloat16* fp, float* rq, cudaStream_t st);
 cudaError_t launch_rownorm(llmcache_bank* bk, const __nv_bfloat16* fp, uint32_t B, uint32_t k, float* rq, cudaStream_t st);
 cudaError_t launch_scan(llmcache_bank* bk, const __nv_bfloat16* q, uint32_t B, cudaStream_t st);
 cudaError_t launch_decide(llmcache_bank* bk, uint32_t B, float tau, const float* rq,
                           const llmcache_probe_io* io, cudaStream_t st);
-cudaError_t launch_touch(llmcache_bank* bk, cudaStream_t st);
 cudaError_t launch_gather(llmcache_bank* bk, const void* h_in, void* h_out,
                           const llmcache_probe_io* io, uint32_t B, cudaStream_t st);
 cudaError_t launch_select_victims(llmcache_bank* bk, const llmcache_probe_io* io, uint32_t B,
@@ -145,6 +143,13 @@ __device__ __forceinline__ unsigned long long evict_key(const PolicyParams& p, u
 __device__ __forceinline__ uint4 ld_stream16(const void* p) {
   uint4 v;
   asm volatile("ld.global.nc.L1::no_allocate.v4.u32 {%0,%1,%2,%3}, [%4];"
+               : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "l"(p));
+  return v;
+}
+// 16-byte read-only load that is kept in issue order (several can be put in flight back to back).
+__device__ __forceinline__ uint4 ld_nc16(const void* p) {
+  uint4 v;
+  asm volatile("ld.global.nc.v4.u32 {%0,%1,%2,%3}, [%4];"
                : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "l"(p));
   return v;
 }

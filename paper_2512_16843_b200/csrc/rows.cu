@@ -2,69 +2,86 @@
 // compaction of miss inputs, and the write-back + insertion of computed layer
 // outputs (Algorithm 1 "C_l[f_X] <- h_l").  Rows are n*d elements and are moved
 // verbatim with 16-byte accesses.
+//
+// Work is counted in units of COPY_UNIT bytes of a row.  The units of all rows to
+// move form one flat list that is cut into equal spans, one per block, so every
+// block moves the same number of bytes whatever the hit / miss counts are (they
+// are only known on the device).
 #include "llmcache_internal.cuh"
 
 namespace llmc {
 
 constexpr int COPY_THREADS = 256;
-constexpr int COPY_UNROLL = COPY_CHUNK / (COPY_THREADS * 16);   // 8 vectors per thread per chunk
+constexpr int COPY_UNROLL = 8;                       // 16-byte vectors in flight per thread
+constexpr uint32_t COPY_UNIT = 4096;                 // bytes
 
 // Copy `bytes` (multiple of 16) from src to up to two destinations.
-__device__ __forceinline__ void copy_chunk(const char* __restrict__ src, char* __restrict__ d0,
+__device__ __forceinline__ void copy_bytes(const char* __restrict__ src, char* __restrict__ d0,
                                            char* __restrict__ d1, uint32_t bytes) {
   const uint32_t nvec = bytes >> 4;
-  if (nvec == COPY_THREADS * COPY_UNROLL) {
+  for (uint32_t base = 0; base < nvec; base += COPY_THREADS * COPY_UNROLL) {
     uint4 v[COPY_UNROLL];
 #pragma unroll
-    for (int u = 0; u < COPY_UNROLL; ++u) v[u] = ld_stream16(src + ((size_t)(u * COPY_THREADS + threadIdx.x) << 4));
+    for (int u = 0; u < COPY_UNROLL; ++u) {
+      const uint32_t i = base + u * COPY_THREADS + threadIdx.x;
+      if (i < nvec) v[u] = ld_stream16(src + ((size_t)i << 4));
+    }
 #pragma unroll
     for (int u = 0; u < COPY_UNROLL; ++u) {
-      const size_t off = (size_t)(u * COPY_THREADS + threadIdx.x) << 4;
-      if (d0) st_stream16(d0 + off, v[u]);
-      if (d1) st_stream16(d1 + off, v[u]);
-    }
-  } else {
-    for (uint32_t i = threadIdx.x; i < nvec; i += COPY_THREADS) {
-      const uint4 v = ld_stream16(src + ((size_t)i << 4));
-      if (d0) st_stream16(d0 + ((size_t)i << 4), v);
-      if (d1) st_stream16(d1 + ((size_t)i << 4), v);
+      const uint32_t i = base + u * COPY_THREADS + threadIdx.x;
+      if (i < nvec) {
+        if (d0) st_stream16(d0 + ((size_t)i << 4), v[u]);
+        if (d1) st_stream16(d1 + ((size_t)i << 4), v[u]);
+      }
     }
   }
 }
 
-// Work items [0, H*cpr_out): hit rows bank.act[slot] -> h_out[b].
-// Work items after that (only if h_miss): miss inputs h_in[b] -> h_miss[m].
+__device__ __forceinline__ void block_span(unsigned long long total, unsigned long long& u0, unsigned long long& u1) {
+  u0 = total * blockIdx.x / gridDim.x;
+  u1 = total * (blockIdx.x + 1) / gridDim.x;
+}
+
+// Units [0, H*upr): hit rows bank.act[slot] -> h_out[b].
+// Units after that (only if h_miss): miss inputs h_in[b] -> h_miss[m].
 __global__ void __launch_bounds__(COPY_THREADS)
 k_gather(const char* __restrict__ act, uint32_t act_rows, char* __restrict__ h_out, size_t row_bytes,
          const char* __restrict__ h_in, char* __restrict__ h_miss, size_t in_row_bytes,
          const int32_t* __restrict__ slot, const int32_t* __restrict__ hit_idx,
          const int32_t* __restrict__ miss_idx, const uint32_t* __restrict__ counts) {
   const uint32_t H = counts[0], M = counts[1];
-  const uint32_t cpr = (uint32_t)((row_bytes + COPY_CHUNK - 1) / COPY_CHUNK);
-  const uint32_t cpr_in = (uint32_t)((in_row_bytes + COPY_CHUNK - 1) / COPY_CHUNK);
-  const unsigned long long n_hit_items = (act && h_out) ? (unsigned long long)H * cpr : 0ull;
-  const unsigned long long n_items = n_hit_items + ((h_in && h_miss) ? (unsigned long long)M * cpr_in : 0ull);
-  for (unsigned long long it = blockIdx.x; it < n_items; it += gridDim.x) {
-    if (it < n_hit_items) {
-      const uint32_t i = (uint32_t)(it / cpr), c = (uint32_t)(it - (unsigned long long)i * cpr);
+  const uint32_t upr = (uint32_t)((row_bytes + COPY_UNIT - 1) / COPY_UNIT);
+  const uint32_t upr_in = (uint32_t)((in_row_bytes + COPY_UNIT - 1) / COPY_UNIT);
+  const unsigned long long n_hit = (act && h_out) ? (unsigned long long)H * upr : 0ull;
+  const unsigned long long total = n_hit + ((h_in && h_miss) ? (unsigned long long)M * upr_in : 0ull);
+  unsigned long long u, u1;
+  block_span(total, u, u1);
+  while (u < u1) {
+    if (u < n_hit) {
+      const uint32_t i = (uint32_t)(u / upr), w0 = (uint32_t)(u - (unsigned long long)i * upr);
+      const unsigned long long left = (u1 < n_hit ? u1 : n_hit) - u;
+      const uint32_t w1 = (uint32_t)min((unsigned long long)upr, w0 + left);
       const int32_t b = hit_idx[i];
       const uint32_t row = (uint32_t)slot[b] % act_rows;
-      const size_t off = (size_t)c * COPY_CHUNK;
-      const uint32_t bytes = (uint32_t)min((size_t)COPY_CHUNK, row_bytes - off);
-      copy_chunk(act + (size_t)row * row_bytes + off, h_out + (size_t)b * row_bytes + off, nullptr, bytes);
+      const size_t off = (size_t)w0 * COPY_UNIT;
+      const uint32_t bytes = (uint32_t)(min(row_bytes, (size_t)w1 * COPY_UNIT) - off);
+      copy_bytes(act + (size_t)row * row_bytes + off, h_out + (size_t)b * row_bytes + off, nullptr, bytes);
+      u += w1 - w0;
     } else {
-      const unsigned long long jt = it - n_hit_items;
-      const uint32_t m = (uint32_t)(jt / cpr_in), c = (uint32_t)(jt - (unsigned long long)m * cpr_in);
+      const unsigned long long jt = u - n_hit;
+      const uint32_t m = (uint32_t)(jt / upr_in), w0 = (uint32_t)(jt - (unsigned long long)m * upr_in);
+      const uint32_t w1 = (uint32_t)min((unsigned long long)upr_in, w0 + (u1 - u));
       const int32_t b = miss_idx[m];
-      const size_t off = (size_t)c * COPY_CHUNK;
-      const uint32_t bytes = (uint32_t)min((size_t)COPY_CHUNK, in_row_bytes - off);
-      copy_chunk(h_in + (size_t)b * in_row_bytes + off, h_miss + (size_t)m * in_row_bytes + off, nullptr, bytes);
+      const size_t off = (size_t)w0 * COPY_UNIT;
+      const uint32_t bytes = (uint32_t)(min(in_row_bytes, (size_t)w1 * COPY_UNIT) - off);
+      copy_bytes(h_in + (size_t)b * in_row_bytes + off, h_miss + (size_t)m * in_row_bytes + off, nullptr, bytes);
+      u += w1 - w0;
     }
   }
 }
 
-// Work item (m, c): chunk c of miss_out[m] -> h_out[miss_idx[m]] and -> act[new_slot[m]].
-// The block that owns chunk 0 also writes the key and the metadata of the new entry.
+// Units of miss_out[m] -> h_out[miss_idx[m]] and -> act[new_slot[m]].  The block whose span holds
+// the first unit of a row also writes the key and the metadata of the new entry.
 __global__ void __launch_bounds__(COPY_THREADS)
 k_scatter_insert(const char* __restrict__ miss_out, char* __restrict__ h_out, char* __restrict__ act,
                  size_t row_bytes, const int32_t* __restrict__ miss_idx, const int32_t* __restrict__ new_slot,
@@ -74,19 +91,22 @@ k_scatter_insert(const char* __restrict__ miss_out, char* __restrict__ h_out, ch
                  uint32_t* __restrict__ last_use, uint32_t* __restrict__ insert_tick, uint32_t* __restrict__ hits,
                  uint32_t* __restrict__ rate, uint32_t* __restrict__ rate_epoch, uint32_t tick, uint32_t epoch) {
   const uint32_t M = counts[1];
-  const uint32_t cpr = (uint32_t)((row_bytes + COPY_CHUNK - 1) / COPY_CHUNK);
-  const unsigned long long n_items = (unsigned long long)M * cpr;
+  const uint32_t upr = (uint32_t)((row_bytes + COPY_UNIT - 1) / COPY_UNIT);
+  const unsigned long long total = (unsigned long long)M * upr;
   const uint32_t kv = k / 8;                      // 16-byte vectors per fingerprint row
-  for (unsigned long long it = blockIdx.x; it < n_items; it += gridDim.x) {
-    const uint32_t m = (uint32_t)(it / cpr), c = (uint32_t)(it - (unsigned long long)m * cpr);
+  unsigned long long u, u1;
+  block_span(total, u, u1);
+  while (u < u1) {
+    const uint32_t m = (uint32_t)(u / upr), w0 = (uint32_t)(u - (unsigned long long)m * upr);
+    const uint32_t w1 = (uint32_t)min((unsigned long long)upr, w0 + (u1 - u));
     const int32_t b = miss_idx[m];
     const int32_t v = new_slot[m];
-    const size_t off = (size_t)c * COPY_CHUNK;
-    const uint32_t bytes = (uint32_t)min((size_t)COPY_CHUNK, row_bytes - off);
+    const size_t off = (size_t)w0 * COPY_UNIT;
+    const uint32_t bytes = (uint32_t)(min(row_bytes, (size_t)w1 * COPY_UNIT) - off);
     char* d0 = h_out ? h_out + (size_t)b * row_bytes + off : nullptr;
     char* d1 = (act && v >= 0) ? act + (size_t)v * row_bytes + off : nullptr;
-    if (miss_out && (d0 || d1)) copy_chunk(miss_out + (size_t)m * row_bytes + off, d0, d1, bytes);
-    if (c == 0 && v >= 0) {
+    if (miss_out && (d0 || d1)) copy_bytes(miss_out + (size_t)m * row_bytes + off, d0, d1, bytes);
+    if (w0 == 0 && v >= 0) {
       for (uint32_t i = threadIdx.x; i < kv; i += COPY_THREADS)
         bank_fp[(size_t)v * kv + i] = q_fp[(size_t)b * kv + i];
       if (threadIdx.x == 0) {
@@ -99,13 +119,15 @@ k_scatter_insert(const char* __restrict__ miss_out, char* __restrict__ h_out, ch
         rate_epoch[v] = epoch;
       }
     }
+    u += w1 - w0;
   }
 }
 
+// Four blocks per SM, but never more blocks than there could be units of work.
 static uint32_t copy_grid(const llmcache_bank* bk, uint32_t B, size_t row_bytes) {
-  const unsigned long long items = (unsigned long long)B * ((row_bytes + COPY_CHUNK - 1) / COPY_CHUNK);
-  unsigned long long g = (unsigned long long)bk->sm_count * 8;
-  if (items < g) g = items;
+  const unsigned long long units = (unsigned long long)B * ((row_bytes + COPY_UNIT - 1) / COPY_UNIT);
+  unsigned long long g = (unsigned long long)bk->sm_count * 4;
+  if (units < g) g = units;
   return g ? (uint32_t)g : 1u;
 }
 

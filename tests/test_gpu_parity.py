@@ -90,6 +90,23 @@ def test_churn_lockstep_many_batches(policy):
     gb.close()
 
 
+def test_large_bank_eviction_path_lockstep():
+    """More than 2048 slots: victim selection takes the radix-select path; must match the oracle's order."""
+    N, n, d, B = 2500, 2, 64, 300
+    gb, ob = make_pair(N, n, d, d, B, "bf16", half_life_ticks=2, min_age_ticks=1, stale_floor_q8=200)
+    bufs = L.ProbeBuffers(B, d, DEV)
+    hot = rand_h(100, n, d, 77, "bf16")
+    inserted = 0
+    for step in range(14):
+        junk = rand_h(B - 100, n, d, 300 + step, "bf16")
+        h = torch.cat([hot, junk])[synth.shuffled(B, 400 + step, DEV)].contiguous()
+        r = U.lockstep_step(gb, ob, bufs, h, "bf16", synth.activations(B, n, d, 500 + step, DEV))
+        inserted += r["inserted"]
+    st = gb.stats()
+    assert inserted > N and st["evictions"] > 0 and st["resident"] == N
+    gb.close()
+
+
 def test_probe_fp_path_and_act_rows_aliasing():
     N, k, B = 5000, 256, 300
     bank_fp, q, src = synth.scan_stress(N, B, k, n_clusters=128, seed=31, device=DEV)
