@@ -80,7 +80,7 @@ typedef struct llmcache_bank_desc {
   int32_t  device;            /* CUDA device ordinal */
   uint32_t capacity;          /* N >= 1 slots */
   uint32_t seq_len;           /* n >= 1 */
-  uint32_t d_model;           /* d, multiple of 8, <= 8192 */
+  uint32_t d_model;           /* d, multiple of 8, <= 7680 (bf16 inputs) or 3840 (f32 inputs) */
   uint32_t fp_dim;            /* k, multiple of 64, <= 2048; must equal d_model when proj == NULL */
   uint32_t hidden_dtype;      /* LLMCACHE_F32 | LLMCACHE_BF16 */
   uint32_t act_rows;          /* rows of the activation store; 0 => capacity.  slot j uses row j % act_rows.
@@ -132,8 +132,9 @@ enum {
   LLMCACHE_K_SCAN = 3,      /* Sec. III-C cosine scan + best slot                  */
   LLMCACHE_K_DECIDE = 4,    /* Sec. IV-A threshold + hit/miss compaction           */
   LLMCACHE_K_TOUCH = 5,     /* (unused: the metadata refresh runs inside DECIDE)  */
-  LLMCACHE_K_GATHER = 6,    /* Algorithm 1 reuse: copy of cached outputs           */
-  LLMCACHE_K_SELECT = 7,    /* Sec. IV-D victim selection                          */
+  LLMCACHE_K_GATHER = 6,    /* Algorithm 1 reuse: copy of cached outputs; one block of it
+                               also picks the victims for the commit (Sec. IV-D)   */
+  LLMCACHE_K_SELECT = 7,    /* (unused: victim selection runs inside GATHER)       */
   LLMCACHE_K_SCATTER = 8,   /* Algorithm 1 insert: write-back + store              */
   LLMCACHE_K_EVICT = 9,     /* Sec. III-E flushes                                  */
   LLMCACHE_K_COUNT = 10
@@ -219,7 +220,8 @@ int llmcache_commit(llmcache_bank_t* bank, const void* miss_out, const llmcache_
 
 /* Refresh controller (Sec. III-E): drop every stale entry, every entry idle
  * for more than max_idle_ticks, all entries, or the n listed slots (device
- * i32).  n_evicted_dev: optional device u32 [1] receiving the count. */
+ * i32).  n_evicted_dev: optional device u32 [1] receiving the count.  Not between a probe and its
+ * commit (LLMCACHE_ERR_STATE): the slots for the open probe's misses are already chosen. */
 int llmcache_evict(llmcache_bank_t* bank, uint32_t mode, const int32_t* slots, uint32_t n,
                    uint32_t* n_evicted_dev, void* stream);
 

@@ -17,7 +17,7 @@ inline uint32_t pow2_ceil(uint32_t x) { uint32_t p = 1; while (p < x) p <<= 1; r
 
 struct Layout {
   size_t fp, rb, valid, last_use, insert_tick, hits, rate, rate_epoch, act, proj, center;
-  size_t pool_partial, best, hitcnt, victims, sort_key, sort_slot, stats, status, misc, total;
+  size_t pool_partial, best, hitcnt, victims, new_slot, sort_key, sort_slot, stats, status, misc, total;
   uint32_t sort_len;
 };
 
@@ -40,8 +40,7 @@ int check_desc(const llmcache_bank_desc* d) {
   if (d->hidden_dtype != LLMCACHE_F32 && d->hidden_dtype != LLMCACHE_BF16) return LLMCACHE_ERR_ARG;
   if (d->cmp != LLMCACHE_GT && d->cmp != LLMCACHE_GE) return LLMCACHE_ERR_ARG;
   if (d->policy != LLMCACHE_LRU && d->policy != LLMCACHE_LRU_STALENESS) return LLMCACHE_ERR_ARG;
-  if (d->d_model % 8 != 0 || d->d_model > 8192) return LLMCACHE_ERR_SHAPE;
-  if (d->hidden_dtype == LLMCACHE_F32 && d->d_model > 4096) return LLMCACHE_ERR_SHAPE;
+  if (d->d_model % 8 != 0 || d->d_model > (d->hidden_dtype == LLMCACHE_BF16 ? 7680u : 3840u)) return LLMCACHE_ERR_SHAPE;
   if (d->fp_dim % 64 != 0 || d->fp_dim > 2048) return LLMCACHE_ERR_SHAPE;
   if (!d->proj && d->fp_dim != d->d_model) return LLMCACHE_ERR_SHAPE;
   if (d->capacity > (1u << 30) || d->max_batch > (1u << 24)) return LLMCACHE_ERR_SHAPE;
@@ -76,6 +75,7 @@ Layout make_layout(const llmcache_bank_desc& d) {
   L.hitcnt = take(N * 4);
   const uint32_t vmax = d.max_batch < d.capacity ? d.max_batch : d.capacity;
   L.victims = take((size_t)vmax * 4);
+  L.new_slot = take((size_t)d.max_batch * 4);
   L.sort_len = pow2_ceil(vmax);
   L.sort_key = take((size_t)L.sort_len * 8);
   L.sort_slot = take((size_t)L.sort_len * 4);
@@ -210,6 +210,7 @@ int llmcache_bank_create(const llmcache_bank_desc* desc, llmcache_bank_t** bank_
   a.best = (unsigned long long*)(base + L.best);
   a.hitcnt = (uint32_t*)(base + L.hitcnt);
   a.victims = (int32_t*)(base + L.victims);
+  a.new_slot = (int32_t*)(base + L.new_slot);
   a.sort_key = (unsigned long long*)(base + L.sort_key);
   a.sort_slot = (uint32_t*)(base + L.sort_slot);
   a.stats = (unsigned long long*)(base + L.stats);
@@ -225,6 +226,7 @@ int llmcache_bank_create(const llmcache_bank_desc* desc, llmcache_bank_t** bank_
     e = cudaMemcpy(a.center, desc->center, (size_t)desc->d_model * 4, cudaMemcpyDefault);
   if (e == cudaSuccess) e = setup_fingerprint_kernels();
   if (e == cudaSuccess) e = setup_scan_kernels();
+  if (e == cudaSuccess) e = setup_rows_kernels();
   if (e == cudaSuccess) e = cudaDeviceSynchronize();
   if (e != cudaSuccess) {
     if (bk->owns_memory) cudaFree(bk->base);
@@ -324,12 +326,8 @@ int llmcache_commit(llmcache_bank_t* bk, const void* miss_out, const llmcache_pr
   cudaStream_t st = (cudaStream_t)stream;
   bk->probe_open = false;
   if (B == 0) return LLMCACHE_OK;
-  // without a caller buffer the slot list goes to the packed-best scratch, which is idle between
-  // probes (8 bytes per sequence) and must be zero again before the next one
-  int32_t* ns = new_slot ? new_slot : reinterpret_cast<int32_t*>(bk->a.best);
-  cudaError_t e = launch_select_victims(bk, io, B, ns, st);
-  if (e == cudaSuccess) e = launch_scatter_insert(bk, miss_out, io, h_out, ns, B, st);
-  if (e == cudaSuccess && !new_slot) e = cudaMemsetAsync(bk->a.best, 0, (size_t)B * 8, st);
+  // the slots were chosen during the probe (inside the gather kernel); here the rows move
+  cudaError_t e = launch_scatter_insert(bk, miss_out, io, h_out, new_slot, B, st);
   if (e != cudaSuccess) return cuda_fail(e, __func__);
   return LLMCACHE_OK;
 }
@@ -339,6 +337,7 @@ int llmcache_evict(llmcache_bank_t* bk, uint32_t mode, const int32_t* slots, uin
   if (!bk) return LLMCACHE_ERR_ARG;
   if (mode > LLMCACHE_EVICT_SLOTS) return LLMCACHE_ERR_ARG;
   if (mode == LLMCACHE_EVICT_SLOTS && n && !slots) return LLMCACHE_ERR_ARG;
+  if (bk->probe_open && bk->last_B) return LLMCACHE_ERR_STATE;   // the open probe's slot choice would go stale
   DeviceGuard guard(bk->desc.device);
   if (!guard.ok) return LLMCACHE_ERR_CUDA;
   cudaError_t e = launch_evict(bk, mode, slots, n, n_evicted_dev, (cudaStream_t)stream);

@@ -37,6 +37,7 @@ k_decide_compact(unsigned long long* __restrict__ best, const float* __restrict_
                  unsigned long long* __restrict__ stats,
                  uint32_t* __restrict__ last_use, uint32_t* __restrict__ hits_total, uint32_t* __restrict__ rate,
                  uint32_t* __restrict__ rate_epoch, uint32_t tick, uint32_t epoch) {
+  griddep_sync();
   __shared__ uint32_t warp_tot[32];
   uint32_t hbase = 0, mbase = 0, ndegen = 0;
   for (uint32_t base = 0; base < B; base += DEC_THREADS) {
@@ -112,12 +113,10 @@ k_decide_compact(unsigned long long* __restrict__ best, const float* __restrict_
 cudaError_t launch_decide(llmcache_bank* bk, uint32_t B, float tau, const float* rq,
                           const llmcache_probe_io* io, cudaStream_t st) {
   ProfScope prof(bk, LLMCACHE_K_DECIDE, st);
-  k_decide_compact<<<1, DEC_THREADS, 0, st>>>(bk->a.best, rq, B, tau, bk->desc.cmp == LLMCACHE_GE,
-                                              io->hit, io->slot, io->score, io->hit_idx, io->miss_idx,
-                                              io->counts, bk->a.hitcnt, bk->a.stats,
-                                              bk->a.last_use, bk->a.hits, bk->a.rate, bk->a.rate_epoch,
-                                              (uint32_t)bk->tick, (uint32_t)(bk->tick / bk->pol.half_life));
-  return cudaGetLastError();
+  return launch_k(k_decide_compact, dim3(1), dim3(DEC_THREADS), 0, st, bk->a.best, rq, B, tau,
+                  (int)(bk->desc.cmp == LLMCACHE_GE), io->hit, io->slot, io->score, io->hit_idx, io->miss_idx,
+                  io->counts, bk->a.hitcnt, bk->a.stats, bk->a.last_use, bk->a.hits, bk->a.rate, bk->a.rate_epoch,
+                  (uint32_t)bk->tick, (uint32_t)(bk->tick / bk->pol.half_life));
 }
 
 }  // namespace llmc

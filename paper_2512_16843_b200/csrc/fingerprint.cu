@@ -1,80 +1,147 @@
 // Fingerprint kernels (Sec. IV-B): pooled reduction over the sequence
 // positions, centring + projection, unit-length scaling, bf16 rounding.
 #include "llmcache_internal.cuh"
+#include "ptx.cuh"
 
 namespace llmc {
 
 // ---------------------------------------------------------------------------
 // Pool.  The B*n rows of the batch are one flat list that is cut into equal
-// spans, one per block, so that every block streams the same number of bytes
-// and the grid is a single wave.  A span may cross sequence boundaries: a block
-// writes one vector of partial sums per sequence it touches,
+// spans, one per block (one block per SM), so every block streams the same
+// number of bytes.  A span may cross sequence boundaries: a block writes one
+// vector of partial sums per sequence it touches,
 //     partial[(block * Jmax + j), :] = sum of its rows of the j-th sequence it touches.
-// A block is V x R threads (rounded up to whole warps): V = 16-byte vectors per
-// row, R = rows taken per pass.  Every thread always owns the same E columns, so
-// the running sums live in registers; the R row groups are combined through
-// shared memory in a fixed order (deterministic).
+//
+// The rows of a span are contiguous in memory.  One producer thread moves them
+// into a ring of shared-memory stages with bulk asynchronous copies (completion
+// counted on an mbarrier per stage), which keeps well over 100 KB of reads in
+// flight per SM without holding them in registers.  The consumer threads form a
+// V x R grid: V = 16-byte vectors per row, R = rows taken per pass; every thread
+// always owns the same E columns, so the running sums live in registers.  At the
+// end of a sequence's rows the R row groups are combined through shared memory
+// in a fixed order (deterministic).  A stage never crosses a sequence boundary.
+// All waits are bounded; on expiry the status word is set and the block drains
+// its copies and leaves.
 // ---------------------------------------------------------------------------
 template <bool BF16>
 __global__ void __launch_bounds__(1024, 1)
-k_pool(const uint4* __restrict__ h, float* __restrict__ partial,
-       uint32_t B, uint32_t n, uint32_t d, uint32_t V, uint32_t R, uint32_t L, uint32_t Jmax) {
+k_pool(const uint4* __restrict__ h, float* __restrict__ partial, uint32_t* __restrict__ status,
+       uint32_t B, uint32_t n, uint32_t d, uint32_t V, uint32_t R, uint32_t L, uint32_t Jmax,
+       uint32_t stage_rows, uint32_t stages, uint32_t cons_threads) {
+  griddep_sync();
   constexpr int E = BF16 ? 8 : 4;
-  extern __shared__ float sm_pool[];           // [R][d]
-  const bool active = threadIdx.x < V * R;
-  const uint32_t col = threadIdx.x % V, rg = threadIdx.x / V;
-  const unsigned long long total = (unsigned long long)B * n;
-  unsigned long long r0 = (unsigned long long)blockIdx.x * L;
-  unsigned long long r1 = r0 + L;
-  if (r1 > total) r1 = total;
-  uint32_t b = (uint32_t)(r0 / n);
-  float* out = partial + (size_t)blockIdx.x * Jmax * d;
+  extern __shared__ __align__(128) uint8_t sm_raw[];
+  const uint32_t row_bytes = V * 16;
+  const uint32_t stage_bytes = stage_rows * row_bytes;
+  const uint32_t ring = smem_u32(sm_raw);
+  float* red = reinterpret_cast<float*>(sm_raw + (size_t)stages * stage_bytes);          // [R][d]
+  uint8_t* tail = reinterpret_cast<uint8_t*>(red + (size_t)R * d);
+  const uint32_t bar0 = smem_u32(tail);                                                  // full[stages], empty[stages]
+  volatile uint32_t* flags = reinterpret_cast<volatile uint32_t*>(tail + 16 * stages);   // [0] abort, [1] go
+  auto full_bar = [&](uint32_t s) { return bar0 + 8 * s; };
+  auto empty_bar = [&](uint32_t s) { return bar0 + 8 * (stages + s); };
 
-  auto add = [](float (&acc)[E], const uint4& v) {
-    if (BF16) {
-      const uint32_t w[4] = {v.x, v.y, v.z, v.w};
-#pragma unroll
-      for (int i = 0; i < 4; ++i) {
-        acc[2 * i]     += __uint_as_float(w[i] << 16);
-        acc[2 * i + 1] += __uint_as_float(w[i] & 0xFFFF0000u);
-      }
-    } else {
-      acc[0] += __uint_as_float(v.x); acc[1] += __uint_as_float(v.y);
-      acc[2] += __uint_as_float(v.z); acc[3] += __uint_as_float(v.w);
-    }
-  };
-
-  while (r0 < r1) {
-    unsigned long long seg_end = (unsigned long long)(b + 1) * n;
-    if (seg_end > r1) seg_end = r1;
-    float acc[E];
-#pragma unroll
-    for (int e = 0; e < E; ++e) acc[e] = 0.f;
-    if (active) {
-      const uint4* base = h + col;
-      unsigned long long t = r0 + rg;
-      for (; t + 3ull * R < seg_end; t += 4ull * R) {        // four rows in flight per thread
-        const uint4 v0 = ld_stream16(base + t * V);
-        const uint4 v1 = ld_stream16(base + (t + R) * V);
-        const uint4 v2 = ld_stream16(base + (t + 2ull * R) * V);
-        const uint4 v3 = ld_stream16(base + (t + 3ull * R) * V);
-        add(acc, v0); add(acc, v1); add(acc, v2); add(acc, v3);
-      }
-      for (; t < seg_end; t += R) add(acc, ld_stream16(base + t * V));
-#pragma unroll
-      for (int e = 0; e < E; ++e) sm_pool[(size_t)rg * d + col * E + e] = acc[e];
-    }
-    __syncthreads();
-    for (uint32_t i = threadIdx.x; i < d; i += blockDim.x) {
-      float sum = 0.f;
-      for (uint32_t r = 0; r < R; ++r) sum += sm_pool[(size_t)r * d + i];
-      out[i] = sum;
-    }
-    __syncthreads();
-    out += d;
-    r0 = seg_end;
-    ++b;
+  if (threadIdx.x == 0) {
+    for (uint32_t s = 0; s < stages; ++s) { mbar_init(full_bar(s), 1); mbar_init(empty_bar(s), cons_threads / 32); }
+    flags[0] = 0; flags[1] = 0;
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
   }
+  __syncthreads();
+
+  const unsigned long long total = (unsigned long long)B * n;
+  unsigned long long r = (unsigned long long)blockIdx.x * L;
+  unsigned long long r1 = r + L;
+  if (r1 > total) r1 = total;
+  uint32_t b = (uint32_t)(r / n);
+  uint32_t it = 0;
+
+  if (threadIdx.x >= cons_threads) {
+    // ---------------------------------------------------------------- producer (one thread)
+    if (threadIdx.x == cons_threads) {
+      bool ok = true;
+      while (r < r1 && ok) {
+        unsigned long long seg_end = (unsigned long long)(b + 1) * n;
+        if (seg_end > r1) seg_end = r1;
+        while (r < seg_end) {
+          const uint32_t rows = (uint32_t)min((unsigned long long)stage_rows, seg_end - r);
+          const uint32_t s = it % stages, ph = (it / stages) & 1u;
+          if (!mbar_wait(empty_bar(s), ph ^ 1u, flags)) { ok = false; break; }
+          mbar_expect_tx(full_bar(s), rows * row_bytes);
+          bulk_load_1d(ring + s * stage_bytes, h + r * V, rows * row_bytes, full_bar(s));
+          r += rows;
+          ++it;
+        }
+        ++b;
+      }
+      if (!ok) {
+        flags[0] = 1;
+        atomicExch(status, 1u);
+        // copies that were started must land before the block's shared memory is released
+        const uint32_t back = it < stages ? it : stages;
+        volatile uint32_t never = 0;
+        for (uint32_t i = 0; i < back; ++i) {
+          const uint32_t itx = it - 1 - i;
+          mbar_wait(full_bar(itx % stages), (itx / stages) & 1u, &never, 200000000ull);
+        }
+      }
+    }
+  } else {
+    // ---------------------------------------------------------------- consumers
+    const bool active = threadIdx.x < V * R;
+    const uint32_t col = threadIdx.x % V, rg = threadIdx.x / V;
+    float* out = partial + (size_t)blockIdx.x * Jmax * d;
+    while (r < r1) {
+      unsigned long long seg_end = (unsigned long long)(b + 1) * n;
+      if (seg_end > r1) seg_end = r1;
+      float acc[E];
+#pragma unroll
+      for (int e = 0; e < E; ++e) acc[e] = 0.f;
+      while (r < seg_end) {
+        const uint32_t rows = (uint32_t)min((unsigned long long)stage_rows, seg_end - r);
+        const uint32_t s = it % stages, ph = (it / stages) & 1u;
+        if (!mbar_wait(full_bar(s), ph, flags)) { flags[0] = 1; atomicExch(status, 1u); }
+        if (active) {
+          const uint32_t src = ring + s * stage_bytes + col * 16;
+          for (uint32_t rr = rg; rr < rows; rr += R) {
+            const uint4 v = lds16(src + rr * row_bytes);
+            if (BF16) {
+              const uint32_t w[4] = {v.x, v.y, v.z, v.w};
+#pragma unroll
+              for (int i = 0; i < 4; ++i) {
+                acc[2 * i]     += __uint_as_float(w[i] << 16);
+                acc[2 * i + 1] += __uint_as_float(w[i] & 0xFFFF0000u);
+              }
+            } else {
+              acc[0] += __uint_as_float(v.x); acc[1] += __uint_as_float(v.y);
+              acc[2] += __uint_as_float(v.z); acc[3] += __uint_as_float(v.w);
+            }
+          }
+        }
+        __syncwarp();
+        if ((threadIdx.x & 31) == 0) mbar_arrive(empty_bar(s));      // this warp is done with the stage
+        r += rows;
+        ++it;
+      }
+      // combine the row groups of this sequence piece (consumer threads only)
+      if (active) {
+#pragma unroll
+        for (int e = 0; e < E; ++e) red[(size_t)rg * d + col * E + e] = acc[e];
+      }
+      if (threadIdx.x == 0) flags[1] = flags[0];
+      asm volatile("bar.sync 1, %0;" ::"r"(cons_threads) : "memory");
+      if (flags[1]) break;                                           // uniform over the consumers
+      for (uint32_t i = threadIdx.x; i < d; i += cons_threads) {
+        float sum = 0.f;
+        for (uint32_t q = 0; q < R; ++q) sum += red[(size_t)q * d + i];
+        out[i] = sum;
+      }
+      asm volatile("bar.sync 1, %0;" ::"r"(cons_threads) : "memory");
+      out += d;
+      ++b;
+    }
+  }
+  __syncthreads();
 }
 
 // ---------------------------------------------------------------------------
@@ -109,6 +176,7 @@ __global__ void __launch_bounds__(PROJ_THREADS)
 k_project(const float* __restrict__ partial, const __nv_bfloat16* __restrict__ proj,
           const float* __restrict__ center, __nv_bfloat16* __restrict__ fp, float* __restrict__ rq,
           uint32_t B, uint32_t n, uint32_t d, uint32_t k, uint32_t L, uint32_t Jmax) {
+  griddep_sync();
   extern __shared__ float sm[];
   float* p = sm;                               // [G][d]
   float* g = p + (size_t)PROJ_G * d;           // [G][k]            (only with projection)
@@ -219,6 +287,7 @@ k_project(const float* __restrict__ partial, const __nv_bfloat16* __restrict__ p
 
 // rq[b] = 1/||fp[b]|| for fingerprints supplied by the caller; one warp per row.
 __global__ void k_rownorm(const __nv_bfloat16* __restrict__ fp, uint32_t B, uint32_t k, float* __restrict__ rq) {
+  griddep_sync();
   const uint32_t row = blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
   const uint32_t lane = threadIdx.x & 31;
   if (row >= B) return;
@@ -246,7 +315,10 @@ size_t project_smem_bytes(uint32_t d, uint32_t k, bool has_proj) {
 }
 
 cudaError_t setup_fingerprint_kernels() {
-  return cudaFuncSetAttribute(k_project, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024);
+  cudaError_t e = cudaFuncSetAttribute(k_project, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024);
+  if (e == cudaSuccess) e = cudaFuncSetAttribute(k_pool<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, 220 * 1024);
+  if (e == cudaSuccess) e = cudaFuncSetAttribute(k_pool<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, 220 * 1024);
+  return e;
 }
 
 // Launch shape of the pooling pass.  The scratch it needs is grid * Jmax * d floats, which never exceeds
@@ -256,35 +328,41 @@ PoolPlan pool_plan(uint32_t B, uint32_t n, uint32_t d, bool bf16, int sm_count) 
   P.V = bf16 ? d / 8 : d / 4;
   P.R = 512 / P.V; if (P.R < 1) P.R = 1;
   if (P.R > n) P.R = n;
-  P.threads = (P.V * P.R + 31) / 32 * 32;
+  P.cons_threads = (P.V * P.R + 31) / 32 * 32;
+  P.threads = P.cons_threads + 32;                                    // + the producer's warp
+  const uint32_t row_bytes = P.V * 16;
+  // a stage holds a whole number of passes of R rows, about 16 KB; the ring about 160 KB
+  uint32_t passes = 16384 / (P.R * row_bytes); if (passes < 1) passes = 1;
+  P.stage_rows = P.R * passes;
+  const uint32_t stage_bytes = P.stage_rows * row_bytes;
+  P.stages = (160 * 1024) / stage_bytes;
+  if (P.stages > 16) P.stages = 16;
+  if (P.stages < 2) P.stages = 2;
   const unsigned long long rows = (unsigned long long)B * n;
-  unsigned long long grid = 4ull * (unsigned long long)sm_count;     // four blocks per SM: one wave
+  unsigned long long grid = (unsigned long long)sm_count;              // one block per SM
   if (grid > POOL_MAX_GRID) grid = POOL_MAX_GRID;
-  const unsigned long long min_rows = 8ull * P.R;                    // keep spans long enough to pipeline
+  const unsigned long long min_rows = 2ull * P.stage_rows;             // keep spans long enough to pipeline
   if (grid * min_rows > rows) grid = (rows + min_rows - 1) / min_rows;
   if (grid < 1) grid = 1;
   P.L = (uint32_t)((rows + grid - 1) / grid);
   P.grid = (uint32_t)((rows + P.L - 1) / P.L);
   P.Jmax = (P.L + n - 1) / n + 1;
-  P.smem = (size_t)P.R * d * sizeof(float);
+  P.smem = (size_t)P.stages * stage_bytes + (size_t)P.R * d * sizeof(float) + 16 * P.stages + 16;
   return P;
 }
 
-static cudaError_t launch_pool(const PoolPlan& P, bool bf16, const void* h_in, float* partial,
+static cudaError_t launch_pool(const PoolPlan& P, bool bf16, const void* h_in, float* partial, uint32_t* status,
                                uint32_t B, uint32_t n, uint32_t d, cudaStream_t st) {
-  if (bf16)
-    k_pool<true><<<P.grid, P.threads, P.smem, st>>>((const uint4*)h_in, partial, B, n, d, P.V, P.R, P.L, P.Jmax);
-  else
-    k_pool<false><<<P.grid, P.threads, P.smem, st>>>((const uint4*)h_in, partial, B, n, d, P.V, P.R, P.L, P.Jmax);
-  return cudaGetLastError();
+  return launch_k(bf16 ? k_pool<true> : k_pool<false>, dim3(P.grid), dim3(P.threads), P.smem, st,
+                  (const uint4*)h_in, partial, status, B, n, d, P.V, P.R, P.L, P.Jmax, P.stage_rows, P.stages,
+                  P.cons_threads);
 }
 
 static cudaError_t launch_project(const PoolPlan& P, const float* partial, const __nv_bfloat16* proj,
                                   const float* center, __nv_bfloat16* fp, float* rq,
                                   uint32_t B, uint32_t n, uint32_t d, uint32_t k, cudaStream_t st) {
-  k_project<<<(B + PROJ_G - 1) / PROJ_G, PROJ_THREADS, project_smem_bytes(d, k, proj != nullptr), st>>>(
-      partial, proj, center, fp, rq, B, n, d, k, P.L, P.Jmax);
-  return cudaGetLastError();
+  return launch_k(k_project, dim3((B + PROJ_G - 1) / PROJ_G), dim3(PROJ_THREADS),
+                  project_smem_bytes(d, k, proj != nullptr), st, partial, proj, center, fp, rq, B, n, d, k, P.L, P.Jmax);
 }
 
 cudaError_t launch_fingerprint(llmcache_bank* bk, const void* h_in, uint32_t B,
@@ -296,7 +374,7 @@ cudaError_t launch_fingerprint(llmcache_bank* bk, const void* h_in, uint32_t B,
   cudaError_t e;
   {
     ProfScope prof(bk, LLMCACHE_K_POOL, st);
-    e = launch_pool(P, bf16, h_in, bk->a.pool_partial, B, D.seq_len, D.d_model, st);
+    e = launch_pool(P, bf16, h_in, bk->a.pool_partial, bk->a.status, B, D.seq_len, D.d_model, st);
   }
   if (e != cudaSuccess) return e;
   ProfScope prof(bk, LLMCACHE_K_PROJECT, st);
@@ -306,8 +384,7 @@ cudaError_t launch_fingerprint(llmcache_bank* bk, const void* h_in, uint32_t B,
 cudaError_t launch_rownorm(llmcache_bank* bk, const __nv_bfloat16* fp, uint32_t B, uint32_t k, float* rq, cudaStream_t st) {
   if (B == 0) return cudaSuccess;
   ProfScope prof(bk, LLMCACHE_K_ROWNORM, st);
-  k_rownorm<<<(B + 7) / 8, 256, 0, st>>>(fp, B, k, rq);
-  return cudaGetLastError();
+  return launch_k(k_rownorm, dim3((B + 7) / 8), dim3(256), 0, st, fp, B, k, rq);
 }
 
 }  // namespace llmc
@@ -323,9 +400,11 @@ namespace {
 
 // Partial sums of the pooling pass, [B, splits, d] floats.  8 MiB per GPU that loads the library.
 static __device__ __align__(256) float g_fp_static_scratch[LLMCACHE_FINGERPRINT_STATIC_MAX_FLOATS];
+// Set by the pooling kernel if one of its bounded waits ever expired (stays zero otherwise).
+static __device__ uint32_t g_fp_static_status;
 
 constexpr int STATIC_MAX_DEVICES = 64;
-struct StaticDev { bool ready = false; float* scratch = nullptr; int sm_count = 0; };
+struct StaticDev { bool ready = false; float* scratch = nullptr; uint32_t* status = nullptr; int sm_count = 0; };
 StaticDev g_static_dev[STATIC_MAX_DEVICES];
 std::mutex g_static_mu;
 thread_local char g_static_err[192] = "";
@@ -340,12 +419,17 @@ cudaError_t static_setup(int dev, StaticDev** out) {
     cudaError_t e = cudaGetSymbolAddress((void**)&ptr, g_fp_static_scratch);
     if (e != cudaSuccess) return e;
     if (!ptr) return cudaErrorInvalidSymbol;
+    uint32_t* sptr = nullptr;
+    e = cudaGetSymbolAddress((void**)&sptr, g_fp_static_status);
+    if (e != cudaSuccess) return e;
+    if (!sptr) return cudaErrorInvalidSymbol;
     int sms = 0;
     e = cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
     if (e != cudaSuccess) return e;
     e = llmc::setup_fingerprint_kernels();
     if (e != cudaSuccess) return e;
     sd.scratch = ptr;
+    sd.status = sptr;
     sd.sm_count = sms;
     sd.ready = true;
   }
@@ -369,7 +453,7 @@ extern "C" int llmcache_fingerprint_static(const void* h_in, uint32_t hidden_dty
     return fail(LLMCACHE_ERR_ARG, "pointers must be 16-byte aligned");
   const bool bf16 = hidden_dtype == LLMCACHE_BF16;
   const uint32_t d = d_model, n = seq_len, k = fp_dim;
-  if (n == 0 || d == 0 || d % 8 != 0 || d > (bf16 ? 8192u : 4096u)) return fail(LLMCACHE_ERR_SHAPE, "d_model not supported");
+  if (n == 0 || d == 0 || d % 8 != 0 || d > (bf16 ? 7680u : 3840u)) return fail(LLMCACHE_ERR_SHAPE, "d_model not supported");
   if (k == 0 || k % 64 != 0 || k > 2048 || (!proj && k != d)) return fail(LLMCACHE_ERR_SHAPE, "fp_dim not supported");
   if (project_smem_bytes(d, k, proj != nullptr) > 200 * 1024) return fail(LLMCACHE_ERR_UNSUPPORTED, "d_model + fp_dim too large");
   if (B == 0) return LLMCACHE_OK;
@@ -394,7 +478,7 @@ extern "C" int llmcache_fingerprint_static(const void* h_in, uint32_t hidden_dty
   cudaStream_t st = (cudaStream_t)stream;
   // every partial sum that the second kernel reads is written by the first one in this call, so
   // nothing in the shared array has to start at zero
-  e = launch_pool(P, bf16, h_in, sd->scratch, B, n, d, st);
+  e = launch_pool(P, bf16, h_in, sd->scratch, sd->status, B, n, d, st);
   if (e == cudaSuccess)
     e = launch_project(P, sd->scratch, (const __nv_bfloat16*)proj, center, (__nv_bfloat16*)fp, rq, B, n, d, k, st);
   if (e != cudaSuccess) return fail(LLMCACHE_ERR_CUDA, cudaGetErrorString(e));

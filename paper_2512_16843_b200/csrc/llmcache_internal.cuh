@@ -39,6 +39,7 @@ struct BankArrays {
   unsigned long long* best; // [max_batch] packed (orderable score << 32 | ~slot); 0 = none
   uint32_t* hitcnt;         // [N] matches per slot within the current probe (zero between calls)
   int32_t*  victims;        // [min(max_batch,N)]
+  int32_t*  new_slot;       // [max_batch] slot each miss of the open probe will be stored in (-1: dropped)
   unsigned long long* sort_key;   // [pow2 >= min(max_batch,N)]
   uint32_t* sort_slot;      // same length
   unsigned long long* stats;      // [ST_COUNT]
@@ -94,7 +95,8 @@ struct ProfScope {
 size_t project_smem_bytes(uint32_t d, uint32_t k, bool has_proj);
 cudaError_t setup_fingerprint_kernels();
 cudaError_t setup_scan_kernels();
-struct PoolPlan { uint32_t V, R, threads, grid, L, Jmax; size_t smem; };
+cudaError_t setup_rows_kernels();
+struct PoolPlan { uint32_t V, R, cons_threads, threads, stage_rows, stages, grid, L, Jmax; size_t smem; };
 PoolPlan pool_plan(uint32_t B, uint32_t n, uint32_t d, bool bf16, int sm_count);
 cudaError_t launch_fingerprint(llmcache_bank* bk, const void* h_in, uint32_t B,
                                __nv_bfloat16* fp, float* rq, cudaStream_t st);
@@ -104,14 +106,38 @@ cudaError_t launch_decide(llmcache_bank* bk, uint32_t B, float tau, const float*
                           const llmcache_probe_io* io, cudaStream_t st);
 cudaError_t launch_gather(llmcache_bank* bk, const void* h_in, void* h_out,
                           const llmcache_probe_io* io, uint32_t B, cudaStream_t st);
-cudaError_t launch_select_victims(llmcache_bank* bk, const llmcache_probe_io* io, uint32_t B,
-                                  int32_t* new_slot, cudaStream_t st);
 cudaError_t launch_scatter_insert(llmcache_bank* bk, const void* miss_out, const llmcache_probe_io* io,
-                                  void* h_out, const int32_t* new_slot, uint32_t B, cudaStream_t st);
+                                  void* h_out, int32_t* new_slot_out, uint32_t B, cudaStream_t st);
 cudaError_t launch_evict(llmcache_bank* bk, uint32_t mode, const int32_t* slots, uint32_t n,
                          uint32_t* n_evicted, cudaStream_t st);
 
+// Launch with programmatic dependent launch allowed: the grid may be scheduled while its predecessor
+// in the stream is still running; every kernel starts with griddep_sync(), which waits until the
+// predecessor has completed and its writes are visible, so only launch latency is overlapped.
+template <typename... KArgs, typename... Args>
+inline cudaError_t launch_k(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t st,
+                            Args&&... args) {
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = grid;
+  cfg.blockDim = block;
+  cfg.dynamicSmemBytes = smem;
+  cfg.stream = st;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[0].val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = 1;
+  return cudaLaunchKernelEx(&cfg, kernel, KArgs(args)...);
+}
+
 // ---- small device helpers ---------------------------------------------------
+// First statement of every kernel: wait for the previous grid of the stream, then let the next one
+// be scheduled.
+__device__ __forceinline__ void griddep_sync() {
+  asm volatile("griddepcontrol.wait;" ::: "memory");
+  asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+}
+
 __device__ __forceinline__ uint32_t float_orderable(float f) {
   uint32_t u = __float_as_uint(f);
   return (u & 0x80000000u) ? ~u : (u | 0x80000000u);

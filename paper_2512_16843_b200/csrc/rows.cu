@@ -8,10 +8,11 @@
 // block moves the same number of bytes whatever the hit / miss counts are (they
 // are only known on the device).
 #include "llmcache_internal.cuh"
+#include "select.cuh"
 
 namespace llmc {
 
-constexpr int COPY_THREADS = 256;
+constexpr int COPY_THREADS = SEL_THREADS;         // 512: the gather kernel's last block runs the victim selection
 constexpr int COPY_UNROLL = 8;                       // 16-byte vectors in flight per thread
 constexpr uint32_t COPY_UNIT = 4096;                 // bytes
 
@@ -37,25 +38,34 @@ __device__ __forceinline__ void copy_bytes(const char* __restrict__ src, char* _
   }
 }
 
-__device__ __forceinline__ void block_span(unsigned long long total, unsigned long long& u0, unsigned long long& u1) {
-  u0 = total * blockIdx.x / gridDim.x;
-  u1 = total * (blockIdx.x + 1) / gridDim.x;
+__device__ __forceinline__ void block_span(unsigned long long total, uint32_t n_blocks,
+                                           unsigned long long& u0, unsigned long long& u1) {
+  u0 = total * blockIdx.x / n_blocks;
+  u1 = total * (blockIdx.x + 1) / n_blocks;
 }
 
 // Units [0, H*upr): hit rows bank.act[slot] -> h_out[b].
 // Units after that (only if h_miss): miss inputs h_in[b] -> h_miss[m].
+// The last block of the grid moves nothing: it chooses, while the others copy, the slots that the
+// misses of this batch will be stored in at commit (Sec. III-E / IV-D); the choice depends only on
+// the bank's metadata after this probe's refresh, which the copy does not touch.
 __global__ void __launch_bounds__(COPY_THREADS)
 k_gather(const char* __restrict__ act, uint32_t act_rows, char* __restrict__ h_out, size_t row_bytes,
          const char* __restrict__ h_in, char* __restrict__ h_miss, size_t in_row_bytes,
          const int32_t* __restrict__ slot, const int32_t* __restrict__ hit_idx,
-         const int32_t* __restrict__ miss_idx, const uint32_t* __restrict__ counts) {
+         const int32_t* __restrict__ miss_idx, const uint32_t* __restrict__ counts, SelectArgs sel) {
+  griddep_sync();
+  if (blockIdx.x == gridDim.x - 1) {
+    select_victims_block(sel);
+    return;
+  }
   const uint32_t H = counts[0], M = counts[1];
   const uint32_t upr = (uint32_t)((row_bytes + COPY_UNIT - 1) / COPY_UNIT);
   const uint32_t upr_in = (uint32_t)((in_row_bytes + COPY_UNIT - 1) / COPY_UNIT);
   const unsigned long long n_hit = (act && h_out) ? (unsigned long long)H * upr : 0ull;
   const unsigned long long total = n_hit + ((h_in && h_miss) ? (unsigned long long)M * upr_in : 0ull);
   unsigned long long u, u1;
-  block_span(total, u, u1);
+  block_span(total, gridDim.x - 1, u, u1);
   while (u < u1) {
     if (u < n_hit) {
       const uint32_t i = (uint32_t)(u / upr), w0 = (uint32_t)(u - (unsigned long long)i * upr);
@@ -89,13 +99,25 @@ k_scatter_insert(const char* __restrict__ miss_out, char* __restrict__ h_out, ch
                  const uint4* __restrict__ q_fp, const float* __restrict__ rq, uint32_t k,
                  uint4* __restrict__ bank_fp, float* __restrict__ rb, uint8_t* __restrict__ valid,
                  uint32_t* __restrict__ last_use, uint32_t* __restrict__ insert_tick, uint32_t* __restrict__ hits,
-                 uint32_t* __restrict__ rate, uint32_t* __restrict__ rate_epoch, uint32_t tick, uint32_t epoch) {
+                 uint32_t* __restrict__ rate, uint32_t* __restrict__ rate_epoch, uint32_t tick, uint32_t epoch,
+                 int32_t* __restrict__ new_slot_out, const uint32_t* __restrict__ tally,
+                 unsigned long long* __restrict__ stats) {
+  griddep_sync();
   const uint32_t M = counts[1];
+  if (blockIdx.x == 0) {
+    if (new_slot_out)
+      for (uint32_t m = threadIdx.x; m < M; m += COPY_THREADS) new_slot_out[m] = new_slot[m];
+    if (threadIdx.x == 0) {
+      stats[ST_INSERT] += tally[0];
+      stats[ST_EVICT] += tally[1];
+      stats[ST_DROP] += tally[2];
+    }
+  }
   const uint32_t upr = (uint32_t)((row_bytes + COPY_UNIT - 1) / COPY_UNIT);
   const unsigned long long total = (unsigned long long)M * upr;
   const uint32_t kv = k / 8;                      // 16-byte vectors per fingerprint row
   unsigned long long u, u1;
-  block_span(total, u, u1);
+  block_span(total, gridDim.x, u, u1);
   while (u < u1) {
     const uint32_t m = (uint32_t)(u / upr), w0 = (uint32_t)(u - (unsigned long long)m * upr);
     const uint32_t w1 = (uint32_t)min((unsigned long long)upr, w0 + (u1 - u));
@@ -123,10 +145,20 @@ k_scatter_insert(const char* __restrict__ miss_out, char* __restrict__ h_out, ch
   }
 }
 
-// Four blocks per SM, but never more blocks than there could be units of work.
-static uint32_t copy_grid(const llmcache_bank* bk, uint32_t B, size_t row_bytes) {
+static int g_gather_occ = 0, g_scatter_occ = 0;      // resident blocks per SM, from the occupancy calculator
+
+cudaError_t setup_rows_kernels() {
+  cudaError_t e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&g_gather_occ, k_gather, COPY_THREADS, 0);
+  if (e == cudaSuccess) e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&g_scatter_occ, k_scatter_insert, COPY_THREADS, 0);
+  if (g_gather_occ < 1) g_gather_occ = 1;
+  if (g_scatter_occ < 1) g_scatter_occ = 1;
+  return e;
+}
+
+// One wave of resident blocks, but never more blocks than there could be units of work.
+static uint32_t copy_grid(const llmcache_bank* bk, uint32_t B, size_t row_bytes, int occ) {
   const unsigned long long units = (unsigned long long)B * ((row_bytes + COPY_UNIT - 1) / COPY_UNIT);
-  unsigned long long g = (unsigned long long)bk->sm_count * 4;
+  unsigned long long g = (unsigned long long)bk->sm_count * (unsigned long long)occ;
   if (units < g) g = units;
   return g ? (uint32_t)g : 1u;
 }
@@ -139,26 +171,43 @@ cudaError_t launch_gather(llmcache_bank* bk, const void* h_in, void* h_out,
   const size_t in_row_bytes = (size_t)D.seq_len * D.d_model * (D.hidden_dtype == LLMCACHE_BF16 ? 2 : 4);
   const bool want_miss = h_in && io->h_miss;
   const bool want_hit = bk->a.act && h_out;
-  if (!want_miss && !want_hit) return cudaSuccess;
+  SelectArgs sel;
+  sel.mv = MetaView{bk->a.valid, bk->a.last_use, bk->a.insert_tick, bk->a.rate, bk->a.rate_epoch};
+  sel.pol = bk->pol;
+  sel.N = D.capacity;
+  sel.tick = (uint32_t)bk->tick;
+  sel.epoch = (uint32_t)(bk->tick / bk->pol.half_life);
+  sel.miss_idx = io->miss_idx;
+  sel.rq = io->rq;
+  sel.counts = io->counts;
+  sel.new_slot = bk->a.new_slot;
+  sel.victims = bk->a.victims;
+  sel.g_key = bk->a.sort_key;
+  sel.g_val = bk->a.sort_slot;
+  sel.sort_cap = bk->sort_len;
+  sel.tally = bk->a.misc;
+  const uint32_t copy_blocks = (want_miss || want_hit) ? copy_grid(bk, B, in_row_bytes, g_gather_occ) : 1u;
   ProfScope prof(bk, LLMCACHE_K_GATHER, st);
-  k_gather<<<copy_grid(bk, B, in_row_bytes), COPY_THREADS, 0, st>>>(
-      (const char*)bk->a.act, D.act_rows, (char*)h_out, row_bytes,
-      (const char*)h_in, (char*)io->h_miss, in_row_bytes, io->slot, io->hit_idx, io->miss_idx, io->counts);
-  return cudaGetLastError();
+  return launch_k(k_gather, dim3(copy_blocks + 1), dim3(COPY_THREADS), 0, st,
+                  (const char*)(want_hit ? bk->a.act : nullptr), D.act_rows, (char*)(want_hit ? h_out : nullptr), row_bytes,
+                  (const char*)(want_miss ? h_in : nullptr), (char*)(want_miss ? io->h_miss : nullptr), in_row_bytes,
+                  (const int32_t*)io->slot, (const int32_t*)io->hit_idx, (const int32_t*)io->miss_idx,
+                  (const uint32_t*)io->counts, sel);
 }
 
 cudaError_t launch_scatter_insert(llmcache_bank* bk, const void* miss_out, const llmcache_probe_io* io,
-                                  void* h_out, const int32_t* new_slot, uint32_t B, cudaStream_t st) {
+                                  void* h_out, int32_t* new_slot_out, uint32_t B, cudaStream_t st) {
   if (B == 0) return cudaSuccess;
   const llmcache_bank_desc& D = bk->desc;
   const size_t row_bytes = (size_t)D.seq_len * D.d_model * 2;
   const uint32_t epoch = (uint32_t)(bk->tick / bk->pol.half_life);
   ProfScope prof(bk, LLMCACHE_K_SCATTER, st);
-  k_scatter_insert<<<copy_grid(bk, B, row_bytes), COPY_THREADS, 0, st>>>(
-      (const char*)miss_out, (char*)h_out, (char*)bk->a.act, row_bytes, io->miss_idx, new_slot, io->counts,
-      (const uint4*)io->fp, io->rq, D.fp_dim, (uint4*)bk->a.fp, bk->a.rb, bk->a.valid,
-      bk->a.last_use, bk->a.insert_tick, bk->a.hits, bk->a.rate, bk->a.rate_epoch, (uint32_t)bk->tick, epoch);
-  return cudaGetLastError();
+  return launch_k(k_scatter_insert, dim3(copy_grid(bk, B, row_bytes, g_scatter_occ)), dim3(COPY_THREADS), 0, st,
+                  (const char*)miss_out, (char*)h_out, (char*)bk->a.act, row_bytes, (const int32_t*)io->miss_idx,
+                  (const int32_t*)bk->a.new_slot, (const uint32_t*)io->counts, (const uint4*)io->fp,
+                  (const float*)io->rq, D.fp_dim, (uint4*)bk->a.fp, bk->a.rb, bk->a.valid, bk->a.last_use,
+                  bk->a.insert_tick, bk->a.hits, bk->a.rate, bk->a.rate_epoch, (uint32_t)bk->tick, epoch,
+                  new_slot_out, (const uint32_t*)bk->a.misc, bk->a.stats);
 }
 
 }  // namespace llmc

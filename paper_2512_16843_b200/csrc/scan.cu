@@ -21,6 +21,7 @@
 // frees its tensor memory and returns.
 #include <cuda.h>
 #include "llmcache_internal.cuh"
+#include "ptx.cuh"
 
 namespace llmc {
 
@@ -33,7 +34,6 @@ constexpr int SCAN_THREADS = 192;  // warp 0: TMA, warp 1: MMA + TMEM owner, war
 constexpr uint32_t A_BYTES = BM * BK * 2;   // 16 KB
 constexpr uint32_t B_BYTES = BN * BK * 2;   // 32 KB
 constexpr uint32_t TMEM_COLS = 512;         // two accumulators of 256 columns
-constexpr unsigned long long WAIT_LIMIT_NS = 2000000000ull;
 
 struct ScanSmem {
   // offsets from the 1024-byte aligned base of dynamic shared memory
@@ -46,43 +46,7 @@ struct ScanSmem {
 };
 constexpr uint32_t SCAN_SMEM_BYTES = ScanSmem::TOTAL + 1024;    // slack for manual alignment
 
-// ---- PTX wrappers -----------------------------------------------------------
-__device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
-
-__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
-  asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count) : "memory");
-}
-__device__ __forceinline__ void mbar_arrive(uint32_t bar) {
-  asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
-}
-__device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes) {
-  asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
-}
-__device__ __forceinline__ unsigned long long global_ns() {
-  unsigned long long t;
-  asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
-  return t;
-}
-// Bounded wait for the phase with the given parity.  Returns false on expiry or abort.
-__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile uint32_t* abort_flag,
-                                          unsigned long long limit_ns = WAIT_LIMIT_NS) {
-  unsigned long long t0 = 0;
-  for (uint32_t spin = 0;; ++spin) {
-    uint32_t done;
-    asm volatile(
-        "{\n\t.reg .pred p;\n\t"
-        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
-        "selp.u32 %0, 1, 0, p;\n\t}"
-        : "=r"(done) : "r"(bar), "r"(parity) : "memory");
-    if (done) return true;
-    if ((spin & 255u) == 255u) {
-      if (*abort_flag) return false;
-      const unsigned long long now = global_ns();
-      if (t0 == 0) t0 = now;
-      else if (now - t0 > limit_ns) return false;
-    }
-  }
-}
+// ---- PTX wrappers (mbarrier helpers come from ptx.cuh) ---------------------
 __device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* map, int c0, int c1, uint32_t bar) {
   asm volatile(
       "cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];"
@@ -134,6 +98,7 @@ k_scan_tc(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CUt
           const float* __restrict__ rb, const uint8_t* __restrict__ valid,
           unsigned long long* __restrict__ best, uint32_t* __restrict__ status,
           uint32_t B, uint32_t N, uint32_t KB, uint32_t MB, uint32_t NB, uint32_t chunk_len, uint32_t n_units) {
+  griddep_sync();
   extern __shared__ uint8_t smem_raw[];
   const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;
   uint8_t* gbase = smem_raw + (base - smem_u32(smem_raw));
@@ -330,9 +295,9 @@ cudaError_t launch_scan(llmcache_bank* bk, const __nv_bfloat16* q, uint32_t B, c
   const uint32_t n_units = MB * chunks;
   const uint32_t grid = n_units < (uint32_t)bk->sm_count ? n_units : (uint32_t)bk->sm_count;
   ProfScope prof(bk, LLMCACHE_K_SCAN, st);
-  k_scan_tc<<<grid, SCAN_THREADS, SCAN_SMEM_BYTES, st>>>(map_q, map_bank, bk->a.rb, bk->a.valid, bk->a.best,
-                                                        bk->a.status, B, N, KB, MB, NB, chunk_len, n_units);
-  return cudaGetLastError();
+  return launch_k(k_scan_tc, dim3(grid), dim3(SCAN_THREADS), SCAN_SMEM_BYTES, st, map_q, map_bank,
+                  (const float*)bk->a.rb, (const uint8_t*)bk->a.valid, bk->a.best, bk->a.status, B, N, KB, MB, NB,
+                  chunk_len, n_units);
 }
 
 }  // namespace llmc
