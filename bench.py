@@ -117,6 +117,25 @@ class ClockSampler:
 
 
 # ------------------------------------------------------------------------------------------------
+def rank_seed(rank):
+    """Every rank (one per GPU) draws its own banks and batches: replicas share no data."""
+    from paper_2512_16843_b200 import synth
+    return synth.BASE_SEED + 2000 + 100000 * rank
+
+
+def aggregate(ms_local, seqs_local, dist=None, device="cpu"):
+    """Whole-job figures from one rank's: time = max over ranks, work = sum over ranks.
+    Returns (ms, sequences, sequences per second)."""
+    ms, seqs = float(ms_local), float(seqs_local)
+    if dist is not None and dist.is_initialized() and dist.get_world_size() > 1:
+        t = torch.tensor([ms], dtype=torch.float64, device=device)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        w = torch.tensor([seqs], dtype=torch.float64, device=device)
+        dist.all_reduce(w, op=dist.ReduceOp.SUM)
+        ms, seqs = float(t.item()), float(w.item())
+    return ms, seqs, seqs / (ms * 1e-3)
+
+
 def build_batches(wl, seeds_tok, count, seed, device):
     """`count` batches of hidden states: 60% edits of the seeds, 40% fresh, shuffled."""
     from paper_2512_16843_b200 import synth
@@ -151,7 +170,7 @@ def run_ours(args):
     if args.pool_batches:
         CFG["pool_batches"] = args.pool_batches
     Lyr, d, n, B, N, k = (CFG[x] for x in ("layers", "d_model", "seq_len", "batch", "bank", "fp_dim"))
-    seed = synth.BASE_SEED + 2000 + 100000 * rank
+    seed = rank_seed(rank)
     wl = synth.TokenWorkload(CFG["vocab"], n, d, seed, dev)
     seeds_tok = wl.tokens(CFG["n_seeds"], seed + 5)
     proj = synth.projection(d, k, seed + 6, dev)
@@ -214,22 +233,21 @@ def run_ours(args):
         one_step()
     e1.record()
     barrier()
-    ms = e0.elapsed_time(e1)
     clocks = sampler.stop() if rank == 0 else None
-    if dist is not None:
-        t = torch.tensor([ms], device=dev)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        ms = float(t.item())
+    seqs = B * Lyr * args.steps
+    ms, _, value = aggregate(e0.elapsed_time(e1), seqs, dist, dev)
     launches = sum(b.stats()["kernel_launches"] for b in banks) - launches0
     hits = sum(b.stats()["hits"] for b in banks) - hits0
-    seqs = B * Lyr * args.steps
-    value = world * seqs / (ms * 1e-3)
 
     # ---- per-kernel device time over the same loop (events around every launch) -------------------
+    # The GPU is held back by a ~2 ms spin before every step so that the host has the whole step enqueued
+    # before it starts: the event pairs then bracket kernel execution, not the host's enqueue rate.
     for b in banks:
         b.profile(True)
     st0 = [b.stats() for b in banks]
-    for _ in range(args.steps):
+    prof_steps = min(args.steps, 50)
+    for _ in range(prof_steps):
+        torch.cuda._sleep(4000000)
         one_step()
     torch.cuda.synchronize()
     prof = {}
@@ -240,7 +258,7 @@ def run_ours(args):
             a[0] += tms
             a[1] += cnt
     st1 = [b.stats() for b in banks]
-    H_avg = sum(s1["hits"] - s0["hits"] for s0, s1 in zip(st0, st1)) / float(Lyr * args.steps)
+    H_avg = sum(s1["hits"] - s0["hits"] for s0, s1 in zip(st0, st1)) / float(Lyr * prof_steps)
     M_avg = B - H_avg
     row = n * d * 2
     algo_bytes = {                                       # algorithmic bytes per launch
@@ -278,12 +296,8 @@ def run_ours(args):
             one_step(host_pool, stage, results)
         e1.record()
         barrier()
-        ems = e0.elapsed_time(e1)
-        if dist is not None:
-            t = torch.tensor([ems], device=dev)
-            dist.all_reduce(t, op=dist.ReduceOp.MAX)
-            ems = float(t.item())
-        e2e = {"value": world * B * Lyr * args.e2e_steps / (ems * 1e-3), "unit": UNIT,
+        ems, _, e2e_value = aggregate(e0.elapsed_time(e1), B * Lyr * args.e2e_steps, dist, dev)
+        e2e = {"value": e2e_value, "unit": UNIT,
                "h2d_bytes_per_step": Lyr * B * n * d * 2, "d2h_bytes_per_step": Lyr * B * 9 + Lyr * 8,
                "steps": args.e2e_steps}
         del host_pool
