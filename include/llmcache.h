@@ -132,9 +132,8 @@ enum {
   LLMCACHE_K_SCAN = 3,      /* Sec. III-C cosine scan + best slot                  */
   LLMCACHE_K_DECIDE = 4,    /* Sec. IV-A threshold + hit/miss compaction           */
   LLMCACHE_K_TOUCH = 5,     /* (unused: the metadata refresh runs inside DECIDE)  */
-  LLMCACHE_K_GATHER = 6,    /* Algorithm 1 reuse: copy of cached outputs; one block of it
-                               also picks the victims for the commit (Sec. IV-D)   */
-  LLMCACHE_K_SELECT = 7,    /* (unused: victim selection runs inside GATHER)       */
+  LLMCACHE_K_GATHER = 6,    /* Algorithm 1 reuse: copy of cached outputs           */
+  LLMCACHE_K_SELECT = 7,    /* Sec. IV-D victim selection (side stream, during GATHER) */
   LLMCACHE_K_SCATTER = 8,   /* Algorithm 1 insert: write-back + store              */
   LLMCACHE_K_EVICT = 9,     /* Sec. III-E flushes                                  */
   LLMCACHE_K_COUNT = 10

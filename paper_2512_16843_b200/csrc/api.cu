@@ -227,8 +227,14 @@ int llmcache_bank_create(const llmcache_bank_desc* desc, llmcache_bank_t** bank_
   if (e == cudaSuccess) e = setup_fingerprint_kernels();
   if (e == cudaSuccess) e = setup_scan_kernels();
   if (e == cudaSuccess) e = setup_rows_kernels();
+  if (e == cudaSuccess) e = cudaStreamCreateWithFlags(&bk->side, cudaStreamNonBlocking);
+  if (e == cudaSuccess) e = cudaEventCreateWithFlags(&bk->ev_fork, cudaEventDisableTiming);
+  if (e == cudaSuccess) e = cudaEventCreateWithFlags(&bk->ev_join, cudaEventDisableTiming);
   if (e == cudaSuccess) e = cudaDeviceSynchronize();
   if (e != cudaSuccess) {
+    if (bk->side) cudaStreamDestroy(bk->side);
+    if (bk->ev_fork) cudaEventDestroy(bk->ev_fork);
+    if (bk->ev_join) cudaEventDestroy(bk->ev_join);
     if (bk->owns_memory) cudaFree(bk->base);
     delete bk;
     return cuda_fail(e, "bank_create");
@@ -242,6 +248,9 @@ int llmcache_bank_destroy(llmcache_bank_t* bk) {
   DeviceGuard guard(bk->desc.device);
   if (!guard.ok) return LLMCACHE_ERR_CUDA;
   cudaError_t e = cudaDeviceSynchronize();
+  if (bk->side) cudaStreamDestroy(bk->side);
+  if (bk->ev_fork) cudaEventDestroy(bk->ev_fork);
+  if (bk->ev_join) cudaEventDestroy(bk->ev_join);
   if (bk->owns_memory && bk->base) cudaFree(bk->base);
   for (int i = 0; i < LLMCACHE_K_COUNT; ++i)
     for (auto& ev : bk->prof_used[i]) bk->prof_free.push_back(ev);
@@ -284,6 +293,11 @@ static int probe_common(llmcache_bank_t* bk, const void* h_in, bool compute_fp, 
   bk->probe_open = true;
   bk->last_B = B;
   cudaError_t e = cudaSuccess;
+  if (bk->join_pending) {          // a previous probe was never committed: its victim selection must be over
+    e = cudaStreamWaitEvent(st, bk->ev_join, 0);
+    bk->join_pending = false;
+  }
+  if (e != cudaSuccess) return cuda_fail(e, __func__);
   if (B == 0) {
     if (io->counts) e = cudaMemsetAsync(io->counts, 0, 2 * sizeof(uint32_t), st);
   } else {
@@ -291,6 +305,13 @@ static int probe_common(llmcache_bank_t* bk, const void* h_in, bool compute_fp, 
     else            e = launch_rownorm(bk, (const __nv_bfloat16*)io->fp, B, bk->desc.fp_dim, io->rq, st);
     if (e == cudaSuccess) e = launch_scan(bk, (const __nv_bfloat16*)io->fp, B, st);
     if (e == cudaSuccess) e = launch_decide(bk, B, tau, io->rq, io, st);
+    // The slots for this batch's misses are chosen now, on the side stream, while the gather runs:
+    // the choice depends only on the metadata after this probe's refresh, which the gather does not touch.
+    if (e == cudaSuccess) e = cudaEventRecord(bk->ev_fork, st);
+    if (e == cudaSuccess) e = cudaStreamWaitEvent(bk->side, bk->ev_fork, 0);
+    if (e == cudaSuccess) e = launch_select_victims(bk, io, B, bk->side);
+    if (e == cudaSuccess) e = cudaEventRecord(bk->ev_join, bk->side);
+    if (e == cudaSuccess) bk->join_pending = true;
     if (e == cudaSuccess) e = launch_gather(bk, h_in, h_out, io, B, st);
   }
   if (e == cudaSuccess && io->counts_host && io->counts)
@@ -326,8 +347,13 @@ int llmcache_commit(llmcache_bank_t* bk, const void* miss_out, const llmcache_pr
   cudaStream_t st = (cudaStream_t)stream;
   bk->probe_open = false;
   if (B == 0) return LLMCACHE_OK;
-  // the slots were chosen during the probe (inside the gather kernel); here the rows move
-  cudaError_t e = launch_scatter_insert(bk, miss_out, io, h_out, new_slot, B, st);
+  // the slots were chosen during the probe (side stream); here the rows move
+  cudaError_t e = cudaSuccess;
+  if (bk->join_pending) {
+    e = cudaStreamWaitEvent(st, bk->ev_join, 0);
+    bk->join_pending = false;
+  }
+  if (e == cudaSuccess) e = launch_scatter_insert(bk, miss_out, io, h_out, new_slot, B, st);
   if (e != cudaSuccess) return cuda_fail(e, __func__);
   return LLMCACHE_OK;
 }

@@ -1,6 +1,7 @@
-// Explicit flushes of the replacement controller (Sec. III-E: "temporal decay factors are used to
-// flush outdated fingerprints").  Victim selection for inserts lives in select.cuh.
+// Replacement controller kernels (Sec. III-E, IV-D): the victim selection for inserts (routine in
+// select.cuh) and the explicit flushes ("temporal decay factors are used to flush outdated fingerprints").
 #include "llmcache_internal.cuh"
+#include "select.cuh"
 
 namespace llmc {
 
@@ -37,6 +38,31 @@ __global__ void k_evict(uint8_t* __restrict__ valid, const uint32_t* __restrict_
     if (n_evicted) atomicAdd(n_evicted, c);
     atomicAdd(stats + ST_FLUSH, (unsigned long long)c);
   }
+}
+
+// One block.  Runs on the bank's side stream, next to the gather of the same probe.
+__global__ void __launch_bounds__(SEL_THREADS) k_select_victims(SelectArgs A) { select_victims_block(A); }
+
+cudaError_t launch_select_victims(llmcache_bank* bk, const llmcache_probe_io* io, uint32_t B, cudaStream_t st) {
+  if (B == 0) return cudaSuccess;
+  SelectArgs sel;
+  sel.mv = MetaView{bk->a.valid, bk->a.last_use, bk->a.insert_tick, bk->a.rate, bk->a.rate_epoch};
+  sel.pol = bk->pol;
+  sel.N = bk->desc.capacity;
+  sel.tick = (uint32_t)bk->tick;
+  sel.epoch = (uint32_t)(bk->tick / bk->pol.half_life);
+  sel.miss_idx = io->miss_idx;
+  sel.rq = io->rq;
+  sel.counts = io->counts;
+  sel.new_slot = bk->a.new_slot;
+  sel.victims = bk->a.victims;
+  sel.g_key = bk->a.sort_key;
+  sel.g_val = bk->a.sort_slot;
+  sel.sort_cap = bk->sort_len;
+  sel.tally = bk->a.misc;
+  ProfScope prof(bk, LLMCACHE_K_SELECT, st);
+  k_select_victims<<<1, SEL_THREADS, 0, st>>>(sel);
+  return cudaGetLastError();
 }
 
 cudaError_t launch_evict(llmcache_bank* bk, uint32_t mode, const int32_t* slots, uint32_t n,

@@ -66,6 +66,10 @@ struct llmcache_bank {
   // TMA descriptor of the fingerprint matrix (opaque 128-byte blob)
   alignas(64) unsigned char tmap_bank[128] = {};
   bool     has_tmap = false;
+  // side stream on which the victim selection of a probe runs next to its gather
+  cudaStream_t side = nullptr;
+  cudaEvent_t  ev_fork = nullptr, ev_join = nullptr;
+  bool     join_pending = false;
   // instrumentation
   uint64_t n_launches = 0;
   bool     prof_on = false;
@@ -106,6 +110,7 @@ cudaError_t launch_decide(llmcache_bank* bk, uint32_t B, float tau, const float*
                           const llmcache_probe_io* io, cudaStream_t st);
 cudaError_t launch_gather(llmcache_bank* bk, const void* h_in, void* h_out,
                           const llmcache_probe_io* io, uint32_t B, cudaStream_t st);
+cudaError_t launch_select_victims(llmcache_bank* bk, const llmcache_probe_io* io, uint32_t B, cudaStream_t st);
 cudaError_t launch_scatter_insert(llmcache_bank* bk, const void* miss_out, const llmcache_probe_io* io,
                                   void* h_out, int32_t* new_slot_out, uint32_t B, cudaStream_t st);
 cudaError_t launch_evict(llmcache_bank* bk, uint32_t mode, const int32_t* slots, uint32_t n,

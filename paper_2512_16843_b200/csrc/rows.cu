@@ -8,33 +8,37 @@
 // block moves the same number of bytes whatever the hit / miss counts are (they
 // are only known on the device).
 #include "llmcache_internal.cuh"
-#include "select.cuh"
 
 namespace llmc {
 
-constexpr int COPY_THREADS = SEL_THREADS;         // 512: the gather kernel's last block runs the victim selection
+constexpr int COPY_THREADS = 256;
 constexpr int COPY_UNROLL = 8;                       // 16-byte vectors in flight per thread
 constexpr uint32_t COPY_UNIT = 4096;                 // bytes
 
-// Copy `bytes` (multiple of 16) from src to up to two destinations.
+// Copy `bytes` (multiple of 16) from src to up to two destinations: whole tiles of
+// COPY_THREADS * COPY_UNROLL vectors with all loads issued before the stores, then the rest.
 __device__ __forceinline__ void copy_bytes(const char* __restrict__ src, char* __restrict__ d0,
                                            char* __restrict__ d1, uint32_t bytes) {
-  const uint32_t nvec = bytes >> 4;
-  for (uint32_t base = 0; base < nvec; base += COPY_THREADS * COPY_UNROLL) {
+  constexpr uint32_t TILE = COPY_THREADS * COPY_UNROLL * 16;          // 32 KB
+  uint32_t done = 0;
+  for (; done + TILE <= bytes; done += TILE) {
+    const size_t base = (size_t)done + ((size_t)threadIdx.x << 4);
     uint4 v[COPY_UNROLL];
 #pragma unroll
-    for (int u = 0; u < COPY_UNROLL; ++u) {
-      const uint32_t i = base + u * COPY_THREADS + threadIdx.x;
-      if (i < nvec) v[u] = ld_stream16(src + ((size_t)i << 4));
-    }
+    for (int u = 0; u < COPY_UNROLL; ++u) v[u] = ld_stream16(src + base + (size_t)u * (COPY_THREADS * 16));
+    if (d0) {
 #pragma unroll
-    for (int u = 0; u < COPY_UNROLL; ++u) {
-      const uint32_t i = base + u * COPY_THREADS + threadIdx.x;
-      if (i < nvec) {
-        if (d0) st_stream16(d0 + ((size_t)i << 4), v[u]);
-        if (d1) st_stream16(d1 + ((size_t)i << 4), v[u]);
-      }
+      for (int u = 0; u < COPY_UNROLL; ++u) st_stream16(d0 + base + (size_t)u * (COPY_THREADS * 16), v[u]);
     }
+    if (d1) {
+#pragma unroll
+      for (int u = 0; u < COPY_UNROLL; ++u) st_stream16(d1 + base + (size_t)u * (COPY_THREADS * 16), v[u]);
+    }
+  }
+  for (uint32_t off = done + (threadIdx.x << 4); off < bytes; off += COPY_THREADS * 16) {
+    const uint4 v = ld_stream16(src + off);
+    if (d0) st_stream16(d0 + off, v);
+    if (d1) st_stream16(d1 + off, v);
   }
 }
 
@@ -46,26 +50,19 @@ __device__ __forceinline__ void block_span(unsigned long long total, uint32_t n_
 
 // Units [0, H*upr): hit rows bank.act[slot] -> h_out[b].
 // Units after that (only if h_miss): miss inputs h_in[b] -> h_miss[m].
-// The last block of the grid moves nothing: it chooses, while the others copy, the slots that the
-// misses of this batch will be stored in at commit (Sec. III-E / IV-D); the choice depends only on
-// the bank's metadata after this probe's refresh, which the copy does not touch.
-__global__ void __launch_bounds__(COPY_THREADS)
+__global__ void __launch_bounds__(COPY_THREADS, 6)
 k_gather(const char* __restrict__ act, uint32_t act_rows, char* __restrict__ h_out, size_t row_bytes,
          const char* __restrict__ h_in, char* __restrict__ h_miss, size_t in_row_bytes,
          const int32_t* __restrict__ slot, const int32_t* __restrict__ hit_idx,
-         const int32_t* __restrict__ miss_idx, const uint32_t* __restrict__ counts, SelectArgs sel) {
+         const int32_t* __restrict__ miss_idx, const uint32_t* __restrict__ counts) {
   griddep_sync();
-  if (blockIdx.x == gridDim.x - 1) {
-    select_victims_block(sel);
-    return;
-  }
   const uint32_t H = counts[0], M = counts[1];
   const uint32_t upr = (uint32_t)((row_bytes + COPY_UNIT - 1) / COPY_UNIT);
   const uint32_t upr_in = (uint32_t)((in_row_bytes + COPY_UNIT - 1) / COPY_UNIT);
   const unsigned long long n_hit = (act && h_out) ? (unsigned long long)H * upr : 0ull;
   const unsigned long long total = n_hit + ((h_in && h_miss) ? (unsigned long long)M * upr_in : 0ull);
   unsigned long long u, u1;
-  block_span(total, gridDim.x - 1, u, u1);
+  block_span(total, gridDim.x, u, u1);
   while (u < u1) {
     if (u < n_hit) {
       const uint32_t i = (uint32_t)(u / upr), w0 = (uint32_t)(u - (unsigned long long)i * upr);
@@ -92,7 +89,7 @@ k_gather(const char* __restrict__ act, uint32_t act_rows, char* __restrict__ h_o
 
 // Units of miss_out[m] -> h_out[miss_idx[m]] and -> act[new_slot[m]].  The block whose span holds
 // the first unit of a row also writes the key and the metadata of the new entry.
-__global__ void __launch_bounds__(COPY_THREADS)
+__global__ void __launch_bounds__(COPY_THREADS, 6)
 k_scatter_insert(const char* __restrict__ miss_out, char* __restrict__ h_out, char* __restrict__ act,
                  size_t row_bytes, const int32_t* __restrict__ miss_idx, const int32_t* __restrict__ new_slot,
                  const uint32_t* __restrict__ counts,
@@ -171,28 +168,13 @@ cudaError_t launch_gather(llmcache_bank* bk, const void* h_in, void* h_out,
   const size_t in_row_bytes = (size_t)D.seq_len * D.d_model * (D.hidden_dtype == LLMCACHE_BF16 ? 2 : 4);
   const bool want_miss = h_in && io->h_miss;
   const bool want_hit = bk->a.act && h_out;
-  SelectArgs sel;
-  sel.mv = MetaView{bk->a.valid, bk->a.last_use, bk->a.insert_tick, bk->a.rate, bk->a.rate_epoch};
-  sel.pol = bk->pol;
-  sel.N = D.capacity;
-  sel.tick = (uint32_t)bk->tick;
-  sel.epoch = (uint32_t)(bk->tick / bk->pol.half_life);
-  sel.miss_idx = io->miss_idx;
-  sel.rq = io->rq;
-  sel.counts = io->counts;
-  sel.new_slot = bk->a.new_slot;
-  sel.victims = bk->a.victims;
-  sel.g_key = bk->a.sort_key;
-  sel.g_val = bk->a.sort_slot;
-  sel.sort_cap = bk->sort_len;
-  sel.tally = bk->a.misc;
-  const uint32_t copy_blocks = (want_miss || want_hit) ? copy_grid(bk, B, in_row_bytes, g_gather_occ) : 1u;
+  if (!want_miss && !want_hit) return cudaSuccess;
   ProfScope prof(bk, LLMCACHE_K_GATHER, st);
-  return launch_k(k_gather, dim3(copy_blocks + 1), dim3(COPY_THREADS), 0, st,
+  return launch_k(k_gather, dim3(copy_grid(bk, B, in_row_bytes, g_gather_occ)), dim3(COPY_THREADS), 0, st,
                   (const char*)(want_hit ? bk->a.act : nullptr), D.act_rows, (char*)(want_hit ? h_out : nullptr), row_bytes,
                   (const char*)(want_miss ? h_in : nullptr), (char*)(want_miss ? io->h_miss : nullptr), in_row_bytes,
                   (const int32_t*)io->slot, (const int32_t*)io->hit_idx, (const int32_t*)io->miss_idx,
-                  (const uint32_t*)io->counts, sel);
+                  (const uint32_t*)io->counts);
 }
 
 cudaError_t launch_scatter_insert(llmcache_bank* bk, const void* miss_out, const llmcache_probe_io* io,
