@@ -39,7 +39,12 @@ CFG = dict(layers=12, d_model=768, seq_len=384, batch=256, vocab=30522, n_seeds=
 
 # DRAM traffic per launch from an ncu capture of the named kernel on this workload, valid only while the
 # kernel's source file is unchanged (sha256 prefix of the file at capture time).
-NCU_TRAFFIC = {}
+NCU_TRAFFIC = {
+    # profiles/bert_base_one_layer_kernels.md (dram__bytes_read.sum + dram__bytes_write.sum of one launch)
+    "pool": {"file": "fingerprint.cu", "sha": "a545ba8d2701", "bytes_per_launch": 158515200},
+    "gather": {"file": "rows.cu", "sha": "40053a7cf26b", "bytes_per_launch": 83940608},
+    "scatter": {"file": "rows.cu", "sha": "40053a7cf26b", "bytes_per_launch": 124369920},
+}
 
 
 def parse():
