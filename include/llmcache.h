@@ -243,6 +243,63 @@ int llmcache_bank_profile_read(llmcache_bank_t* bank, uint32_t kernel_id, double
 /* Sticky device-side status (LLMCACHE_OK or LLMCACHE_ERR_TIMEOUT).  Synchronises the device. */
 int llmcache_bank_status(llmcache_bank_t* bank);
 
+/* ------------------------------------------------------------------------------------------------
+ * Miss-path transformer layer f_l and the layer-wise caching loop.
+ *
+ * Sec. IV-A: h_l = f_l(h_{l-1}); Algorithm 1 runs f_l only for the inputs that found no match.  The
+ * layer is the textbook one (multi-head self-attention, output projection, residual, layer norm,
+ * GELU feed-forward, residual, layer norm), in two arrangements: post-norm / bidirectional / GELU(erf)
+ * (BERT-style) and pre-norm / causal / GELU(tanh) (GPT-2-style).  Head size is 64.
+ * Weights are bf16 matrices in [out_features, in_features] row-major layout and f32 vectors, all
+ * DEVICE pointers, 16-byte aligned, borrowed: they must outlive the layer object.
+ * ------------------------------------------------------------------------------------------------ */
+typedef struct llmcache_layer llmcache_layer_t;
+
+typedef struct llmcache_layer_desc {
+  uint32_t struct_size;
+  int32_t  device;
+  uint32_t d_model;          /* d = 64 * heads */
+  uint32_t heads;
+  uint32_t ffn;              /* feed-forward width, multiple of 64 */
+  uint32_t seq_len;          /* n */
+  uint32_t max_seqs;         /* most sequences one forward call will pass */
+  uint32_t pre_ln;           /* 0: post-norm (BERT-style), 1: pre-norm (GPT-2-style) */
+  uint32_t causal;           /* 1: position i attends to positions <= i */
+  uint32_t tanh_gelu;        /* 0: GELU with erf, 1: tanh formula */
+  float    eps;              /* layer-norm epsilon (<= 0 => 1e-5) */
+  const void*  w_qkv;  const float* b_qkv;     /* [3d, d], [3d]  rows: q | k | v */
+  const void*  w_o;    const float* b_o;       /* [d, d], [d] */
+  const float* ln1_g;  const float* ln1_b;     /* [d] */
+  const void*  w_1;    const float* b_1;       /* [ffn, d], [ffn] */
+  const void*  w_2;    const float* b_2;       /* [d, ffn], [d] */
+  const float* ln2_g;  const float* ln2_b;     /* [d] */
+  void*    workspace;        /* device scratch (256-byte aligned) or NULL => the library cudaMallocs it;
+                                layers that never run concurrently may share one workspace */
+  size_t   workspace_bytes;  /* llmcache_layer_bytes tells how much is needed */
+} llmcache_layer_desc;
+
+int llmcache_layer_bytes(const llmcache_layer_desc* desc, size_t* bytes_out);
+int llmcache_layer_create(const llmcache_layer_desc* desc, llmcache_layer_t** layer_out);
+int llmcache_layer_destroy(llmcache_layer_t* layer);
+
+/* out[s] = f_l(x[s]) for the first sequences of x: device bf16 [n_seqs, n, d] -> device bf16 [n_seqs, n, d].
+ * n_seqs_dev: optional DEVICE u32: only min(n_seqs, *n_seqs_dev) sequences are processed (pass the miss
+ * count io->counts + 1 of the preceding probe: no host sync is needed).  x and out must not overlap. */
+int llmcache_layer_forward(llmcache_layer_t* layer, const void* x, uint32_t n_seqs, const uint32_t* n_seqs_dev,
+                           void* out, void* stream);
+/* LLMCACHE_OK or LLMCACHE_ERR_TIMEOUT (a bounded device-side wait expired).  Synchronises the device. */
+int llmcache_layer_status(llmcache_layer_t* layer);
+
+/* Algorithm 1 (LLMCache-Infer) for a batch of B sequences, without any host sync: for l = 1..n_layers,
+ * probe banks[l] with the current hidden states (hits take the stored output), run layers[l] on the
+ * compacted misses, commit (write back + insert).  banks == NULL runs every layer in full (no caching).
+ * h0: device bf16 [B,n,d].  buf_a, buf_b: device [B,n,d] bf16 ping-pong outputs; h_miss, miss_out: device
+ * [B,n,d] scratch (unused without banks); io: probe buffers for B.  *h_final receives the pointer (buf_a or
+ * buf_b) that holds h_L once the stream has run. */
+int llmcache_infer(llmcache_bank_t** banks, llmcache_layer_t** layers, uint32_t n_layers, const void* h0, uint32_t B,
+                   float tau, void* buf_a, void* buf_b, void* h_miss, void* miss_out, llmcache_probe_io* io,
+                   void** h_final, void* stream);
+
 #ifdef __cplusplus
 }
 #endif

@@ -32,6 +32,8 @@ EXPORTS = [
     "llmcache_commit", "llmcache_evict", "llmcache_bank_export", "llmcache_bank_import",
     "llmcache_bank_stats", "llmcache_bank_status", "llmcache_bank_profile", "llmcache_bank_profile_read",
     "llmcache_fingerprint_static", "llmcache_fingerprint_static_error",
+    "llmcache_layer_bytes", "llmcache_layer_create", "llmcache_layer_destroy", "llmcache_layer_forward",
+    "llmcache_layer_status", "llmcache_infer",
 ]
 FINGERPRINT_STATIC_MAX_FLOATS = 2 * 1024 * 1024
 KERNEL_NAMES = ["pool", "project", "rownorm", "scan", "decide", "touch", "gather", "select", "scatter", "evict"]
@@ -55,6 +57,21 @@ class ProbeIO(C.Structure):
         ("miss_idx", C.c_void_p), ("counts", C.c_void_p), ("counts_host", C.c_void_p),
         ("fp", C.c_void_p), ("rq", C.c_void_p), ("h_miss", C.c_void_p), ("generation", C.c_uint64),
     ]
+
+
+class LayerDesc(C.Structure):
+    _fields_ = [
+        ("struct_size", C.c_uint32), ("device", C.c_int32), ("d_model", C.c_uint32), ("heads", C.c_uint32),
+        ("ffn", C.c_uint32), ("seq_len", C.c_uint32), ("max_seqs", C.c_uint32), ("pre_ln", C.c_uint32),
+        ("causal", C.c_uint32), ("tanh_gelu", C.c_uint32), ("eps", C.c_float),
+        ("w_qkv", C.c_void_p), ("b_qkv", C.c_void_p), ("w_o", C.c_void_p), ("b_o", C.c_void_p),
+        ("ln1_g", C.c_void_p), ("ln1_b", C.c_void_p), ("w_1", C.c_void_p), ("b_1", C.c_void_p),
+        ("w_2", C.c_void_p), ("b_2", C.c_void_p), ("ln2_g", C.c_void_p), ("ln2_b", C.c_void_p),
+        ("workspace", C.c_void_p), ("workspace_bytes", C.c_size_t),
+    ]
+
+
+WEIGHT_NAMES = ("w_qkv", "b_qkv", "w_o", "b_o", "ln1_g", "ln1_b", "w_1", "b_1", "w_2", "b_2", "ln2_g", "ln2_b")
 
 
 class Stats(C.Structure):
@@ -101,6 +118,13 @@ def lib():
         L.llmcache_bank_status.argtypes = [vp]
         L.llmcache_bank_profile.argtypes = [vp, C.c_int]
         L.llmcache_bank_profile_read.argtypes = [vp, u32, C.POINTER(C.c_double), C.POINTER(C.c_uint64)]
+        L.llmcache_layer_bytes.argtypes = [C.POINTER(LayerDesc), C.POINTER(C.c_size_t)]
+        L.llmcache_layer_create.argtypes = [C.POINTER(LayerDesc), C.POINTER(vp)]
+        L.llmcache_layer_destroy.argtypes = [vp]
+        L.llmcache_layer_forward.argtypes = [vp, vp, u32, vp, vp, vp]
+        L.llmcache_layer_status.argtypes = [vp]
+        L.llmcache_infer.argtypes = [C.POINTER(vp), C.POINTER(vp), u32, vp, u32, C.c_float, vp, vp, vp, vp,
+                                     C.POINTER(ProbeIO), C.POINTER(vp), vp]
         L.llmcache_fingerprint_static.argtypes = [vp, u32, u32, u32, u32, u32, vp, vp, vp, vp, vp]
         L.llmcache_fingerprint_static_error.restype = C.c_char_p
         L.llmcache_fingerprint_static_error.argtypes = []
@@ -356,3 +380,82 @@ class Bank:
     def profile_read(self) -> dict:
         """{kernel name: (total ms, launches)} since the last read."""
         return {name: llmcache_bank_profile_read(self.handle, i) for i, name in enumerate(KERNEL_NAMES)}
+
+
+# ----------------------------------------------------------------------------
+# Miss-path transformer layer and the layer-wise caching loop
+# ----------------------------------------------------------------------------
+def llmcache_layer_bytes(desc: LayerDesc) -> int:
+    out = C.c_size_t(0)
+    _check(lib().llmcache_layer_bytes(C.byref(desc), C.byref(out)), "llmcache_layer_bytes")
+    return int(out.value)
+
+
+def llmcache_layer_create(desc: LayerDesc) -> int:
+    out = C.c_void_p(None)
+    _check(lib().llmcache_layer_create(C.byref(desc), C.byref(out)), "llmcache_layer_create")
+    return out.value
+
+
+def llmcache_layer_destroy(layer: int) -> None:
+    _check(lib().llmcache_layer_destroy(layer), "llmcache_layer_destroy")
+
+
+def llmcache_layer_forward(layer, x, n_seqs, n_seqs_dev, out, stream=None) -> None:
+    _check(lib().llmcache_layer_forward(layer, _ptr(x), n_seqs, _ptr(n_seqs_dev), _ptr(out), _stream(stream)),
+           "llmcache_layer_forward")
+
+
+def llmcache_layer_status(layer) -> int:
+    return int(lib().llmcache_layer_status(layer))
+
+
+def llmcache_infer(banks, layers, h0, B, tau, buf_a, buf_b, h_miss, miss_out, io, stream=None) -> int:
+    """Algorithm 1 over all layers; returns the device address (buf_a or buf_b) that will hold h_L."""
+    n = len(layers)
+    larr = (C.c_void_p * n)(*layers)
+    barr = (C.c_void_p * n)(*banks) if banks is not None else None
+    final = C.c_void_p(None)
+    tau = float("nan") if tau is None else tau
+    _check(lib().llmcache_infer(barr, larr, n, _ptr(h0), B, tau, _ptr(buf_a), _ptr(buf_b), _ptr(h_miss),
+                                _ptr(miss_out), C.byref(io) if io is not None else None, C.byref(final),
+                                _stream(stream)), "llmcache_infer")
+    return final.value
+
+
+class Layer:
+    """Owner of one llmcache_layer_t handle; keeps the weight tensors alive (the library borrows them)."""
+
+    def __init__(self, weights: dict, *, device=0, heads, seq_len, max_seqs, pre_ln=False, causal=False,
+                 tanh_gelu=False, eps=1e-5, workspace: Optional[torch.Tensor] = None):
+        self.weights = {k: weights[k].contiguous() for k in WEIGHT_NAMES}
+        d = LayerDesc()
+        d.struct_size = C.sizeof(LayerDesc)
+        d.device = device
+        d.d_model = self.weights["w_o"].shape[0]
+        d.heads, d.ffn, d.seq_len, d.max_seqs = heads, self.weights["w_1"].shape[0], seq_len, max_seqs
+        d.pre_ln, d.causal, d.tanh_gelu, d.eps = int(pre_ln), int(causal), int(tanh_gelu), eps
+        for k in WEIGHT_NAMES:
+            setattr(d, k, self.weights[k].data_ptr())
+        self.workspace = workspace
+        if workspace is not None:
+            d.workspace, d.workspace_bytes = workspace.data_ptr(), workspace.numel() * workspace.element_size()
+        self.desc = d
+        self.handle = llmcache_layer_create(d)
+
+    def forward(self, x, out, n_seqs=None, n_seqs_dev=None, stream=None):
+        llmcache_layer_forward(self.handle, x, x.shape[0] if n_seqs is None else n_seqs, n_seqs_dev, out, stream)
+
+    def status(self) -> int:
+        return llmcache_layer_status(self.handle)
+
+    def close(self):
+        if getattr(self, "handle", None):
+            llmcache_layer_destroy(self.handle)
+            self.handle = None
+
+    def __del__(self):
+        try:
+            self.close()
+        except Exception:
+            pass

@@ -1,0 +1,21 @@
+// Miss-path transformer layer: shared declarations.
+#pragma once
+#include "llmcache_internal.cuh"
+
+namespace llmc {
+
+enum { LAYER_ACT_NONE = 0, LAYER_ACT_GELU_ERF = 1, LAYER_ACT_GELU_TANH = 2 };
+
+cudaError_t setup_gemm_kernel();
+cudaError_t launch_gemm(const __nv_bfloat16* a, const __nv_bfloat16* w, const float* bias,
+                        const __nv_bfloat16* residual, __nv_bfloat16* out, uint32_t* status, uint32_t M_max,
+                        uint32_t N, uint32_t K, const uint32_t* m_seq_dev, uint32_t rows_per_seq, uint32_t act,
+                        int sm_count, cudaStream_t st);
+
+cudaError_t launch_layernorm(const __nv_bfloat16* x, const float* g, const float* b, __nv_bfloat16* y, uint32_t M_max,
+                             uint32_t d, const uint32_t* m_seq_dev, uint32_t rows_per_seq, float eps, int sm_count,
+                             cudaStream_t st);
+cudaError_t launch_attention(const __nv_bfloat16* qkv, __nv_bfloat16* out, uint32_t n, uint32_t d, uint32_t heads,
+                             uint32_t seq_max, const uint32_t* m_seq_dev, int causal, cudaStream_t st);
+
+}  // namespace llmc

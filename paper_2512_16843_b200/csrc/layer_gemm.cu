@@ -1,0 +1,232 @@
+// Dense layer of the miss path: C[M, N] = act(A[M, K] . W[N, K]^T + bias) (+ residual), bf16 in and
+// out, fp32 accumulation.  The transformer layer f_l that runs on the misses (Algorithm 1,
+// "h_l <- f_l(h_{l-1})") is made of four of these.  Same machinery as the bank scan: TMA (128-byte
+// swizzle) into a 4-stage ring, tcgen05.mma 128 x 256 x 16 into two TMEM accumulators, epilogue warps
+// that drain one accumulator while the next tile's MMAs run.  The number of valid rows may come from
+// device memory (the miss count of the probe that precedes it), so no host sync is needed.
+// All mbarrier waits are bounded (status word, see scan.cu).
+#include <cuda.h>
+#include "llmcache_internal.cuh"
+#include "ptx.cuh"
+#include "layer.cuh"
+
+namespace llmc {
+
+namespace {
+constexpr int GM = 128, GN = 256, GK = 64, GSTAGES = 4, G_UMMA_K = 16;
+constexpr int GEMM_THREADS = 192;
+constexpr uint32_t GA_BYTES = GM * GK * 2, GB_BYTES = GN * GK * 2;
+constexpr uint32_t G_TMEM_COLS = 512;
+struct GemmSmem {
+  static constexpr uint32_t A = 0;
+  static constexpr uint32_t B = A + GSTAGES * GA_BYTES;
+  static constexpr uint32_t BIAS = B + GSTAGES * GB_BYTES;       // float [2][GN]
+  static constexpr uint32_t BAR = BIAS + 2 * GN * 4;
+  static constexpr uint32_t MISC = BAR + 16 * 8;
+  static constexpr uint32_t TOTAL = MISC + 64;
+};
+constexpr uint32_t GEMM_SMEM_BYTES = GemmSmem::TOTAL + 1024;
+constexpr uint32_t G_IDESC = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(GN >> 3) << 17) | ((uint32_t)(GM >> 4) << 24);
+
+__device__ __forceinline__ float gelu_erf_f(float x) { return 0.5f * x * (1.0f + erff(x * 0.70710678118654752f)); }
+__device__ __forceinline__ float gelu_tanh_f(float x) {
+  return 0.5f * x * (1.0f + tanhf(0.7978845608028654f * (x + 0.044715f * x * x * x)));
+}
+__device__ __forceinline__ uint32_t pack_bf16(float a, float b) {
+  const __nv_bfloat162 v = __floats2bfloat162_rn(a, b);
+  return *reinterpret_cast<const uint32_t*>(&v);
+}
+}  // namespace
+
+__global__ void __launch_bounds__(GEMM_THREADS, 1)
+k_gemm_tc(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_w,
+          const float* __restrict__ bias, const __nv_bfloat16* __restrict__ residual,
+          __nv_bfloat16* __restrict__ out, uint32_t* __restrict__ status,
+          uint32_t M_max, uint32_t N, uint32_t KB, const uint32_t* __restrict__ m_seq_dev, uint32_t rows_per_seq,
+          uint32_t act) {
+  griddep_sync();
+  extern __shared__ uint8_t smem_raw[];
+  const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;
+  uint8_t* gbase = smem_raw + (base - smem_u32(smem_raw));
+  const uint32_t sA = base + GemmSmem::A, sB = base + GemmSmem::B;
+  float* sbias = reinterpret_cast<float*>(gbase + GemmSmem::BIAS);
+  const uint32_t bar0 = base + GemmSmem::BAR;
+  auto full_bar = [&](uint32_t s) { return bar0 + 8 * s; };
+  auto empty_bar = [&](uint32_t s) { return bar0 + 8 * (GSTAGES + s); };
+  auto tfull_bar = [&](uint32_t b) { return bar0 + 8 * (2 * GSTAGES + b); };
+  auto tempty_bar = [&](uint32_t b) { return bar0 + 8 * (2 * GSTAGES + 2 + b); };
+  volatile uint32_t* misc = reinterpret_cast<volatile uint32_t*>(gbase + GemmSmem::MISC);
+  volatile uint32_t* tmem_slot = misc + 0;
+  volatile uint32_t* abort_flag = misc + 1;
+  volatile uint32_t* epi_go = misc + 2;
+  const uint32_t warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+
+  // rows that hold data: all of them, or (sequences counted on the device) x (rows per sequence)
+  uint32_t M = M_max;
+  if (m_seq_dev) {
+    const unsigned long long m = (unsigned long long)(*m_seq_dev) * rows_per_seq;
+    M = m < M_max ? (uint32_t)m : M_max;
+  }
+  const uint32_t MB = (M + GM - 1) / GM, NB = (N + GN - 1) / GN;
+  const uint32_t n_tiles = MB * NB;
+
+  if (threadIdx.x == 0) {
+    for (uint32_t s = 0; s < GSTAGES; ++s) { mbar_init(full_bar(s), 1); mbar_init(empty_bar(s), 1); }
+    for (uint32_t b = 0; b < 2; ++b) { mbar_init(tfull_bar(b), 1); mbar_init(tempty_bar(b), 128); }
+    misc[1] = 0; misc[2] = 0; misc[3] = 0;
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+  }
+  if (warp == 1) {
+    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;"
+                 ::"r"(smem_u32((const void*)tmem_slot)), "r"(G_TMEM_COLS) : "memory");
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+  }
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  const uint32_t tmem_base = *tmem_slot;
+
+  uint32_t issued = 0;
+  if (warp == 0) {
+    if (lane == 0) {                                   // ---- TMA producer
+      bool ok = true;
+      for (uint32_t t = blockIdx.x; t < n_tiles && ok; t += gridDim.x) {
+        const uint32_t mb = t / NB, nb = t % NB;       // consecutive blocks share the A tile in L2
+        for (uint32_t kb = 0; kb < KB; ++kb) {
+          const uint32_t s = issued % GSTAGES, ph = (issued / GSTAGES) & 1u;
+          if (!mbar_wait(empty_bar(s), ph ^ 1u, abort_flag)) { ok = false; break; }
+          mbar_expect_tx(full_bar(s), GA_BYTES + GB_BYTES);
+          tma_load_2d(sA + s * GA_BYTES, &map_a, (int)(kb * GK), (int)(mb * GM), full_bar(s));
+          tma_load_2d(sB + s * GB_BYTES, &map_w, (int)(kb * GK), (int)(nb * GN), full_bar(s));
+          ++issued;
+        }
+      }
+      if (!ok) { *abort_flag = 1; atomicExch(status, 1u); }
+    }
+  } else if (warp == 1) {
+    if (lane == 0) {                                   // ---- MMA issuer
+      bool ok = true;
+      uint32_t it = 0, tile = 0;
+      for (uint32_t t = blockIdx.x; t < n_tiles && ok; t += gridDim.x, ++tile) {
+        const uint32_t buf = tile & 1u, bph = (tile >> 1) & 1u;
+        if (!mbar_wait(tempty_bar(buf), bph ^ 1u, abort_flag)) { ok = false; break; }
+        tc_fence_after();
+        const uint32_t d_tmem = tmem_base + buf * GN;
+        for (uint32_t kb = 0; kb < KB; ++kb, ++it) {
+          const uint32_t s = it % GSTAGES, ph = (it / GSTAGES) & 1u;
+          if (!mbar_wait(full_bar(s), ph, abort_flag)) { ok = false; break; }
+          tc_fence_after();
+          const uint64_t da = smem_desc_sw128(sA + s * GA_BYTES), db = smem_desc_sw128(sB + s * GB_BYTES);
+#pragma unroll
+          for (uint32_t kk = 0; kk < GK / G_UMMA_K; ++kk)
+            tc_mma_bf16(d_tmem, da + kk * (G_UMMA_K * 2 / 16), db + kk * (G_UMMA_K * 2 / 16), G_IDESC, (kb | kk) != 0u);
+          tc_commit(empty_bar(s));
+        }
+        if (ok) tc_commit(tfull_bar(buf));
+      }
+      if (!ok) { *abort_flag = 1; atomicExch(status, 1u); }
+    }
+  } else {
+    // ---- epilogue: bias, activation, residual, bf16 store; thread = one output row of the tile
+    const uint32_t et = threadIdx.x - 64, quarter = warp & 3u;
+    const uint32_t row_in_tile = quarter * 32 + lane;
+    uint32_t tile = 0;
+    for (uint32_t t = blockIdx.x; t < n_tiles; t += gridDim.x, ++tile) {
+      const uint32_t mb = t / NB, nb = t % NB;
+      const uint32_t buf = tile & 1u, bph = (tile >> 1) & 1u;
+      float* bt = sbias + buf * GN;
+      for (uint32_t x = et; x < GN; x += 128) {
+        const uint32_t c = nb * GN + x;
+        bt[x] = (bias && c < N) ? bias[c] : 0.f;
+      }
+      if (et == 0) epi_go[buf] = *abort_flag;
+      asm volatile("bar.sync 1, 128;" ::: "memory");
+      if (epi_go[buf]) break;
+      if (!mbar_wait(tfull_bar(buf), bph, abort_flag)) { *abort_flag = 1; atomicExch(status, 1u); }
+      tc_fence_after();
+      const uint32_t taddr = tmem_base + buf * GN + ((quarter * 32u) << 16);
+      const uint32_t row = mb * GM + row_in_tile;
+      const bool row_ok = row < M;
+#pragma unroll 1
+      for (uint32_t c = 0; c < GN; c += 32) {
+        uint32_t v[32];
+        tc_ld_32x32(taddr + c, v);
+        tc_wait_ld();
+        const uint32_t col0 = nb * GN + c;
+        if (row_ok && col0 < N) {                       // N is a multiple of 64: a 32-column group is all in or all out
+          float f[32];
+#pragma unroll
+          for (int i = 0; i < 32; ++i) f[i] = __uint_as_float(v[i]) + bt[c + i];
+          if (act == LAYER_ACT_GELU_ERF) {
+#pragma unroll
+            for (int i = 0; i < 32; ++i) f[i] = gelu_erf_f(f[i]);
+          } else if (act == LAYER_ACT_GELU_TANH) {
+#pragma unroll
+            for (int i = 0; i < 32; ++i) f[i] = gelu_tanh_f(f[i]);
+          }
+          const size_t off = (size_t)row * N + col0;
+          if (residual) {
+            const uint4* r4 = reinterpret_cast<const uint4*>(residual + off);
+#pragma unroll
+            for (int q = 0; q < 4; ++q) {
+              const uint4 r = r4[q];
+              const uint32_t w[4] = {r.x, r.y, r.z, r.w};
+#pragma unroll
+              for (int u = 0; u < 4; ++u) {
+                f[q * 8 + 2 * u]     += __uint_as_float(w[u] << 16);
+                f[q * 8 + 2 * u + 1] += __uint_as_float(w[u] & 0xFFFF0000u);
+              }
+            }
+          }
+          uint4* o4 = reinterpret_cast<uint4*>(out + off);
+#pragma unroll
+          for (int q = 0; q < 4; ++q)
+            o4[q] = make_uint4(pack_bf16(f[q * 8], f[q * 8 + 1]), pack_bf16(f[q * 8 + 2], f[q * 8 + 3]),
+                               pack_bf16(f[q * 8 + 4], f[q * 8 + 5]), pack_bf16(f[q * 8 + 6], f[q * 8 + 7]));
+        }
+      }
+      tc_fence_before();
+      mbar_arrive(tempty_bar(buf));
+    }
+  }
+
+  tc_fence_before();
+  __syncthreads();
+  if (threadIdx.x == 0 && *abort_flag) {
+    const uint32_t back = issued < (uint32_t)GSTAGES ? issued : (uint32_t)GSTAGES;
+    volatile uint32_t never = 0;
+    for (uint32_t i = 0; i < back; ++i) {
+      const uint32_t itx = issued - 1 - i;
+      mbar_wait(full_bar(itx % GSTAGES), (itx / GSTAGES) & 1u, &never, 200000000ull);
+    }
+  }
+  __syncthreads();
+  if (warp == 1) {
+    tc_fence_after();
+    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(G_TMEM_COLS) : "memory");
+  }
+}
+
+cudaError_t setup_gemm_kernel() {
+  cudaError_t e = tensor_map_setup();
+  if (e != cudaSuccess) return e;
+  return cudaFuncSetAttribute(k_gemm_tc, cudaFuncAttributeMaxDynamicSharedMemorySize, GEMM_SMEM_BYTES);
+}
+
+// out[M, N] = act(a[M, K] . w[N, K]^T + bias) (+ residual).  K, N multiples of 64.
+cudaError_t launch_gemm(const __nv_bfloat16* a, const __nv_bfloat16* w, const float* bias,
+                        const __nv_bfloat16* residual, __nv_bfloat16* out, uint32_t* status, uint32_t M_max,
+                        uint32_t N, uint32_t K, const uint32_t* m_seq_dev, uint32_t rows_per_seq, uint32_t act,
+                        int sm_count, cudaStream_t st) {
+  if (M_max == 0) return cudaSuccess;
+  alignas(64) CUtensorMap map_a, map_w;
+  if (!make_tensor_map_bf16(&map_a, a, M_max, K, GM) || !make_tensor_map_bf16(&map_w, w, N, K, GN))
+    return cudaErrorInvalidValue;
+  const uint32_t tiles = ((M_max + GM - 1) / GM) * ((N + GN - 1) / GN);
+  const uint32_t grid = tiles < (uint32_t)sm_count ? tiles : (uint32_t)sm_count;
+  return launch_k(k_gemm_tc, dim3(grid), dim3(GEMM_THREADS), GEMM_SMEM_BYTES, st, map_a, map_w, bias, residual, out,
+                  status, M_max, N, K / GK, m_seq_dev, rows_per_seq, act);
+}
+
+}  // namespace llmc

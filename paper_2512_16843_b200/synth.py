@@ -169,3 +169,14 @@ def scan_stress(n_bank, n_query, k, n_clusters=4096, spread=0.1, near_fraction=0
     source[:n_near] = src
     perm = torch.randperm(n_query, generator=g, device=device)
     return bank, q[perm].to(torch.bfloat16).contiguous(), source[perm]
+
+
+def layer_weights(d_model, ffn, seed, device="cpu"):
+    """Random-init transformer layer weights: bf16 matrices in [out, in] layout ~ N(0, 0.02^2) (the usual
+    initialisation of BERT / GPT-2), f32 biases ~ N(0, 0.02^2), layer-norm gains 1 + N(0, 0.02^2)."""
+    mat = lambda o, i, s: randn((o, i), seed + s, device, dtype=torch.bfloat16, scale=0.02)
+    vec = lambda n, s, base=0.0: (randn((n,), seed + s, device, scale=0.02) + base).contiguous()
+    return {"w_qkv": mat(3 * d_model, d_model, 1), "b_qkv": vec(3 * d_model, 2), "w_o": mat(d_model, d_model, 3),
+            "b_o": vec(d_model, 4), "ln1_g": vec(d_model, 5, 1.0), "ln1_b": vec(d_model, 6),
+            "w_1": mat(ffn, d_model, 7), "b_1": vec(ffn, 8), "w_2": mat(d_model, ffn, 9), "b_2": vec(d_model, 10),
+            "ln2_g": vec(d_model, 11, 1.0), "ln2_b": vec(d_model, 12)}

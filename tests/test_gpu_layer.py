@@ -1,0 +1,134 @@
+"""Miss-path transformer layer and the layer-wise caching loop (Algorithm 1) against the oracle.
+
+Tolerance (derived): the CUDA layer keeps seven intermediate tensors in bf16 and accumulates in fp32.
+Against the oracle that rounds at the same storage points the remaining differences are fp32 vs float64
+accumulation, the fast exponential, and the occasional bf16 rounding that falls the other way (one step =
+2^-8 relative on that element): root-mean-square error <= 4e-3 of the output's RMS and no element further
+than 4 bf16 steps of the element + 2 % of the output's RMS (an element near zero inherits the rounding
+steps of the larger terms it is the sum of).  Against the oracle that rounds nothing: RMS error <= 2e-2."""
+import numpy as np
+import pytest
+import torch
+
+from oracle import llmcache_oracle as O
+from oracle import transformer_oracle as T
+from paper_2512_16843_b200 import binding as L
+from paper_2512_16843_b200 import synth
+
+pytestmark = pytest.mark.gpu
+DEV = "cuda"
+
+
+def oracle_weights(w):
+    conv = lambda t: synth.bf16_bits(t) if t.dtype == torch.bfloat16 else t.cpu().numpy()
+    return T.LayerWeights(**{k: conv(w[k]) for k in L.WEIGHT_NAMES})
+
+
+def rel_rms(a, b):
+    return float(np.sqrt(np.mean((a - b) ** 2)) / np.sqrt(np.mean(b ** 2)))
+
+
+def check_layer_output(got_bits, x_bits, ow, heads, **kw):
+    got = O.bf16_to_f32(got_bits).astype(np.float64)
+    ref_r = O.bf16_to_f32(T.layer_forward(x_bits, ow, heads, round_bf16=True, **kw)).astype(np.float64)
+    ref_e = T.layer_forward_f64(x_bits, ow, heads, **kw)
+    assert rel_rms(got, ref_r) <= 4e-3, rel_rms(got, ref_r)
+    assert np.all(np.abs(got - ref_r) <= 4 * 2.0 ** -8 * np.abs(ref_r) + 0.02 * np.sqrt(np.mean(ref_r ** 2)))
+    assert rel_rms(got, ref_e) <= 2e-2, rel_rms(got, ref_e)
+
+
+@pytest.mark.parametrize("n,d,heads,ffn,S,pre_ln,causal,tanh", [
+    (40, 128, 2, 256, 3, False, False, False),       # ragged everywhere
+    (130, 192, 3, 320, 2, True, True, True),         # two query tiles, causal, odd tile counts
+    (128, 768, 12, 3072, 2, False, False, False),    # BERT-base layer
+    (256, 768, 12, 3072, 1, True, True, True),       # GPT-2-small layer
+])
+def test_layer_forward_matches_oracle(n, d, heads, ffn, S, pre_ln, causal, tanh):
+    w = synth.layer_weights(d, ffn, 100 + d + n, DEV)
+    # larger weights than the 0.02 initialisation so that every sub-block matters in the output
+    for k in ("w_qkv", "w_o", "w_1", "w_2"):
+        w[k] = (w[k].float() * 3.0).to(torch.bfloat16)
+    layer = L.Layer(w, heads=heads, seq_len=n, max_seqs=S, pre_ln=pre_ln, causal=causal, tanh_gelu=tanh)
+    x = synth.randn((S, n, d), 7, DEV, torch.bfloat16)
+    out = torch.zeros_like(x)
+    layer.forward(x, out)
+    torch.cuda.synchronize()
+    assert layer.status() == L.OK
+    ow = oracle_weights(w)
+    for s in range(S):
+        check_layer_output(synth.bf16_bits(out[s]), synth.bf16_bits(x[s]), ow, heads,
+                           pre_ln=pre_ln, causal=causal, tanh_gelu=tanh)
+    layer.close()
+
+
+def test_layer_forward_with_device_side_count():
+    n, d, heads, ffn, S = 64, 128, 2, 256, 5
+    w = synth.layer_weights(d, ffn, 31, DEV)
+    layer = L.Layer(w, heads=heads, seq_len=n, max_seqs=S)
+    x = synth.randn((S, n, d), 8, DEV, torch.bfloat16)
+    full = torch.zeros_like(x)
+    layer.forward(x, full)
+    for count in (0, 2, 5, 9):
+        out = torch.full_like(x, 7.0)
+        cnt = torch.tensor([count], dtype=torch.int32, device=DEV)
+        layer.forward(x, out, n_seqs_dev=cnt)
+        torch.cuda.synchronize()
+        m = min(count, S)
+        assert torch.equal(out[:m].view(torch.int16), full[:m].view(torch.int16))     # same bits as the full run
+        assert torch.all(out[m:] == 7.0)                                             # nothing beyond the count
+    with pytest.raises(L.LLMCacheError) as e:
+        layer.forward(torch.zeros((S + 1, n, d), dtype=torch.bfloat16, device=DEV), torch.zeros((S + 1, n, d), dtype=torch.bfloat16, device=DEV))
+    assert e.value.status == L.ERR_SHAPE
+    layer.close()
+
+
+@pytest.mark.parametrize("pre_ln", [False, True])
+def test_infer_algorithm1_matches_oracle_and_chain_property(pre_ln):
+    n, d, heads, ffn, B, Lyr, N, k = 48, 128, 2, 256, 12, 3, 64, 64
+    ws = [synth.layer_weights(d, ffn, 200 + 20 * l, DEV) for l in range(Lyr)]
+    for w in ws:
+        for key in ("w_qkv", "w_o", "w_1", "w_2"):
+            w[key] = (w[key].float() * 3.0).to(torch.bfloat16)
+    proj = synth.projection(d, k, 9, DEV)
+    kw = dict(pre_ln=pre_ln, causal=pre_ln, tanh_gelu=pre_ln)
+    layers = [L.Layer(w, heads=heads, seq_len=n, max_seqs=B, **kw) for w in ws]
+    banks = [L.Bank(capacity=N, seq_len=n, d_model=d, fp_dim=k, max_batch=B, proj=proj, tau=0.9) for _ in range(Lyr)]
+    obanks = [O.Bank(capacity=N, seq_len=n, d_model=d, fp_dim=k, tau=0.9, proj=synth.bf16_bits(proj)) for _ in range(Lyr)]
+    ows = [oracle_weights(w) for w in ws]
+    bufs = L.ProbeBuffers(B, k, DEV)
+    mk = lambda: torch.zeros((B, n, d), dtype=torch.bfloat16, device=DEV)
+    buf_a, buf_b, h_miss, miss_out = mk(), mk(), mk(), mk()
+    handles_b, handles_l = [b.handle for b in banks], [l.handle for l in layers]
+
+    def run(h0, use_banks=True):
+        ptr = L.llmcache_infer(handles_b if use_banks else None, handles_l, h0, B, None, buf_a, buf_b, h_miss, miss_out, bufs.io)
+        torch.cuda.synchronize()
+        return (buf_a if ptr == buf_a.data_ptr() else buf_b).clone()
+
+    h0 = synth.randn((B, n, d), 3, DEV, torch.bfloat16)
+    plain = run(h0, use_banks=False)                     # no caching: every layer in full
+    out1 = run(h0)                                       # empty banks: all miss, same computation
+    assert torch.equal(plain.view(torch.int16), out1.view(torch.int16))
+    ref1, hits1 = T.infer(obanks, ows, synth.bf16_bits(h0), heads, round_bf16=True, **kw)
+    assert hits1 == [0] * Lyr and [b.stats()["hits"] for b in banks] == [0] * Lyr
+    got = O.bf16_to_f32(synth.bf16_bits(out1)).astype(np.float64)
+    ref = O.bf16_to_f32(ref1).astype(np.float64).reshape(got.shape)
+    assert rel_rms(got, ref) <= 1e-2
+    # same batch again: every layer is served from its bank; the output has the same bits (Algorithm 1)
+    out2 = run(h0)
+    assert [b.stats()["hits"] for b in banks] == [B] * Lyr
+    assert torch.equal(out1.view(torch.int16), out2.view(torch.int16))
+    ref2, hits2 = T.infer(obanks, ows, synth.bf16_bits(h0), heads, round_bf16=True, **kw)
+    assert hits2 == [B] * Lyr
+    # a mixed batch: near-duplicates hit at layer 1 and hence at every deeper layer with the donor's output
+    mixed = h0.clone()
+    mixed[1] = (h0[0].float() + 0.02 * synth.randn((n, d), 4, DEV)).to(torch.bfloat16)
+    mixed[5:9] = synth.randn((4, n, d), 5, DEV, torch.bfloat16)
+    out3 = run(mixed)
+    ref3, hits3 = T.infer(obanks, ows, synth.bf16_bits(mixed), heads, round_bf16=True, **kw)
+    gpu_hits = [b.stats()["hits"] - B for b in banks]
+    assert gpu_hits == hits3 == [B - 4] * Lyr
+    assert torch.equal(out3[1].view(torch.int16), out1[0].view(torch.int16))
+    assert all(l.status() == L.OK for l in layers) and all(b.status() == L.OK for b in banks)
+    for o in layers + banks:
+        o.close()
