@@ -3,7 +3,9 @@
 Tolerance (derived): the CUDA layer keeps seven intermediate tensors in bf16 and accumulates in fp32.
 Against the oracle that rounds at the same storage points the remaining differences are fp32 vs float64
 accumulation, the fast exponential, and the occasional bf16 rounding that falls the other way (one step =
-2^-8 relative on that element): root-mean-square error <= 4e-3 of the output's RMS and no element further
+2^-8 relative on that element), and the bf16 rounding of the attention probabilities that feed the
+tensor-core P V product (about 1e-3 relative each, which the oracle does not have):
+root-mean-square error <= 6e-3 of the output's RMS (1.5 bf16 steps) and no element further
 than 4 bf16 steps of the element + 2 % of the output's RMS (an element near zero inherits the rounding
 steps of the larger terms it is the sum of).  Against the oracle that rounds nothing: RMS error <= 2e-2."""
 import numpy as np
@@ -32,7 +34,7 @@ def check_layer_output(got_bits, x_bits, ow, heads, **kw):
     got = O.bf16_to_f32(got_bits).astype(np.float64)
     ref_r = O.bf16_to_f32(T.layer_forward(x_bits, ow, heads, round_bf16=True, **kw)).astype(np.float64)
     ref_e = T.layer_forward_f64(x_bits, ow, heads, **kw)
-    assert rel_rms(got, ref_r) <= 4e-3, rel_rms(got, ref_r)
+    assert rel_rms(got, ref_r) <= 6e-3, rel_rms(got, ref_r)
     assert np.all(np.abs(got - ref_r) <= 4 * 2.0 ** -8 * np.abs(ref_r) + 0.02 * np.sqrt(np.mean(ref_r ** 2)))
     assert rel_rms(got, ref_e) <= 2e-2, rel_rms(got, ref_e)
 
