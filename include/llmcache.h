@@ -300,6 +300,18 @@ int llmcache_infer(llmcache_bank_t** banks, llmcache_layer_t** layers, uint32_t 
                    float tau, void* buf_a, void* buf_b, void* h_miss, void* miss_out, llmcache_probe_io* io,
                    void** h_final, void* stream);
 
+/* Divergence monitor (Sec. III-E: "tracking differences in successive outputs for a given fingerprint";
+ * Sec. IV-D: "revalidates fingerprints").  Call after the commit of a probe, with that probe's h_in and io.
+ * For every stride-th hit (ascending batch order) the layer is recomputed on the sequence's input and
+ * compared with the stored output it was served: rel = ||f_l(h) - h'|| / ||f_l(h)||.  Entries with
+ * rel > bound are invalidated (not those re-inserted during the current tick).
+ * h_sample, out_sample: device bf16 scratch [ceil(B/stride), n, d]; rel_out: device f32 [ceil(B/stride)];
+ * counters_dev: device u32 [2] = {samples checked, entries invalidated}.  The layer must have
+ * max_seqs >= ceil(B/stride).  bf16 banks that store activations only. */
+int llmcache_divergence_check(llmcache_bank_t* bank, llmcache_layer_t* layer, const void* h_in,
+                              const llmcache_probe_io* io, uint32_t stride, float bound, void* h_sample,
+                              void* out_sample, float* rel_out, uint32_t* counters_dev, void* stream);
+
 #ifdef __cplusplus
 }
 #endif

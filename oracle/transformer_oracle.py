@@ -152,3 +152,27 @@ def infer(banks: List[O.Bank], layers: List[LayerWeights], h0_bits: np.ndarray, 
         hits.append(int(pr.hit.sum()))
         h = h_out.reshape(B, n, d)
     return h.reshape(B, n * d), hits
+
+
+def divergence_check(bank: O.Bank, w: LayerWeights, h_bits: np.ndarray, pr: O.ProbeResult, heads: int,
+                     stride: int, bound: float, pre_ln=False, causal=False, tanh_gelu=False, round_bf16=False):
+    """Divergence monitor (Sec. III-E "tracking differences in successive outputs for a given fingerprint";
+    Sec. IV-D "revalidates fingerprints").  For every `stride`-th hit of the probe (in ascending batch
+    order) the layer is recomputed on that sequence's input and compared with the stored output it was
+    served: rel = ||f_l(h) - h'||_2 / ||f_l(h)||_2.  An entry whose rel exceeds `bound` is invalidated,
+    unless it was (re)inserted during the current tick.  Returns (list of (b, slot, rel), number invalidated)."""
+    checked, dropped = [], 0
+    n, d = bank.seq_len, bank.d_model
+    for i in range(0, len(pr.hit_idx), stride):
+        b = int(pr.hit_idx[i])
+        slot = int(pr.slot[b])
+        fresh = O.bf16_to_f32(layer_forward(h_bits[b].reshape(n, d), w, heads, pre_ln, causal, tanh_gelu,
+                                            round_bf16)).astype(np.float64).reshape(-1)
+        stored = O.bf16_to_f32(bank.act[slot % bank.act_rows]).astype(np.float64)
+        den = float(np.sqrt(np.sum(fresh * fresh)))
+        rel = float(np.sqrt(np.sum((fresh - stored) ** 2))) / den if den > 0 else 0.0
+        checked.append((b, slot, rel))
+        if rel > bound and bank.valid[slot] and int(bank.insert_tick[slot]) != bank.tick:
+            bank.valid[slot] = 0
+            dropped += 1
+    return checked, dropped

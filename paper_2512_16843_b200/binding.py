@@ -33,7 +33,7 @@ EXPORTS = [
     "llmcache_bank_stats", "llmcache_bank_status", "llmcache_bank_profile", "llmcache_bank_profile_read",
     "llmcache_fingerprint_static", "llmcache_fingerprint_static_error",
     "llmcache_layer_bytes", "llmcache_layer_create", "llmcache_layer_destroy", "llmcache_layer_forward",
-    "llmcache_layer_status", "llmcache_infer",
+    "llmcache_layer_status", "llmcache_infer", "llmcache_divergence_check",
 ]
 FINGERPRINT_STATIC_MAX_FLOATS = 2 * 1024 * 1024
 KERNEL_NAMES = ["pool", "project", "rownorm", "scan", "decide", "touch", "gather", "select", "scatter", "evict"]
@@ -125,6 +125,7 @@ def lib():
         L.llmcache_layer_status.argtypes = [vp]
         L.llmcache_infer.argtypes = [C.POINTER(vp), C.POINTER(vp), u32, vp, u32, C.c_float, vp, vp, vp, vp,
                                      C.POINTER(ProbeIO), C.POINTER(vp), vp]
+        L.llmcache_divergence_check.argtypes = [vp, vp, vp, C.POINTER(ProbeIO), u32, C.c_float, vp, vp, vp, vp, vp]
         L.llmcache_fingerprint_static.argtypes = [vp, u32, u32, u32, u32, u32, vp, vp, vp, vp, vp]
         L.llmcache_fingerprint_static_error.restype = C.c_char_p
         L.llmcache_fingerprint_static_error.argtypes = []
@@ -421,6 +422,13 @@ def llmcache_infer(banks, layers, h0, B, tau, buf_a, buf_b, h_miss, miss_out, io
                                 _ptr(miss_out), C.byref(io) if io is not None else None, C.byref(final),
                                 _stream(stream)), "llmcache_infer")
     return final.value
+
+
+def llmcache_divergence_check(bank, layer, h_in, io, stride, bound, h_sample, out_sample, rel_out, counters_dev,
+                              stream=None) -> None:
+    _check(lib().llmcache_divergence_check(bank, layer, _ptr(h_in), C.byref(io), stride, bound, _ptr(h_sample),
+                                           _ptr(out_sample), _ptr(rel_out), _ptr(counters_dev), _stream(stream)),
+           "llmcache_divergence_check")
 
 
 class Layer:

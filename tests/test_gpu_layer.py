@@ -134,3 +134,52 @@ def test_infer_algorithm1_matches_oracle_and_chain_property(pre_ln):
     assert all(l.status() == L.OK for l in layers) and all(b.status() == L.OK for b in banks)
     for o in layers + banks:
         o.close()
+
+
+def test_divergence_monitor_matches_oracle():
+    """Stored outputs that no longer match what the layer produces are found and invalidated; the relative
+    differences agree with the oracle's within the layer tolerance (absolute 1e-2 on a quantity of order
+    0..1), decisions within that distance of the bound would be reported, not failed (none here)."""
+    n, d, heads, ffn, B, N, k, stride = 32, 128, 2, 256, 20, 64, 128, 3
+    w = synth.layer_weights(d, ffn, 77, DEV)
+    for key in ("w_qkv", "w_o", "w_1", "w_2"):
+        w[key] = (w[key].float() * 3.0).to(torch.bfloat16)
+    layer = L.Layer(w, heads=heads, seq_len=n, max_seqs=B)
+    bank = L.Bank(capacity=N, seq_len=n, d_model=d, fp_dim=k, max_batch=B, tau=0.9)
+    bufs = L.ProbeBuffers(B, k, DEV)
+    h = synth.randn((B, n, d), 5, DEV, torch.bfloat16)
+    h_out = torch.zeros((B, n * d), dtype=torch.bfloat16, device=DEV)
+    outs = torch.zeros((B, n, d), dtype=torch.bfloat16, device=DEV)
+    layer.forward(h, outs)
+    bank.probe(h, bufs, h_out=h_out)
+    bank.commit(outs, bufs, h_out=h_out)
+    torch.cuda.synchronize()
+    # make three stored outputs stale (slots 0, 6 and 7 are the entries of sequences 0, 6, 7)
+    act = bank.export(L.WHAT_ACT)
+    for s_, f in ((0, 1.3), (6, 0.5), (7, 1.02)):
+        act[s_] = (act[s_].float() * f).to(torch.bfloat16)
+    bank.import_(L.WHAT_ACT, act)
+    bank.probe(h, bufs, h_out=h_out)
+    bank.commit(outs, bufs, h_out=h_out)              # all hits: nothing to insert
+    torch.cuda.synchronize()
+    assert int(bufs.counts[0]) == B
+    S = (B + stride - 1) // stride
+    h_sample = torch.zeros((S, n, d), dtype=torch.bfloat16, device=DEV)
+    out_sample = torch.zeros_like(h_sample)
+    rel = torch.zeros(S, dtype=torch.float32, device=DEV)
+    cnt = torch.zeros(2, dtype=torch.int32, device=DEV)
+    from tests import parity_util as U
+    ob = U.oracle_bank_like(bank)
+    U.pull_state(bank, ob)
+    pr = U.gpu_probe_result(bufs, B, ob.tick)
+    L.llmcache_divergence_check(bank.handle, layer.handle, h, bufs.io, stride, 0.1, h_sample, out_sample, rel, cnt)
+    torch.cuda.synchronize()
+    checked, dropped = T.divergence_check(ob, oracle_weights(w), synth.bf16_bits(h), pr, heads, stride, 0.1,
+                                          round_bf16=True)
+    assert cnt.tolist() == [len(checked), dropped] and dropped == 2        # samples 0, 3, 6, ...: slots 0 and 6
+    got = rel.cpu().numpy()
+    for i, (_, slot, r) in enumerate(checked):
+        assert abs(got[i] - r) <= 1e-2, (i, slot, got[i], r)
+    assert np.array_equal(bank.export(L.WHAT_VALID).numpy(), ob.valid)
+    assert bank.status() == L.OK and layer.status() == L.OK
+    layer.close(); bank.close()

@@ -117,3 +117,25 @@ def test_infer_chain_property_of_the_caching_loop():
     near[1] = bf16_bits(O.bf16_to_f32(h0[0]) + 0.02 * r.standard_normal((n, d)).astype(np.float32))
     out3, hits3 = T.infer(banks, layers, near, heads)
     assert hits3 == [B, B, B] and np.array_equal(out3[1], out1[0])
+
+
+def test_divergence_monitor_flags_only_entries_whose_stored_output_drifted():
+    r = rng(6)
+    B, n, d, heads, ffn = 6, 8, 64, 4, 128
+    w = make_weights(r, d, ffn)
+    bank = O.Bank(capacity=16, seq_len=n, d_model=d, fp_dim=d, tau=0.9)
+    h = bf16_bits(r.standard_normal((B, n, d)))
+    outs = np.stack([T.layer_forward(h[b], w, heads).reshape(-1) for b in range(B)])
+    O.commit(bank, O.probe(bank, h, "bf16"), outs)
+    # corrupt the stored output of slot 2 (a stale entry: the layer no longer produces it)
+    bank.act[2] = bf16_bits(O.bf16_to_f32(bank.act[2]) * 1.5)
+    pr = O.probe(bank, h, "bf16")
+    assert pr.hit.sum() == B
+    checked, dropped = T.divergence_check(bank, w, h, pr, heads, stride=1, bound=0.05)
+    rels = {slot: rel for _, slot, rel in checked}
+    assert dropped == 1 and bank.valid[2] == 0 and bank.valid.sum() == B - 1
+    assert abs(rels[2] - 0.5) < 0.01 and all(rel == 0.0 for s, rel in rels.items() if s != 2)
+    # sampling: every third hit only
+    pr = O.probe(bank, h, "bf16")
+    checked, dropped = T.divergence_check(bank, w, h, pr, heads, stride=3, bound=0.05)
+    assert [b for b, _, _ in checked] == [int(pr.hit_idx[i]) for i in range(0, len(pr.hit_idx), 3)] and dropped == 0
