@@ -451,3 +451,63 @@ def evict(bank: Bank, mode: int, slots=None) -> int:
             bank.valid[j] = 0
             removed += 1
     return removed
+
+
+# --------------------------------------------------------------------------
+# SimHash fingerprints (Sec. III-A "MinHash or SimHash-based techniques"; Sec. IV-B "SimHash or PCA")
+# --------------------------------------------------------------------------
+def simhash_bits(fp_bf16: np.ndarray) -> np.ndarray:
+    """k-bit code of a fingerprint: bit c = sign bit of the projected component c (random-hyperplane
+    SimHash: the projection matrix is the hyperplane matrix).  The stored bf16 fingerprint is a positive
+    multiple of the projection, so its sign bits are the code.  Returns uint8 [B, k] of 0/1."""
+    return ((np.asarray(fp_bf16, dtype=np.uint16) >> 15) & 1).astype(np.uint8)
+
+
+def hamming_threshold(tau: float, k: int) -> int:
+    """Largest Hamming distance that still counts as a match: the angle estimate of SimHash is
+    theta = pi * ham / k, and a match needs cos(theta) > tau, i.e. ham < k * acos(tau) / pi."""
+    if tau >= 1.0:
+        return -1
+    if tau <= -1.0:
+        return k
+    x = k * float(np.arccos(np.float64(tau))) / float(np.pi)
+    h = int(np.ceil(x)) - 1          # largest integer strictly below x
+    return max(-1, min(k, h))
+
+
+def probe_simhash(bank: Bank, q_bf16, rq, tau: Optional[float] = None, h_out: Optional[np.ndarray] = None):
+    """Probe by SimHash codes: nearest occupied key in Hamming distance (ties: lowest slot), hit iff the
+    distance is within hamming_threshold(tau, k); reported score = cos(pi * ham / k) (float32).
+    Everything after the decision is as in probe_fp.  Returns (ProbeResult, ham int32 [B])."""
+    bank.tick += 1
+    tau = bank.tau if tau is None else tau
+    k = bank.fp_dim
+    qb = simhash_bits(q_bf16)
+    kb = simhash_bits(bank.fp)
+    B = qb.shape[0]
+    ham = np.full((B,), -1, dtype=np.int32)
+    best = np.full((B,), -np.inf, dtype=np.float32)
+    bslot = np.full((B,), -1, dtype=np.int32)
+    occ = np.nonzero(bank.valid)[0]
+    for b in range(B):
+        if rq[b] <= 0:
+            best[b] = 0.0
+            continue
+        if len(occ) == 0:
+            continue
+        d = (kb[occ] != qb[b][None, :]).sum(axis=1)
+        i = int(np.argmin(d))                      # first minimum = lowest slot
+        ham[b] = int(d[i])
+        bslot[b] = int(occ[i])
+        best[b] = np.float32(np.cos(np.pi * float(d[i]) / k))
+    hmax = hamming_threshold(tau, k)
+    hit = ((ham >= 0) & (ham <= hmax)).astype(np.uint8)
+    slot = np.where(hit != 0, bslot, -1).astype(np.int32)
+    hit_idx, miss_idx = compact(hit)
+    if h_out is not None and bank.act is not None:
+        for b in hit_idx.tolist():
+            h_out[b] = bank.act[int(slot[b]) % bank.act_rows]
+    touch(bank, slot[hit_idx])
+    pr = ProbeResult(fp=q_bf16, rq=rq, score=best, second=None, best_slot=bslot, hit=hit, slot=slot,
+                     hit_idx=hit_idx, miss_idx=miss_idx, tick=bank.tick)
+    return pr, ham

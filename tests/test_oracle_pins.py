@@ -533,3 +533,43 @@ def test_act_rows_aliasing_maps_slot_modulo():
     pr = O.probe(bank, h, "f32", h_out=h_out)
     assert pr.slot.tolist() == list(range(6))
     assert np.array_equal(h_out[5], acts[5]) and np.array_equal(h_out[1], acts[5])   # rows 1 and 5 share storage
+
+
+# --------------------------------------------------------------------------------- SimHash ---
+def test_simhash_bits_hamming_brute_force_and_threshold():
+    r = rng(40)
+    g = r.standard_normal((6, 64))
+    q, rq = O.normalise(g)
+    bits_ = O.simhash_bits(q)
+    assert np.array_equal(bits_, (g < 0).astype(np.uint8))                 # sign of the projection
+    assert O.hamming_threshold(1.0, 256) == -1 and O.hamming_threshold(-1.0, 256) == 256
+    for tau in (0.0, 0.5, 0.82, 0.9):
+        hm = O.hamming_threshold(tau, 256)
+        assert math.cos(math.pi * hm / 256) > tau >= math.cos(math.pi * (hm + 1) / 256) - 1e-12
+    bank = _mk_bank(N=8, n=2, d=64, k=64)
+    base = _rand_h(r, 5, 2, 64)
+    O.commit(bank, O.probe(bank, base, "f32"), _rand_act(r, 5, 2, 64))
+    qh = base[[3, 1]] + 0.05 * _rand_h(r, 2, 2, 64)
+    fq, rqq = O.fingerprint(qh, "f32")
+    pr, ham = O.probe_simhash(bank, fq, rqq, tau=0.8)
+    for b in range(2):
+        qb = [int(x) >> 15 for x in fq[b]]
+        dist = [sum(1 for c in range(64) if qb[c] != (int(bank.fp[j][c]) >> 15)) for j in range(5)]
+        assert ham[b] == min(dist) and pr.best_slot[b] == dist.index(min(dist))
+        assert abs(pr.score[b] - math.cos(math.pi * min(dist) / 64)) < 1e-6
+    assert pr.slot.tolist() == [3, 1]
+    fs, rs = O.fingerprint(base[:1], "f32")                                 # identical input: distance 0, score 1
+    pr, ham = O.probe_simhash(bank, fs, rs, tau=0.99)
+    assert ham[0] == 0 and pr.score[0] == 1.0 and pr.hit[0] == 1
+
+
+def test_simhash_angle_estimate_is_unbiased_for_random_hyperplanes():
+    # P(sign differs) = theta / pi for a random hyperplane: the mean normalised distance estimates the angle
+    r = rng(41)
+    d, k = 48, 4096
+    a = r.standard_normal(d); b = a + 0.6 * r.standard_normal(d)
+    theta = math.acos(float(a @ b / (np.linalg.norm(a) * np.linalg.norm(b))))
+    P = r.standard_normal((d, k))
+    ha = O.simhash_bits(O.normalise((a @ P)[None])[0]); hb = O.simhash_bits(O.normalise((b @ P)[None])[0])
+    frac = float((ha != hb).mean())
+    assert abs(frac - theta / math.pi) < 4 * math.sqrt(0.25 / k)
