@@ -201,6 +201,15 @@ const char* llmcache_fingerprint_static_error(void);
 int llmcache_probe(llmcache_bank_t* bank, const void* h_in, uint32_t B, float tau,
                    void* h_out, llmcache_probe_io* io, void* stream);
 
+/* Lookup by SimHash codes (Sec. III-A, IV-B: "SimHash ... compact and comparable vectors"): the code of a
+ * fingerprint is the sign bit of each projected component (the projection matrix is the random-hyperplane
+ * matrix), k bits per key instead of 2k bytes.  The scan finds the occupied key nearest in Hamming distance
+ * (ties: lowest slot); hit iff cos(pi * ham / k) > tau, i.e. ham < k * acos(tau) / pi; io->score receives
+ * that angle estimate.  Everything else (compaction, gather, metadata, commit) is as in llmcache_probe.
+ * The bank's codes are re-packed from its stored fingerprints when these changed since the last call. */
+int llmcache_probe_simhash(llmcache_bank_t* bank, const void* h_in, uint32_t B, float tau,
+                           void* h_out, llmcache_probe_io* io, void* stream);
+
 /* Same with precomputed fingerprints (Algorithm 1 computes f_X once and reuses
  * it at every layer): io->fp holds bf16 [B,k] on entry; io->rq is written.
  * h_in may be NULL (then io->h_miss is not produced). */

@@ -33,7 +33,7 @@ EXPORTS = [
     "llmcache_bank_stats", "llmcache_bank_status", "llmcache_bank_profile", "llmcache_bank_profile_read",
     "llmcache_fingerprint_static", "llmcache_fingerprint_static_error",
     "llmcache_layer_bytes", "llmcache_layer_create", "llmcache_layer_destroy", "llmcache_layer_forward",
-    "llmcache_layer_status", "llmcache_infer", "llmcache_divergence_check",
+    "llmcache_layer_status", "llmcache_infer", "llmcache_divergence_check", "llmcache_probe_simhash",
 ]
 FINGERPRINT_STATIC_MAX_FLOATS = 2 * 1024 * 1024
 KERNEL_NAMES = ["pool", "project", "rownorm", "scan", "decide", "touch", "gather", "select", "scatter", "evict"]
@@ -110,6 +110,7 @@ def lib():
         L.llmcache_fingerprint.argtypes = [vp, vp, u32, vp, vp, vp]
         L.llmcache_probe.argtypes = [vp, vp, u32, C.c_float, vp, C.POINTER(ProbeIO), vp]
         L.llmcache_probe_fp.argtypes = [vp, vp, u32, C.c_float, vp, C.POINTER(ProbeIO), vp]
+        L.llmcache_probe_simhash.argtypes = [vp, vp, u32, C.c_float, vp, C.POINTER(ProbeIO), vp]
         L.llmcache_commit.argtypes = [vp, vp, C.POINTER(ProbeIO), vp, i32p, vp]
         L.llmcache_evict.argtypes = [vp, u32, vp, u32, vp, vp]
         L.llmcache_bank_export.argtypes = [vp, u32, vp, C.c_size_t, vp]
@@ -221,6 +222,12 @@ def llmcache_probe(bank, h_in, B, tau, h_out, io: ProbeIO, stream=None) -> None:
     tau = float("nan") if tau is None else tau
     _check(lib().llmcache_probe(bank, _ptr(h_in), B, tau, _ptr(h_out), C.byref(io), _stream(stream)),
            "llmcache_probe")
+
+
+def llmcache_probe_simhash(bank, h_in, B, tau, h_out, io: ProbeIO, stream=None) -> None:
+    tau = float("nan") if tau is None else tau
+    _check(lib().llmcache_probe_simhash(bank, _ptr(h_in), B, tau, _ptr(h_out), C.byref(io), _stream(stream)),
+           "llmcache_probe_simhash")
 
 
 def llmcache_probe_fp(bank, h_in, B, tau, h_out, io: ProbeIO, stream=None) -> None:

@@ -17,7 +17,7 @@ inline uint32_t pow2_ceil(uint32_t x) { uint32_t p = 1; while (p < x) p <<= 1; r
 
 struct Layout {
   size_t fp, rb, valid, last_use, insert_tick, hits, rate, rate_epoch, act, proj, center;
-  size_t pool_partial, best, hitcnt, victims, new_slot, sort_key, sort_slot, stats, status, misc, total;
+  size_t pool_partial, best, hitcnt, victims, new_slot, bits, qbits, sort_key, sort_slot, stats, status, misc, total;
   uint32_t sort_len;
 };
 
@@ -76,6 +76,8 @@ Layout make_layout(const llmcache_bank_desc& d) {
   const uint32_t vmax = d.max_batch < d.capacity ? d.max_batch : d.capacity;
   L.victims = take((size_t)vmax * 4);
   L.new_slot = take((size_t)d.max_batch * 4);
+  L.bits = take(N * (k / 8));
+  L.qbits = take((size_t)d.max_batch * (k / 8));
   L.sort_len = pow2_ceil(vmax);
   L.sort_key = take((size_t)L.sort_len * 8);
   L.sort_slot = take((size_t)L.sort_len * 4);
@@ -211,6 +213,8 @@ int llmcache_bank_create(const llmcache_bank_desc* desc, llmcache_bank_t** bank_
   a.hitcnt = (uint32_t*)(base + L.hitcnt);
   a.victims = (int32_t*)(base + L.victims);
   a.new_slot = (int32_t*)(base + L.new_slot);
+  a.bits = (uint32_t*)(base + L.bits);
+  a.qbits = (uint32_t*)(base + L.qbits);
   a.sort_key = (unsigned long long*)(base + L.sort_key);
   a.sort_slot = (uint32_t*)(base + L.sort_slot);
   a.stats = (unsigned long long*)(base + L.stats);
@@ -269,8 +273,21 @@ int llmcache_fingerprint(llmcache_bank_t* bk, const void* h_in, uint32_t B, void
   return e == cudaSuccess ? LLMCACHE_OK : cuda_fail(e, __func__);
 }
 
+// Largest Hamming distance that still matches: the SimHash angle estimate is pi * ham / k and a match
+// needs cos(angle) > tau, i.e. ham < k * acos(tau) / pi.
+static int32_t hamming_threshold(float tau, uint32_t k) {
+  const double t = (double)tau;
+  if (t >= 1.0) return -1;
+  if (t <= -1.0) return (int32_t)k;
+  const double x = (double)k * std::acos(t) / 3.14159265358979323846;
+  long h = (long)std::ceil(x) - 1;
+  if (h < -1) h = -1;
+  if (h > (long)k) h = (long)k;
+  return (int32_t)h;
+}
+
 static int probe_common(llmcache_bank_t* bk, const void* h_in, bool compute_fp, uint32_t B, float tau,
-                        void* h_out, llmcache_probe_io* io, void* stream) {
+                        void* h_out, llmcache_probe_io* io, void* stream, bool simhash = false) {
   if (!bk) return LLMCACHE_ERR_ARG;
   if (B > bk->desc.max_batch) return LLMCACHE_ERR_SHAPE;
   if (B) {
@@ -303,8 +320,13 @@ static int probe_common(llmcache_bank_t* bk, const void* h_in, bool compute_fp, 
   } else {
     if (compute_fp) e = launch_fingerprint(bk, h_in, B, (__nv_bfloat16*)io->fp, io->rq, st);
     else            e = launch_rownorm(bk, (const __nv_bfloat16*)io->fp, B, bk->desc.fp_dim, io->rq, st);
-    if (e == cudaSuccess) e = launch_scan(bk, (const __nv_bfloat16*)io->fp, B, st);
-    if (e == cudaSuccess) e = launch_decide(bk, B, tau, io->rq, io, st);
+    if (simhash) {
+      if (e == cudaSuccess) e = launch_simhash_scan(bk, (const __nv_bfloat16*)io->fp, B, st);
+      if (e == cudaSuccess) e = launch_decide(bk, B, tau, io->rq, io, st, bk->desc.fp_dim, hamming_threshold(tau, bk->desc.fp_dim));
+    } else {
+      if (e == cudaSuccess) e = launch_scan(bk, (const __nv_bfloat16*)io->fp, B, st);
+      if (e == cudaSuccess) e = launch_decide(bk, B, tau, io->rq, io, st);
+    }
     // The slots for this batch's misses are chosen now, on the side stream, while the gather runs:
     // the choice depends only on the metadata after this probe's refresh, which the gather does not touch.
     if (e == cudaSuccess) e = cudaEventRecord(bk->ev_fork, st);
@@ -323,6 +345,11 @@ static int probe_common(llmcache_bank_t* bk, const void* h_in, bool compute_fp, 
 int llmcache_probe(llmcache_bank_t* bk, const void* h_in, uint32_t B, float tau, void* h_out,
                    llmcache_probe_io* io, void* stream) {
   return probe_common(bk, h_in, true, B, tau, h_out, io, stream);
+}
+
+int llmcache_probe_simhash(llmcache_bank_t* bk, const void* h_in, uint32_t B, float tau, void* h_out,
+                           llmcache_probe_io* io, void* stream) {
+  return probe_common(bk, h_in, true, B, tau, h_out, io, stream, true);
 }
 
 int llmcache_probe_fp(llmcache_bank_t* bk, const void* h_in, uint32_t B, float tau, void* h_out,
@@ -353,6 +380,7 @@ int llmcache_commit(llmcache_bank_t* bk, const void* miss_out, const llmcache_pr
     e = cudaStreamWaitEvent(st, bk->ev_join, 0);
     bk->join_pending = false;
   }
+  bk->bits_dirty = true;
   if (e == cudaSuccess) e = launch_scatter_insert(bk, miss_out, io, h_out, new_slot, B, st);
   if (e != cudaSuccess) return cuda_fail(e, __func__);
   return LLMCACHE_OK;
@@ -404,6 +432,7 @@ int llmcache_bank_import(llmcache_bank_t* bk, uint32_t what, const void* ptr, si
   int rc = array_of(bk, what, &dst, &sz);
   if (rc != LLMCACHE_OK) return rc;
   if (bytes != sz) return LLMCACHE_ERR_SHAPE;
+  if (what == LLMCACHE_WHAT_FP) bk->bits_dirty = true;
   cudaError_t e = cudaMemcpyAsync(dst, ptr, sz, cudaMemcpyDefault, (cudaStream_t)stream);
   if (e != cudaSuccess) return cuda_fail(e, __func__);
   return LLMCACHE_OK;

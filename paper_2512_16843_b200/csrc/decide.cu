@@ -36,7 +36,8 @@ k_decide_compact(unsigned long long* __restrict__ best, const float* __restrict_
                  uint32_t* __restrict__ counts, uint32_t* __restrict__ hitcnt,
                  unsigned long long* __restrict__ stats,
                  uint32_t* __restrict__ last_use, uint32_t* __restrict__ hits_total, uint32_t* __restrict__ rate,
-                 uint32_t* __restrict__ rate_epoch, uint32_t tick, uint32_t epoch) {
+                 uint32_t* __restrict__ rate_epoch, uint32_t tick, uint32_t epoch,
+                 uint32_t sim_k, int32_t ham_max) {
   griddep_sync();
   __shared__ uint32_t warp_tot[32];
   uint32_t hbase = 0, mbase = 0, ndegen = 0;
@@ -55,9 +56,16 @@ k_decide_compact(unsigned long long* __restrict__ best, const float* __restrict_
       } else if (pk == 0ull) {
         sc = -INFINITY;                                 // no occupied slot
       } else {
-        sc = orderable_float((uint32_t)(pk >> 32)) * r;
         sl = (int32_t)(0xFFFFFFFFu - (uint32_t)pk);
-        is_hit = cmp_ge ? (sc >= tau) : (sc > tau);
+        if (sim_k) {
+          // SimHash scan: the upper word is the inverted Hamming distance; the angle estimate is pi * ham / k
+          const uint32_t ham = 0xFFFFFFFFu - (uint32_t)(pk >> 32);
+          sc = cospif((float)ham / (float)sim_k);
+          is_hit = (int32_t)ham <= ham_max;
+        } else {
+          sc = orderable_float((uint32_t)(pk >> 32)) * r;
+          is_hit = cmp_ge ? (sc >= tau) : (sc > tau);
+        }
       }
       if (!is_hit) sl = -1;
       hit[b] = is_hit ? 1 : 0;
@@ -111,12 +119,12 @@ k_decide_compact(unsigned long long* __restrict__ best, const float* __restrict_
 }
 
 cudaError_t launch_decide(llmcache_bank* bk, uint32_t B, float tau, const float* rq,
-                          const llmcache_probe_io* io, cudaStream_t st) {
+                          const llmcache_probe_io* io, cudaStream_t st, uint32_t sim_k, int32_t ham_max) {
   ProfScope prof(bk, LLMCACHE_K_DECIDE, st);
   return launch_k(k_decide_compact, dim3(1), dim3(DEC_THREADS), 0, st, bk->a.best, rq, B, tau,
                   (int)(bk->desc.cmp == LLMCACHE_GE), io->hit, io->slot, io->score, io->hit_idx, io->miss_idx,
                   io->counts, bk->a.hitcnt, bk->a.stats, bk->a.last_use, bk->a.hits, bk->a.rate, bk->a.rate_epoch,
-                  (uint32_t)bk->tick, (uint32_t)(bk->tick / bk->pol.half_life));
+                  (uint32_t)bk->tick, (uint32_t)(bk->tick / bk->pol.half_life), sim_k, ham_max);
 }
 
 }  // namespace llmc

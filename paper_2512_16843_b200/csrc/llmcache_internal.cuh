@@ -39,6 +39,8 @@ struct BankArrays {
   unsigned long long* best; // [max_batch] packed (orderable score << 32 | ~slot); 0 = none
   uint32_t* hitcnt;         // [N] matches per slot within the current probe (zero between calls)
   int32_t*  victims;        // [min(max_batch,N)]
+  uint32_t* bits;           // [N, k/32] SimHash codes of the stored fingerprints (sign bits), packed lazily
+  uint32_t* qbits;          // [max_batch, k/32]
   int32_t*  new_slot;       // [max_batch] slot each miss of the open probe will be stored in (-1: dropped)
   unsigned long long* sort_key;   // [pow2 >= min(max_batch,N)]
   uint32_t* sort_slot;      // same length
@@ -70,6 +72,7 @@ struct llmcache_bank {
   cudaStream_t side = nullptr;
   cudaEvent_t  ev_fork = nullptr, ev_join = nullptr;
   bool     join_pending = false;
+  bool     bits_dirty = true;    // stored fingerprints changed since the SimHash codes were packed
   // instrumentation
   uint64_t n_launches = 0;
   bool     prof_on = false;
@@ -107,7 +110,8 @@ cudaError_t launch_fingerprint(llmcache_bank* bk, const void* h_in, uint32_t B,
 cudaError_t launch_rownorm(llmcache_bank* bk, const __nv_bfloat16* fp, uint32_t B, uint32_t k, float* rq, cudaStream_t st);
 cudaError_t launch_scan(llmcache_bank* bk, const __nv_bfloat16* q, uint32_t B, cudaStream_t st);
 cudaError_t launch_decide(llmcache_bank* bk, uint32_t B, float tau, const float* rq,
-                          const llmcache_probe_io* io, cudaStream_t st);
+                          const llmcache_probe_io* io, cudaStream_t st, uint32_t sim_k = 0, int32_t ham_max = -1);
+cudaError_t launch_simhash_scan(llmcache_bank* bk, const __nv_bfloat16* q, uint32_t B, cudaStream_t st);
 cudaError_t launch_gather(llmcache_bank* bk, const void* h_in, void* h_out,
                           const llmcache_probe_io* io, uint32_t B, cudaStream_t st);
 cudaError_t launch_select_victims(llmcache_bank* bk, const llmcache_probe_io* io, uint32_t B, cudaStream_t st);

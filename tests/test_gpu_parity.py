@@ -289,3 +289,44 @@ def test_arena_supplied_by_caller_and_repeatability():
     with pytest.raises(L.LLMCacheError) as e:
         L.Bank(capacity=64, seq_len=8, d_model=64, fp_dim=64, max_batch=16, arena=arena.data_ptr() + off, arena_bytes=1024)
     assert e.value.status == L.ERR_NOMEM
+
+
+@pytest.mark.parametrize("N,n,d,k,B", [(300, 8, 128, 128, 70), (2048, 4, 768, 256, 256)])
+def test_simhash_probe_matches_oracle_bit_for_bit(N, n, d, k, B):
+    """SimHash lookup is integer work on the sign codes of the fingerprints: distances, slots, flags, gathered
+    rows and metadata must match the oracle exactly (the oracle is given the GPU's query fingerprints, which
+    are checked against its own within the usual tolerance); the reported angle estimate within 1e-6."""
+    proj = synth.projection(d, k, 3, DEV) if k != d else None
+    gb, ob = make_pair(N, n, d, k, B, "bf16", proj, None, tau=0.8)
+    bufs = L.ProbeBuffers(B, k, DEV)
+    base = rand_h(B, n, d, 61, "bf16")
+    for step in range(3):
+        h = base.clone()
+        if step:                                         # two thirds noisy repeats, one third new
+            h[: 2 * B // 3] = (base[: 2 * B // 3].float() + 0.15 * synth.randn((2 * B // 3, n, d), 70 + step, DEV)).to(torch.bfloat16)
+            h[2 * B // 3:] = rand_h(B - 2 * B // 3, n, d, 80 + step, "bf16")
+        U.pull_state(gb, ob)
+        h_out = torch.zeros((B, n * d), dtype=torch.bfloat16, device=DEV)
+        L.llmcache_probe_simhash(gb.handle, h, B, None, h_out, bufs.io)
+        torch.cuda.synchronize()
+        fq, rq = O.fingerprint(U.bits(h), "bf16", ob.proj, ob.center)
+        U.compare_fingerprints(U.bits(bufs.fp[:B]), bufs.rq[:B].cpu().numpy(), fq, rq)
+        exp_out = np.zeros((B, n * d), dtype=np.uint16)
+        pr, ham = O.probe_simhash(ob, U.bits(bufs.fp[:B]), bufs.rq[:B].cpu().numpy(), 0.8, exp_out)
+        assert np.array_equal(bufs.hit[:B].cpu().numpy(), pr.hit)
+        assert np.array_equal(bufs.slot[:B].cpu().numpy(), pr.slot)
+        assert np.allclose(bufs.score[:B].cpu().numpy(), pr.score, rtol=0, atol=1e-6)
+        H = int(pr.hit.sum())
+        assert bufs.counts.tolist() == [H, B - H]
+        assert np.array_equal(U.bits(h_out), exp_out)
+        U.assert_state_equal(gb, ob, with_act=False, where="after simhash probe")
+        mo = synth.activations(B, n, d, 90 + step, DEV)
+        gb.commit(mo, bufs, h_out=h_out)
+        torch.cuda.synchronize()
+        gp = U.gpu_probe_result(bufs, B, ob.tick)
+        new = O.commit(ob, gp, U.bits(mo[:B - H]), exp_out)
+        assert np.array_equal(bufs.new_slot[:B - H].cpu().numpy(), new)
+        U.assert_state_equal(gb, ob, where="after commit")
+        if step:
+            assert 0 < H < B
+    gb.close()
