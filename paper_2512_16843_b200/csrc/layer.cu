@@ -65,7 +65,7 @@ k_layernorm(const __nv_bfloat16* __restrict__ x, const float* __restrict__ g, co
 // Multi-head scaled dot-product self-attention, head size 64, on tensor cores (mma.sync m16n8k16,
 // bf16 inputs, fp32 accumulation).  One block of 4 warps per (sequence, head, tile of 64 queries);
 // a warp owns 16 query rows.  Keys and values pass through shared memory in tiles of 64 positions
-// (16-byte chunks XOR-swizzled by row so that ldmatrix is conflict-free); S = Q K^T stays in
+// (cp.async, double-buffered; 16-byte chunks XOR-swizzled by row so that ldmatrix is conflict-free); S = Q K^T stays in
 // registers, softmax is computed on line (running maximum and sum per row), P is re-used as the A
 // operand of P V straight from the accumulator layout.  causal: position i attends to j <= i.
 // qkv: [tokens, 3d] (q | k | v per token); out: [tokens, d].
@@ -92,11 +92,11 @@ __device__ __forceinline__ uint32_t pack2_bf16(float a, float b) {
 // byte offset of 16-byte chunk `c` (0..7) of row `r` in a [64][64] bf16 tile
 __device__ __forceinline__ uint32_t tile_off(uint32_t r, uint32_t c) { return r * 128u + ((c ^ (r & 7u)) << 4); }
 
-__global__ void __launch_bounds__(ATT_THREADS)
+__global__ void __launch_bounds__(ATT_THREADS, 4)
 k_attention(const __nv_bfloat16* __restrict__ qkv, __nv_bfloat16* __restrict__ out, uint32_t n, uint32_t d,
             uint32_t heads, uint32_t seq_max, const uint32_t* __restrict__ m_seq_dev, int causal) {
   griddep_sync();
-  __shared__ __align__(128) uint8_t sq[ATT_Q * 128], sk[ATT_KT * 128], sv[ATT_KT * 128];
+  __shared__ __align__(128) uint8_t sq[ATT_Q * 128], sk[2][ATT_KT * 128], sv[2][ATT_KT * 128];   // K/V double-buffered
   uint32_t n_seq = seq_max;
   if (m_seq_dev) n_seq = min(seq_max, *m_seq_dev);
   const uint32_t qtiles = (n + ATT_Q - 1) / ATT_Q;
@@ -117,6 +117,20 @@ k_attention(const __nv_bfloat16* __restrict__ qkv, __nv_bfloat16* __restrict__ o
       *reinterpret_cast<uint4*>(dst + tile_off(r, c)) = w;
     }
   };
+  // same, asynchronously (cp.async, 16 bytes per copy); rows beyond the sequence are zero-filled
+  auto stage_async = [&](uint8_t* dst, uint32_t which, uint32_t p0) {
+    for (uint32_t idx = threadIdx.x; idx < 64 * 8; idx += ATT_THREADS) {
+      const uint32_t r = idx >> 3, c = idx & 7u;
+      const uint32_t sa = smem_u32_of(dst) + tile_off(r, c);
+      if (p0 + r < n) {
+        const __nv_bfloat16* src = qkv + (tok0 + p0 + r) * 3 * d + which * d + h * ATT_DH + c * 8;
+        asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(sa), "l"(src) : "memory");
+      } else {
+        *reinterpret_cast<uint4*>(dst + tile_off(r, c)) = make_uint4(0, 0, 0, 0);
+      }
+    }
+    asm volatile("cp.async.commit_group;" ::: "memory");
+  };
   stage(sq, 0, q0);
   __syncthreads();
   // Q fragments of this warp's 16 rows: 4 k-steps of 16 head dims
@@ -135,11 +149,21 @@ k_attention(const __nv_bfloat16* __restrict__ qkv, __nv_bfloat16* __restrict__ o
   const uint32_t j_end = causal ? last_q + 1 : n;
   const float scale = 0.125f;                                                       // 1 / sqrt(64)
 
-  for (uint32_t j0 = 0; j0 < j_end; j0 += ATT_KT) {
+  stage_async(sk[0], 1, 0);
+  stage_async(sv[0], 2, 0);
+  uint32_t cur = 0;
+  for (uint32_t j0 = 0; j0 < j_end; j0 += ATT_KT, cur ^= 1u) {
+    // fetch the next tile into the other buffer while this one is used
+    if (j0 + ATT_KT < j_end) {
+      stage_async(sk[cur ^ 1u], 1, j0 + ATT_KT);
+      stage_async(sv[cur ^ 1u], 2, j0 + ATT_KT);
+      asm volatile("cp.async.wait_group 2;" ::: "memory");          // the two groups of the current tile are done
+    } else {
+      asm volatile("cp.async.wait_group 0;" ::: "memory");
+    }
     __syncthreads();
-    stage(sk, 1, j0);
-    stage(sv, 2, j0);
-    __syncthreads();
+    const uint8_t* skc = sk[cur];
+    const uint8_t* svc = sv[cur];
     // S = Q K^T for 16 rows x 64 keys
     float sacc[8][4];
 #pragma unroll
@@ -151,7 +175,7 @@ k_attention(const __nv_bfloat16* __restrict__ qkv, __nv_bfloat16* __restrict__ o
         uint32_t kb[4];
         const uint32_t mi = lane >> 3;
         const uint32_t krow = np * 16 + (mi >> 1) * 8 + (lane & 7u);
-        ldsm_x4(smem_u32_of(sk) + tile_off(krow, ks * 2 + (mi & 1u)), kb);
+        ldsm_x4(smem_u32_of(skc) + tile_off(krow, ks * 2 + (mi & 1u)), kb);
         mma_bf16_16816(sacc[np * 2], qa[ks], kb[0], kb[1]);
         mma_bf16_16816(sacc[np * 2 + 1], qa[ks], kb[2], kb[3]);
       }
@@ -210,11 +234,12 @@ k_attention(const __nv_bfloat16* __restrict__ qkv, __nv_bfloat16* __restrict__ o
         uint32_t vb[4];
         const uint32_t mi = lane >> 3;
         const uint32_t vrow = kk * 16 + (mi & 1u) * 8 + (lane & 7u);
-        ldsm_x4_t(smem_u32_of(sv) + tile_off(vrow, np * 2 + (mi >> 1)), vb);
+        ldsm_x4_t(smem_u32_of(svc) + tile_off(vrow, np * 2 + (mi >> 1)), vb);
         mma_bf16_16816(o[np * 2], pa, vb[0], vb[1]);
         mma_bf16_16816(o[np * 2 + 1], pa, vb[2], vb[3]);
       }
     }
+    __syncthreads();                                                 // all warps are done with this buffer
   }
   // normalise and store: thread holds rows g, g+8, columns i*8 + 2*t4 .. +1
 #pragma unroll
