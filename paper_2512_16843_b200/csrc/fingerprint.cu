@@ -238,15 +238,22 @@ k_project(const float* __restrict__ partial, const __nv_bfloat16* __restrict__ p
           }
         };
         constexpr int INFL = 8;                                    // rows in flight
-        uint32_t i = sl;
-        for (; i + (INFL - 1) * slices < d; i += INFL * slices) {
+        // This thread's rows are sl, sl + slices, ...  Every block reads the same matrix, so each block
+        // starts at a different one of them (and wraps): the blocks then ask for different lines at any
+        // moment instead of all hitting one L2 line together.
+        const uint32_t nrow = sl < d ? (d - sl + slices - 1) / slices : 0u;
+        const uint32_t rot = nrow ? (blockIdx.x * 5u) % nrow : 0u;
+        auto row_of = [&](uint32_t t) { uint32_t tt = t + rot; if (tt >= nrow) tt -= nrow; return sl + tt * slices; };
+        uint32_t t = 0;
+        for (; t + INFL <= nrow; t += INFL) {
           uint4 w[INFL];
+          uint32_t ri[INFL];
 #pragma unroll
-          for (int u = 0; u < INFL; ++u) w[u] = ld_nc16(P4 + (size_t)(i + u * slices) * ncg + cg);
+          for (int u = 0; u < INFL; ++u) { ri[u] = row_of(t + u); w[u] = ld_nc16(P4 + (size_t)ri[u] * ncg + cg); }
 #pragma unroll
-          for (int u = 0; u < INFL; ++u) fma_row(w[u], i + u * slices);
+          for (int u = 0; u < INFL; ++u) fma_row(w[u], ri[u]);
         }
-        for (; i < d; i += slices) fma_row(ld_nc16(P4 + (size_t)i * ncg + cg), i);
+        for (; t < nrow; ++t) { const uint32_t i = row_of(t); fma_row(ld_nc16(P4 + (size_t)i * ncg + cg), i); }
 #pragma unroll
         for (int gi = 0; gi < PROJ_G; ++gi)
 #pragma unroll
