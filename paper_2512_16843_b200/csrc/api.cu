@@ -329,11 +329,16 @@ static int probe_common(llmcache_bank_t* bk, const void* h_in, bool compute_fp, 
     }
     // The slots for this batch's misses are chosen now, on the side stream, while the gather runs:
     // the choice depends only on the metadata after this probe's refresh, which the gather does not touch.
-    if (e == cudaSuccess) e = cudaEventRecord(bk->ev_fork, st);
-    if (e == cudaSuccess) e = cudaStreamWaitEvent(bk->side, bk->ev_fork, 0);
-    if (e == cudaSuccess) e = launch_select_victims(bk, io, B, bk->side);
-    if (e == cudaSuccess) e = cudaEventRecord(bk->ev_join, bk->side);
-    if (e == cudaSuccess) bk->join_pending = true;
+    // (A one-block pass over a very large bank takes milliseconds; there it is left to the commit, so that
+    // probes that are never committed do not pay for it.)
+    bk->select_deferred = bk->desc.capacity > 65536u;
+    if (!bk->select_deferred) {
+      if (e == cudaSuccess) e = cudaEventRecord(bk->ev_fork, st);
+      if (e == cudaSuccess) e = cudaStreamWaitEvent(bk->side, bk->ev_fork, 0);
+      if (e == cudaSuccess) e = launch_select_victims(bk, io, B, bk->side);
+      if (e == cudaSuccess) e = cudaEventRecord(bk->ev_join, bk->side);
+      if (e == cudaSuccess) bk->join_pending = true;
+    }
     if (e == cudaSuccess) e = launch_gather(bk, h_in, h_out, io, B, st);
   }
   if (e == cudaSuccess && io->counts_host && io->counts)
@@ -381,6 +386,8 @@ int llmcache_commit(llmcache_bank_t* bk, const void* miss_out, const llmcache_pr
     bk->join_pending = false;
   }
   bk->bits_dirty = true;
+  if (e == cudaSuccess && bk->select_deferred) e = launch_select_victims(bk, io, B, st);
+  bk->select_deferred = false;
   if (e == cudaSuccess) e = launch_scatter_insert(bk, miss_out, io, h_out, new_slot, B, st);
   if (e != cudaSuccess) return cuda_fail(e, __func__);
   return LLMCACHE_OK;

@@ -72,6 +72,7 @@ struct llmcache_bank {
   cudaStream_t side = nullptr;
   cudaEvent_t  ev_fork = nullptr, ev_join = nullptr;
   bool     join_pending = false;
+  bool     select_deferred = false;   // large bank: the victim selection runs at commit instead
   bool     bits_dirty = true;    // stored fingerprints changed since the SimHash codes were packed
   // instrumentation
   uint64_t n_launches = 0;
