@@ -37,6 +37,86 @@ UNIT = "sequences/s"
 CFG = dict(layers=12, d_model=768, seq_len=384, batch=256, vocab=30522, n_seeds=64, edit_fraction=0.60,
            edit_positions=0.10, bank=2048, fp_dim=256, tau=0.90, pool_batches=24)
 
+# Other shapes of the same step (parity-test configurations; `--workload`): not the headline line.
+WORKLOADS = {
+    "bert_base": CFG,
+    # GPT-2-small-shaped decoder: batch 32 x seq_len 1024, half of each batch are repeats of 64 hot documents
+    # (512-token prefix of one of 8 seed documents + fixed suffix), half have fresh random suffixes
+    "gpt2_small": dict(layers=12, d_model=768, seq_len=1024, batch=32, vocab=50257, n_seeds=8, bank=1024, fp_dim=256,
+                       tau=0.90, pool_batches=24, kind="prefix", hot=64, prefix=512, repeat_fraction=0.5),
+    # BERT-large-shaped encoder under churn: batch 512 x seq_len 512, 75% near one of 256 drifting centres
+    # (shift 0.02 per batch, noise 0.05), 25% junk that never repeats, LRU + staleness eviction
+    "bert_large_churn": dict(layers=24, d_model=1024, seq_len=512, batch=512, bank=1024, fp_dim=256, tau=0.90,
+                             pool_batches=10, kind="cluster", centres=256, near_fraction=0.75, drift=0.02, noise=0.05),
+}
+
+
+def describe(name, cfg):
+    head = {"bert_base": "BERT-base-shaped encoder", "gpt2_small": "GPT-2-small-shaped decoder",
+            "bert_large_churn": "BERT-large-shaped encoder under churn"}[name]
+    tail = {"bert_base": "60% token-level edits of 64 seeds",
+            "gpt2_small": "half repeats of 64 hot documents (512-token shared prefixes), half fresh suffixes",
+            "bert_large_churn": "75% near 256 drifting centres (shift 0.02 per batch), 25% junk, LRU + staleness eviction"}[name]
+    return (f"{head}: {cfg['layers']} per-layer banks x {cfg['bank']} entries (bf16 {cfg['seq_len']}x{cfg['d_model']}), "
+            f"batch {cfg['batch']} x seq_len {cfg['seq_len']}, d_model {cfg['d_model']}, fp_dim {cfg['fp_dim']} (projected), "
+            f"tau {cfg['tau']:.2f}, {tail}")
+
+
+def make_inputs(cfg, seed, dev):
+    """(warm batches, rotating pool of batches) of bf16 hidden states [B, n, d] for a workload."""
+    from paper_2512_16843_b200 import synth
+    B, n, d, N, P = cfg["batch"], cfg["seq_len"], cfg["d_model"], cfg["bank"], cfg["pool_batches"]
+    kind = cfg.get("kind", "edits")
+    if kind == "edits":
+        wl = synth.TokenWorkload(cfg["vocab"], n, d, seed, dev)
+        seeds_tok = wl.tokens(cfg["n_seeds"], seed + 5)
+        pool = build_batches(wl, seeds_tok, P, seed + 1000, dev)
+        warm = [wl.hidden(torch.cat([seeds_tok, wl.tokens(B - cfg["n_seeds"], seed + 7)]))]
+        warm += [wl.hidden(wl.tokens(B, seed + 20 + i)) for i in range(1, N // B)]
+        return warm, pool
+    if kind == "prefix":
+        wl = synth.TokenWorkload(cfg["vocab"], n, d, seed, dev)
+        seeds_tok = wl.tokens(cfg["n_seeds"], seed + 5)
+        hot_tok, _ = wl.with_shared_prefix(seeds_tok, cfg["hot"], cfg["prefix"], seed + 6)
+        n_rep = int(round(B * cfg["repeat_fraction"]))
+        g = torch.Generator().manual_seed(seed + 8)
+        pool = []
+        for i in range(P):
+            pick = torch.randint(0, cfg["hot"], (n_rep,), generator=g).to(dev)
+            fresh, _ = wl.with_shared_prefix(seeds_tok, B - n_rep, cfg["prefix"], seed + 100 + i)
+            tok = torch.cat([hot_tok[pick], fresh])[synth.shuffled(B, seed + 200 + i, dev)]
+            pool.append(wl.hidden(tok))
+        warm = [wl.hidden(hot_tok[i:i + B]) for i in range(0, cfg["hot"], B)]
+        warm += [wl.hidden(wl.with_shared_prefix(seeds_tok, B, cfg["prefix"], seed + 300 + i)[0])
+                 for i in range((N - cfg["hot"]) // B)]
+        return warm, pool
+    # cluster: drifting centres in hidden-state space
+    C = cfg["centres"]
+    centres = synth.randn((C, n, d), seed + 1, dev, torch.bfloat16)
+    g = torch.Generator().manual_seed(seed + 2)
+    n_near = int(round(B * cfg["near_fraction"]))
+
+    def batch(i):
+        h = torch.empty((B, n, d), dtype=torch.bfloat16, device=dev)
+        pick = torch.randint(0, C, (n_near,), generator=g).to(dev)
+        for i0 in range(0, n_near, 64):
+            sl = slice(i0, min(n_near, i0 + 64))
+            h[sl] = (centres[pick[sl]].float() + synth.randn((sl.stop - sl.start, n, d), seed + 1000 * (i + 1) + i0, dev,
+                                                             scale=cfg["noise"])).to(torch.bfloat16)
+        h[n_near:] = synth.randn((B - n_near, n, d), seed + 500000 + i, dev, torch.bfloat16)
+        return h[synth.shuffled(B, seed + 600000 + i, dev)].contiguous()
+
+    warm = [batch(-1 - i) for i in range(max(1, N // B))]
+    pool = []
+    for i in range(P):
+        for c0 in range(0, C, 64):                       # drift the centres between batches
+            centres[c0:c0 + 64] = (centres[c0:c0 + 64].float()
+                                   + synth.randn((min(64, C - c0), n, d), seed + 700000 + 10 * i + c0, dev,
+                                                 scale=cfg["drift"])).to(torch.bfloat16)
+        pool.append(batch(i))
+    return warm, pool
+
+
 # DRAM traffic per launch from an ncu capture of the named kernel on this workload, valid only while the
 # kernel's source file is unchanged (sha256 prefix of the file at capture time).
 NCU_TRAFFIC = {
@@ -55,7 +135,7 @@ def parse():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--e2e-steps", type=int, default=3)
     ap.add_argument("--no-cpu-baseline", action="store_true")
-    ap.add_argument("--workload", default="bert_base", choices=["bert_base", "scan_stress", "e2e_bert_base"])
+    ap.add_argument("--workload", default="bert_base", choices=["bert_base", "gpt2_small", "bert_large_churn", "scan_stress", "e2e_bert_base"])
     ap.add_argument("--bank", type=int, default=65536, help="scan_stress: number of bank entries")
     ap.add_argument("--queries", type=int, default=65536, help="scan_stress: queries per batch")
     ap.add_argument("--layers", type=int, default=0, help="bert_base: number of per-layer banks (default 12; fewer only for profiler captures)")
@@ -170,26 +250,22 @@ def run_ours(args):
     if world > 1:
         import torch.distributed as dist
         dist.init_process_group("nccl", device_id=dev)
+    cfg = dict(WORKLOADS[args.workload])
     if args.layers:
-        CFG["layers"] = args.layers
+        cfg["layers"] = args.layers
     if args.pool_batches:
-        CFG["pool_batches"] = args.pool_batches
-    Lyr, d, n, B, N, k = (CFG[x] for x in ("layers", "d_model", "seq_len", "batch", "bank", "fp_dim"))
+        cfg["pool_batches"] = args.pool_batches
+    Lyr, d, n, B, N, k = (cfg[x] for x in ("layers", "d_model", "seq_len", "batch", "bank", "fp_dim"))
     seed = rank_seed(rank)
-    wl = synth.TokenWorkload(CFG["vocab"], n, d, seed, dev)
-    seeds_tok = wl.tokens(CFG["n_seeds"], seed + 5)
     proj = synth.projection(d, k, seed + 6, dev)
     banks = [L.Bank(device=local, capacity=N, seq_len=n, d_model=d, fp_dim=k, max_batch=B, hidden_dtype=L.BF16,
-                    proj=proj, tau=CFG["tau"], policy=L.LRU_STALENESS) for _ in range(Lyr)]
+                    proj=proj, tau=cfg["tau"], policy=L.LRU_STALENESS) for _ in range(Lyr)]
     bufs = [L.ProbeBuffers(B, k, dev) for _ in range(Lyr)]
-    P = CFG["pool_batches"]
-    pool = build_batches(wl, seeds_tok, P, seed + 1000, dev)
+    P = cfg["pool_batches"]
+    warm, pool = make_inputs(cfg, seed, dev)
     miss_out = [synth.activations(B, n, d, seed + 50 + i, dev) for i in range(2)]
     h_out = [torch.empty((B, n * d), dtype=torch.bfloat16, device=dev) for _ in range(3)]
-    # warm every bank to capacity through the library: the seeds, then fresh sequences
-    warm = [wl.hidden(torch.cat([seeds_tok, wl.tokens(B - CFG["n_seeds"], seed + 7)]))]
-    for i in range(1, N // B):
-        warm.append(wl.hidden(wl.tokens(B, seed + 20 + i)))
+    # warm every bank to capacity through the library
     for l in range(Lyr):
         for i, hb in enumerate(warm):
             banks[l].probe(hb, bufs[l], h_out=h_out[0])
@@ -279,7 +355,7 @@ def run_ours(args):
     peaks, peak_kind = measured_peaks()
     achieved = algo_bytes[dom] / (kernels[dom]["ms_per_launch"] * 1e-3) / 1e9
     roof = {"kernel": dom, "bound": "hbm", "achieved": achieved, "peak": peaks["hbm_gbs"], "unit": "GB/s",
-            "frac": achieved / peaks["hbm_gbs"], "peak_kind": "of " + peak_kind, "traffic": ncu_traffic(dom),
+            "frac": achieved / peaks["hbm_gbs"], "peak_kind": "of " + peak_kind, "traffic": ncu_traffic(dom) if args.workload == "bert_base" else None,
             "algorithmic_bytes_per_launch": algo_bytes[dom], "all_kernels": {}}
     for name in kernels:
         ent = dict(kernels[name])
@@ -310,18 +386,16 @@ def run_ours(args):
 
     cpu = None
     if rank == 0 and world == 1 and not args.no_cpu_baseline:
-        cpu = cpu_baseline_from_gpu_state(banks, pool, proj, counter[0])
+        cpu = cpu_baseline_from_gpu_state(banks, pool, proj, counter[0], cfg)
 
     if rank == 0:
         out = {"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
                "warmup": args.warmup, "ms_per_step": ms / args.steps, "higher_is_better": True, "scaling": "weak",
                "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
-               "config": {"workload": "BERT-base-shaped encoder: 12 per-layer banks x 2048 entries (bf16 384x768), "
-                                      "batch 256 x seq_len 384, d_model 768, fp_dim 256 (projected), tau 0.90, "
-                                      "60% token-level edits of 64 seeds",
-                          "step": "probe + commit on each of 12 layers", "hit_fraction": hits / float(seqs),
-                          "l2": "inputs larger than L2: every layer of a step reads a different 151 MB batch out "
-                                "of a pool of 24, plus 1.2 GB of bank rows per layer",
+               "config": {"workload": describe(args.workload, cfg),
+                          "step": f"probe + commit on each of {Lyr} layers", "hit_fraction": hits / float(seqs),
+                          "l2": f"inputs larger than L2: every layer of a step reads a different {B * n * d * 2 / 1e6:.0f} MB "
+                                f"batch out of a pool of {P}, plus {N * n * d * 2 / 1e9:.2f} GB of bank rows per layer",
                           "parallelism": "independent replicas per GPU, no collective" if world > 1 else "single GPU"},
                "e2e": e2e, "gpu_launches": launches, "roofline": roof, "cpu_baseline": cpu, "clocks": clocks}
         print(json.dumps(out))
@@ -515,13 +589,13 @@ def blas_threads():
         return 1
 
 
-def cpu_baseline_from_gpu_state(banks, pool, proj, step, budget_s=15.0, max_layers=12, steps_per_layer=8):
+def cpu_baseline_from_gpu_state(banks, pool, proj, step, cfg, budget_s=15.0, max_layers=12, steps_per_layer=8):
     """The oracle, as it stands, on the same batches and the banks' current contents."""
     from oracle import llmcache_oracle as O
     from paper_2512_16843_b200 import binding as L
     from paper_2512_16843_b200 import synth
     from tests import parity_util as U
-    Lyr, B, P = CFG["layers"], CFG["batch"], CFG["pool_batches"]
+    Lyr, B, P = cfg["layers"], cfg["batch"], cfg["pool_batches"]
     done, t_total = 0, 0.0
     for l in range(min(Lyr, max_layers)):
         ob = U.oracle_bank_like(banks[l], proj, None)
