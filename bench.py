@@ -640,10 +640,10 @@ def run_reference(args):
         pr = O.probe(ob, synth.bf16_bits(wl.hidden(tok)), "bf16")
         O.commit(ob, pr, acts[:len(pr.miss_idx)])
     total = args.warmup + args.steps
-    batches = build_batches(wl, seeds_tok, total, seed + 1000, "cpu")
     hits = 0
     t_timed = 0.0
-    for i, hb in enumerate(batches):
+    for i in range(total):
+        hb = build_batches(wl, seeds_tok, 1, seed + 1000 + 10 * i, "cpu")[0]      # generated outside the timed part
         h = synth.bf16_bits(hb)
         t0 = time.perf_counter()
         pr = O.probe(ob, h, "bf16", h_out=h_out)
