@@ -330,3 +330,25 @@ def test_simhash_probe_matches_oracle_bit_for_bit(N, n, d, k, B):
         if step:
             assert 0 < H < B
     gb.close()
+
+
+@pytest.mark.parametrize("dtype,d,k", [("bf16", 7680, 2048), ("f32", 3840, 2048), ("bf16", 2048, 2048)])
+def test_maximum_widths(dtype, d, k):
+    """Largest d_model per input type and largest fingerprint width, with and without a projection."""
+    N, n, B = 33, 5, 9
+    proj = synth.projection(d, k, 17, DEV) if k != d else None
+    gb, ob = make_pair(N, n, d, k, B, dtype, proj, None)
+    bufs = L.ProbeBuffers(B, k, DEV)
+    base = rand_h(B, n, d, 19, dtype)
+    for step in range(3):
+        h = base.clone()
+        if step:
+            h[B // 2:] = rand_h(B - B // 2, n, d, 23 + step, dtype)
+        r = U.lockstep_step(gb, ob, bufs, h, dtype, synth.activations(B, n, d, 29 + step, DEV))
+    assert r["H"] >= B // 2
+    for bad in (7688, 8192):
+        with pytest.raises(L.LLMCacheError) as e:
+            L.Bank(capacity=4, seq_len=2, d_model=bad, fp_dim=bad if bad <= 2048 else 2048, max_batch=2,
+                   proj=synth.projection(bad, 2048, 1, DEV))
+        assert e.value.status == L.ERR_SHAPE
+    gb.close()
