@@ -363,6 +363,30 @@ def probe(bank: Bank, h, dtype: str, tau: Optional[float] = None,
     return probe_fp(bank, q, rq, tau, h_out, keep_scores)
 
 
+def probe_pooled(bank: Bank, p, tau: Optional[float] = None,
+                 h_out: Optional[np.ndarray] = None, keep_scores: bool = False) -> ProbeResult:
+    """Probe when the embedding aggregation (Sec. IV-B bullet 1) of the layer's
+    input is already at hand: p [B, d] are the position means.  A layer's input
+    is the previous layer's output, so p can be taken while that output is
+    written; the result is by definition that of probe() on the same hidden
+    states."""
+    q, rq = normalise(project(np.asarray(p, dtype=np.float64), bank.proj, bank.center))
+    return probe_fp(bank, q, rq, tau, h_out, keep_scores)
+
+
+def fingerprint_augmented(h, dtype: str, attn, attn_dtype: str, proj_bf16=None, center_f32=None):
+    """Sec. IV-B with the optional second bullet ("Prefix Attention Stats": the
+    fingerprint may also draw on the initial self-attention outputs): the
+    position mean of the first layer's self-attention output attn [B, n, d] is
+    appended to the position mean of the embeddings h [B, n, d]; the 2d-wide
+    vector is then projected (proj [2d, k], center [2d]) and normalised like any
+    other.  How the two parts are combined is not given in the paper;
+    concatenation before the projection is the reading taken here.
+    Returns (fp uint16 [B,k], rq f32 [B])."""
+    p = np.concatenate([pool(h, dtype), pool(attn, attn_dtype)], axis=1)
+    return normalise(project(p, proj_bf16, center_f32))
+
+
 # --------------------------------------------------------------------------
 # Insert on miss and eviction (Algorithm 1 "C_l[f_X] <- h_l"; Sec. III-E, IV-D)
 # --------------------------------------------------------------------------

@@ -573,3 +573,52 @@ def test_simhash_angle_estimate_is_unbiased_for_random_hyperplanes():
     ha = O.simhash_bits(O.normalise((a @ P)[None])[0]); hb = O.simhash_bits(O.normalise((b @ P)[None])[0])
     frac = float((ha != hb).mean())
     assert abs(frac - theta / math.pi) < 4 * math.sqrt(0.25 / k)
+
+
+# ------------------------------------------------ pooled probing, augmented ---
+def test_probe_pooled_equals_probe_on_the_hidden_states_and_exact_means():
+    # position means in exact rational arithmetic of the written layer output -> same decisions as probe()
+    r = rng(77)
+    B, n, d, k, N = 6, 5, 16, 64, 8
+    P = O.bf16_round((r.standard_normal((d, k)) / math.sqrt(k)).astype(np.float32))
+    h = O.bf16_round(r.standard_normal((B, n, d)).astype(np.float32))
+    bank_a = O.Bank(capacity=N, seq_len=n, d_model=d, fp_dim=k, proj=P, tau=0.5)
+    bank_b = O.Bank(capacity=N, seq_len=n, d_model=d, fp_dim=k, proj=P, tau=0.5)
+    for bk in (bank_a, bank_b):
+        pr = O.probe(bk, h[:4], "bf16")
+        O.commit(bk, pr, h[:4].reshape(4, -1))
+    vals = O.bf16_to_f32(h)
+    means = np.array([[float(sum(Fraction(float(vals[b, t, i])) for t in range(n)) / n) for i in range(d)]
+                      for b in range(B)])
+    pa = O.probe(bank_a, h, "bf16")
+    pb = O.probe_pooled(bank_b, means)
+    assert np.array_equal(pa.fp, pb.fp) and np.array_equal(pa.hit, pb.hit) and np.array_equal(pa.slot, pb.slot)
+    assert pa.hit[:4].all() and not pa.hit[4:].any()
+    assert np.array_equal(pa.score, pb.score)
+
+
+def test_fingerprint_augmented_block_structure():
+    # a block-diagonal projection separates the two parts: each block equals the plain projection of its part
+    r = rng(78)
+    B, n, d, k = 4, 7, 8, 64
+    h = r.standard_normal((B, n, d)).astype(np.float32)
+    a = O.bf16_round(r.standard_normal((B, n, d)).astype(np.float32))
+    P1 = O.bf16_round(r.standard_normal((d, k // 2)).astype(np.float32))
+    P2 = O.bf16_round(r.standard_normal((d, k // 2)).astype(np.float32))
+    Pfull = np.zeros((2 * d, k), dtype=np.uint16)
+    Pfull[:d, :k // 2] = P1
+    Pfull[d:, k // 2:] = P2
+    fp, rq = O.fingerprint_augmented(h, "f32", a, "bf16", Pfull, None)
+    g1 = h.astype(np.float64).mean(axis=1) @ O.bf16_to_f32(P1).astype(np.float64)
+    g2 = O.bf16_to_f32(a).astype(np.float64).mean(axis=1) @ O.bf16_to_f32(P2).astype(np.float64)
+    g = np.concatenate([g1, g2], axis=1)
+    want = g / np.linalg.norm(g, axis=1, keepdims=True)
+    got = O.bf16_to_f32(fp).astype(np.float64)
+    assert np.max(np.abs(got - want)) <= 2.0 ** -8          # one bf16 rounding of values below 1
+    # zeroing the attention part reduces it to the plain fingerprint with the first block
+    fp0, _ = O.fingerprint_augmented(h, "f32", np.zeros_like(a), "bf16", Pfull, None)
+    fpp, _ = O.fingerprint(h, "f32", np.ascontiguousarray(Pfull[:d]), None)
+    assert np.array_equal(fp0, fpp)
+    # swapping the two inputs is not the same fingerprint (the order of the parts matters)
+    fps, _ = O.fingerprint_augmented(O.bf16_to_f32(a), "f32", O.bf16_round(h), "bf16", Pfull, None)
+    assert not np.array_equal(fps, fp)
