@@ -41,7 +41,7 @@
 extern "C" {
 #endif
 
-#define LLMCACHE_ABI_VERSION 1u
+#define LLMCACHE_ABI_VERSION 2u
 
 typedef struct llmcache_bank llmcache_bank_t;
 
@@ -94,6 +94,7 @@ typedef struct llmcache_bank_desc {
   uint32_t min_age_ticks;     /* ... and at least this old                              (0 => 4) */
   uint32_t max_idle_ticks;    /* LLMCACHE_EVICT_IDLE drops entries unused for longer    (0 => 32) */
   uint32_t store_act;         /* 1 = keep layer outputs (normal); 0 = keys only (scan benchmarks) */
+  uint32_t fused_pool;        /* 1 = reserve the scratch llmcache_bank_pool_out needs (bf16 outputs, store_act) */
   const void*  proj;          /* device, bf16 [d,k] row-major projection (Sec. IV-B "Dimensionality
                                  Reduction"), copied at create; NULL => identity (k == d) */
   const float* center;        /* device, f32 [d] subtracted before projection, copied; NULL => 0 */
@@ -136,7 +137,9 @@ enum {
   LLMCACHE_K_SELECT = 7,    /* Sec. IV-D victim selection (side stream, during GATHER) */
   LLMCACHE_K_SCATTER = 8,   /* Algorithm 1 insert: write-back + store              */
   LLMCACHE_K_EVICT = 9,     /* Sec. III-E flushes                                  */
-  LLMCACHE_K_COUNT = 10
+  LLMCACHE_K_INSERT = 10,   /* keys + metadata of new entries (when the rows move in a pooling pass) */
+  LLMCACHE_K_POOL_FINISH = 11, /* partial column sums -> position means               */
+  LLMCACHE_K_COUNT = 12
 };
 
 uint32_t    llmcache_abi_version(void);
@@ -158,6 +161,20 @@ int llmcache_bank_destroy(llmcache_bank_t* bank);
  * h_in: device [B,n,d] of the bank's hidden_dtype.  fp: device bf16 [B,k].  rq: device f32 [B]. */
 int llmcache_fingerprint(llmcache_bank_t* bank, const void* h_in, uint32_t B,
                          void* fp, float* rq, void* stream);
+
+/* The two halves of llmcache_fingerprint, for callers that have the position means from elsewhere, or
+ * that build the fingerprint from more than one tensor (Sec. IV-B lists, besides the aggregated
+ * embeddings, optional "Prefix Attention Stats" taken from the first self-attention outputs: pool both
+ * tensors into the two halves of one [B, 2d] array and fingerprint that with a bank whose d_model is 2d).
+ *   llmcache_pool: pooled[b * ld + c] = mean over the n positions of h_in[b, :, c], c < d_model (step
+ *     "Embedding Aggregation").  h_in: device [B,n,d] of the bank's hidden_dtype; pooled: device f32,
+ *     ld >= d_model floats between sequences (a column offset is applied by the caller to `pooled`).
+ *   llmcache_fingerprint_pooled: fp[b] = unit-length bf16 of (pooled[b, :d_model] - center) . proj (step
+ *     "Dimensionality Reduction"); same result as llmcache_fingerprint when pooled holds the means of h_in
+ *     (up to the order of the fp32 sums).  seq_len of the bank plays no part. */
+int llmcache_pool(llmcache_bank_t* bank, const void* h_in, uint32_t B, float* pooled, uint32_t ld, void* stream);
+int llmcache_fingerprint_pooled(llmcache_bank_t* bank, const float* pooled, uint32_t ld, uint32_t B,
+                                void* fp, float* rq, void* stream);
 
 /* Fingerprint for callers that must not allocate device memory.  (The paper has no counterpart:
  * this is a packaging variant of llmcache_fingerprint, same kernels, same result.)
@@ -215,6 +232,22 @@ int llmcache_probe_simhash(llmcache_bank_t* bank, const void* h_in, uint32_t B, 
  * h_in may be NULL (then io->h_miss is not produced). */
 int llmcache_probe_fp(llmcache_bank_t* bank, const void* h_in, uint32_t B, float tau,
                       void* h_out, llmcache_probe_io* io, void* stream);
+
+/* llmcache_probe when the position means of h_in are already known (see llmcache_bank_pool_out):
+ * pooled: device f32, pooled[b * ld + c] = mean_t h_in[b,t,c].  h_in is only needed for io->h_miss and
+ * may be NULL otherwise.  Everything else as llmcache_probe. */
+int llmcache_probe_pooled(llmcache_bank_t* bank, const float* pooled, uint32_t ld, const void* h_in, uint32_t B,
+                          float tau, void* h_out, llmcache_probe_io* io, void* stream);
+
+/* Fingerprint-on-write.  Algorithm 1 feeds layer l+1 with the output of layer l, and the fingerprint of
+ * that input starts with its mean over the positions (Sec. IV-B).  With pooled_out set, the passes
+ * that write the rows of h_out -- the copy of reused outputs in llmcache_probe*, the write-back in
+ * llmcache_commit -- also sum what they move, and after the commit
+ *     pooled_out[b * ld + c] = mean_t h_out[b,t,c]      (device f32, every b < B of the probe)
+ * ready for llmcache_probe_pooled on the next layer's bank, which then does not read h_out at all.
+ * Needs a bank created with fused_pool = 1 and store_act = 1; every probe must then pass h_out, and
+ * every commit miss_out.  pooled_out == NULL switches it off.  ld >= d_model. */
+int llmcache_bank_pool_out(llmcache_bank_t* bank, float* pooled_out, uint32_t ld);
 
 /* After the layer ran on the misses (Algorithm 1 else-branch, "C_l[f_X] <- h_l";
  * victim choice per Sec. III-E / IV-D).  miss_out: device bf16 [M,n,d] in the
@@ -308,6 +341,13 @@ int llmcache_layer_status(llmcache_layer_t* layer);
 int llmcache_infer(llmcache_bank_t** banks, llmcache_layer_t** layers, uint32_t n_layers, const void* h0, uint32_t B,
                    float tau, void* buf_a, void* buf_b, void* h_miss, void* miss_out, llmcache_probe_io* io,
                    void** h_final, void* stream);
+/* The same loop with fingerprint-on-write: only layer 1 pools its input; every later probe takes the
+ * position means that the previous layer's row movers produced (llmcache_bank_pool_out /
+ * llmcache_probe_pooled).  pooled: device f32 [B, d] scratch.  The banks must have fused_pool = 1; their
+ * pool_out setting is overwritten and left switched off. */
+int llmcache_infer_pooled(llmcache_bank_t** banks, llmcache_layer_t** layers, uint32_t n_layers, const void* h0,
+                          uint32_t B, float tau, void* buf_a, void* buf_b, void* h_miss, void* miss_out,
+                          llmcache_probe_io* io, float* pooled, void** h_final, void* stream);
 
 /* Divergence monitor (Sec. III-E: "tracking differences in successive outputs for a given fingerprint";
  * Sec. IV-D: "revalidates fingerprints").  Call after the commit of a probe, with that probe's h_in and io.

@@ -34,9 +34,12 @@ EXPORTS = [
     "llmcache_fingerprint_static", "llmcache_fingerprint_static_error",
     "llmcache_layer_bytes", "llmcache_layer_create", "llmcache_layer_destroy", "llmcache_layer_forward",
     "llmcache_layer_status", "llmcache_infer", "llmcache_divergence_check", "llmcache_probe_simhash",
+    "llmcache_pool", "llmcache_fingerprint_pooled", "llmcache_probe_pooled", "llmcache_bank_pool_out",
+    "llmcache_infer_pooled",
 ]
 FINGERPRINT_STATIC_MAX_FLOATS = 2 * 1024 * 1024
-KERNEL_NAMES = ["pool", "project", "rownorm", "scan", "decide", "touch", "gather", "select", "scatter", "evict"]
+KERNEL_NAMES = ["pool", "project", "rownorm", "scan", "decide", "touch", "gather", "select", "scatter", "evict",
+                "insert", "pool_finish"]
 
 
 class BankDesc(C.Structure):
@@ -47,6 +50,7 @@ class BankDesc(C.Structure):
         ("tau", C.c_float), ("cmp", C.c_uint32), ("policy", C.c_uint32),
         ("half_life_ticks", C.c_uint32), ("stale_floor_q8", C.c_uint32),
         ("min_age_ticks", C.c_uint32), ("max_idle_ticks", C.c_uint32), ("store_act", C.c_uint32),
+        ("fused_pool", C.c_uint32),
         ("proj", C.c_void_p), ("center", C.c_void_p), ("arena", C.c_void_p), ("arena_bytes", C.c_size_t),
     ]
 
@@ -127,6 +131,12 @@ def lib():
         L.llmcache_infer.argtypes = [C.POINTER(vp), C.POINTER(vp), u32, vp, u32, C.c_float, vp, vp, vp, vp,
                                      C.POINTER(ProbeIO), C.POINTER(vp), vp]
         L.llmcache_divergence_check.argtypes = [vp, vp, vp, C.POINTER(ProbeIO), u32, C.c_float, vp, vp, vp, vp, vp]
+        L.llmcache_pool.argtypes = [vp, vp, u32, vp, u32, vp]
+        L.llmcache_fingerprint_pooled.argtypes = [vp, vp, u32, u32, vp, vp, vp]
+        L.llmcache_probe_pooled.argtypes = [vp, vp, u32, vp, u32, C.c_float, vp, C.POINTER(ProbeIO), vp]
+        L.llmcache_bank_pool_out.argtypes = [vp, vp, u32]
+        L.llmcache_infer_pooled.argtypes = [C.POINTER(vp), C.POINTER(vp), u32, vp, u32, C.c_float, vp, vp, vp, vp,
+                                            C.POINTER(ProbeIO), vp, C.POINTER(vp), vp]
         L.llmcache_fingerprint_static.argtypes = [vp, u32, u32, u32, u32, u32, vp, vp, vp, vp, vp]
         L.llmcache_fingerprint_static_error.restype = C.c_char_p
         L.llmcache_fingerprint_static_error.argtypes = []
@@ -172,7 +182,7 @@ def llmcache_abi_version() -> int:
 
 def make_desc(*, device=0, capacity, seq_len, d_model, fp_dim, hidden_dtype=BF16, act_rows=0, max_batch,
               tau=0.9, cmp=GT, policy=LRU_STALENESS, half_life_ticks=0, stale_floor_q8=0, min_age_ticks=0,
-              max_idle_ticks=0, store_act=1, proj=None, center=None, arena=None, arena_bytes=0) -> BankDesc:
+              max_idle_ticks=0, store_act=1, fused_pool=0, proj=None, center=None, arena=None, arena_bytes=0) -> BankDesc:
     d = BankDesc()
     d.struct_size = C.sizeof(BankDesc)
     d.device, d.capacity, d.seq_len, d.d_model, d.fp_dim = device, capacity, seq_len, d_model, fp_dim
@@ -180,6 +190,7 @@ def make_desc(*, device=0, capacity, seq_len, d_model, fp_dim, hidden_dtype=BF16
     d.tau, d.cmp, d.policy = tau, cmp, policy
     d.half_life_ticks, d.stale_floor_q8 = half_life_ticks, stale_floor_q8
     d.min_age_ticks, d.max_idle_ticks, d.store_act = min_age_ticks, max_idle_ticks, store_act
+    d.fused_pool = fused_pool
     d.proj, d.center, d.arena, d.arena_bytes = _ptr(proj), _ptr(center), _ptr(arena), arena_bytes
     return d
 
@@ -234,6 +245,25 @@ def llmcache_probe_fp(bank, h_in, B, tau, h_out, io: ProbeIO, stream=None) -> No
     tau = float("nan") if tau is None else tau
     _check(lib().llmcache_probe_fp(bank, _ptr(h_in), B, tau, _ptr(h_out), C.byref(io), _stream(stream)),
            "llmcache_probe_fp")
+
+
+def llmcache_pool(bank, h_in, B, pooled, ld, stream=None) -> None:
+    _check(lib().llmcache_pool(bank, _ptr(h_in), B, _ptr(pooled), ld, _stream(stream)), "llmcache_pool")
+
+
+def llmcache_fingerprint_pooled(bank, pooled, ld, B, fp, rq, stream=None) -> None:
+    _check(lib().llmcache_fingerprint_pooled(bank, _ptr(pooled), ld, B, _ptr(fp), _ptr(rq), _stream(stream)),
+           "llmcache_fingerprint_pooled")
+
+
+def llmcache_probe_pooled(bank, pooled, ld, h_in, B, tau, h_out, io: ProbeIO, stream=None) -> None:
+    tau = float("nan") if tau is None else tau
+    _check(lib().llmcache_probe_pooled(bank, _ptr(pooled), ld, _ptr(h_in), B, tau, _ptr(h_out), C.byref(io),
+                                       _stream(stream)), "llmcache_probe_pooled")
+
+
+def llmcache_bank_pool_out(bank, pooled_out, ld) -> None:
+    _check(lib().llmcache_bank_pool_out(bank, _ptr(pooled_out), ld), "llmcache_bank_pool_out")
 
 
 def llmcache_commit(bank, miss_out, io: ProbeIO, h_out, new_slot, stream=None) -> None:
@@ -366,6 +396,22 @@ class Bank:
         B = h_in.shape[0] if B is None else B
         llmcache_probe(self.handle, h_in, B, tau, h_out, bufs.io, stream)
 
+    def probe_pooled(self, pooled, bufs: ProbeBuffers, B, h_out=None, tau=None, h_in=None, stream=None):
+        llmcache_probe_pooled(self.handle, pooled, pooled.stride(0), h_in, B, tau, h_out, bufs.io, stream)
+
+    def pool_out(self, pooled_out):
+        """Position means of the rows written by the next probes + commits go to pooled_out [B, >=d] f32
+        (None switches it off)."""
+        llmcache_bank_pool_out(self.handle, pooled_out, 0 if pooled_out is None else pooled_out.stride(0))
+        self._pool_out = pooled_out
+
+    def pool(self, h_in, pooled, B=None, stream=None):
+        llmcache_pool(self.handle, h_in, h_in.shape[0] if B is None else B, pooled, pooled.stride(0), stream)
+
+    def fingerprint_pooled(self, pooled, fp, rq, B=None, stream=None):
+        llmcache_fingerprint_pooled(self.handle, pooled, pooled.stride(0), pooled.shape[0] if B is None else B,
+                                    fp, rq, stream)
+
     def probe_fp(self, bufs: ProbeBuffers, B, h_out=None, tau=None, h_in=None, stream=None):
         llmcache_probe_fp(self.handle, h_in, B, tau, h_out, bufs.io, stream)
 
@@ -428,6 +474,19 @@ def llmcache_infer(banks, layers, h0, B, tau, buf_a, buf_b, h_miss, miss_out, io
     _check(lib().llmcache_infer(barr, larr, n, _ptr(h0), B, tau, _ptr(buf_a), _ptr(buf_b), _ptr(h_miss),
                                 _ptr(miss_out), C.byref(io) if io is not None else None, C.byref(final),
                                 _stream(stream)), "llmcache_infer")
+    return final.value
+
+
+def llmcache_infer_pooled(banks, layers, h0, B, tau, buf_a, buf_b, h_miss, miss_out, io, pooled, stream=None) -> int:
+    """Algorithm 1 with fingerprint-on-write; returns the device address that will hold h_L."""
+    n = len(layers)
+    larr = (C.c_void_p * n)(*layers)
+    barr = (C.c_void_p * n)(*banks)
+    final = C.c_void_p(None)
+    tau = float("nan") if tau is None else tau
+    _check(lib().llmcache_infer_pooled(barr, larr, n, _ptr(h0), B, tau, _ptr(buf_a), _ptr(buf_b), _ptr(h_miss),
+                                       _ptr(miss_out), C.byref(io), _ptr(pooled), C.byref(final), _stream(stream)),
+           "llmcache_infer_pooled")
     return final.value
 
 

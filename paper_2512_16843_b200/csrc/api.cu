@@ -17,7 +17,7 @@ inline uint32_t pow2_ceil(uint32_t x) { uint32_t p = 1; while (p < x) p <<= 1; r
 
 struct Layout {
   size_t fp, rb, valid, last_use, insert_tick, hits, rate, rate_epoch, act, proj, center;
-  size_t pool_partial, best, hitcnt, victims, new_slot, bits, qbits, sort_key, sort_slot, stats, status, misc, total;
+  size_t pool_partial, move_partial, best, hitcnt, victims, new_slot, bits, qbits, sort_key, sort_slot, stats, status, misc, total;
   uint32_t sort_len;
 };
 
@@ -45,6 +45,7 @@ int check_desc(const llmcache_bank_desc* d) {
   if (!d->proj && d->fp_dim != d->d_model) return LLMCACHE_ERR_SHAPE;
   if (d->capacity > (1u << 30) || d->max_batch > (1u << 24)) return LLMCACHE_ERR_SHAPE;
   if (d->act_rows > d->capacity) return LLMCACHE_ERR_SHAPE;
+  if (d->fused_pool > 1 || (d->fused_pool && !d->store_act)) return LLMCACHE_ERR_ARG;
   if (!(d->tau == d->tau)) return LLMCACHE_ERR_ARG;
   if (project_smem_bytes(d->d_model, d->fp_dim, d->proj != nullptr) > 200 * 1024) return LLMCACHE_ERR_UNSUPPORTED;
   if (d->arena && ((uintptr_t)d->arena % ALIGN) != 0) return LLMCACHE_ERR_ARG;
@@ -71,6 +72,7 @@ Layout make_layout(const llmcache_bank_desc& d) {
   L.center = take(d.center ? dm * 4 : 0);
   // scratch: one vector of partial sums per (pool block, sequence it touches)
   L.pool_partial = take(((size_t)d.max_batch + 3 * POOL_MAX_GRID) * dm * 4);
+  L.move_partial = take(d.fused_pool ? 2 * move_partial_floats(d.max_batch, d.d_model) * 4 : 0);
   L.best = take((size_t)d.max_batch * 8);
   L.hitcnt = take(N * 4);
   const uint32_t vmax = d.max_batch < d.capacity ? d.max_batch : d.capacity;
@@ -209,6 +211,7 @@ int llmcache_bank_create(const llmcache_bank_desc* desc, llmcache_bank_t** bank_
   a.proj = desc->proj ? (__nv_bfloat16*)(base + L.proj) : nullptr;
   a.center = desc->center ? (float*)(base + L.center) : nullptr;
   a.pool_partial = (float*)(base + L.pool_partial);
+  a.move_partial = desc->fused_pool ? (float*)(base + L.move_partial) : nullptr;
   a.best = (unsigned long long*)(base + L.best);
   a.hitcnt = (uint32_t*)(base + L.hitcnt);
   a.victims = (int32_t*)(base + L.victims);
@@ -231,6 +234,7 @@ int llmcache_bank_create(const llmcache_bank_desc* desc, llmcache_bank_t** bank_
   if (e == cudaSuccess) e = setup_fingerprint_kernels();
   if (e == cudaSuccess) e = setup_scan_kernels();
   if (e == cudaSuccess) e = setup_rows_kernels();
+  if (e == cudaSuccess) e = setup_move_kernels();
   if (e == cudaSuccess) e = cudaStreamCreateWithFlags(&bk->side, cudaStreamNonBlocking);
   if (e == cudaSuccess) e = cudaEventCreateWithFlags(&bk->ev_fork, cudaEventDisableTiming);
   if (e == cudaSuccess) e = cudaEventCreateWithFlags(&bk->ev_join, cudaEventDisableTiming);
@@ -273,6 +277,39 @@ int llmcache_fingerprint(llmcache_bank_t* bk, const void* h_in, uint32_t B, void
   return e == cudaSuccess ? LLMCACHE_OK : cuda_fail(e, __func__);
 }
 
+int llmcache_pool(llmcache_bank_t* bk, const void* h_in, uint32_t B, float* pooled, uint32_t ld, void* stream) {
+  if (!bk || (B && (!h_in || !pooled))) return LLMCACHE_ERR_ARG;
+  if (B > bk->desc.max_batch || ld < bk->desc.d_model) return LLMCACHE_ERR_SHAPE;
+  if (!aligned16(h_in) || ((uintptr_t)pooled & 3u)) return LLMCACHE_ERR_ARG;
+  DeviceGuard guard(bk->desc.device);
+  if (!guard.ok) return LLMCACHE_ERR_CUDA;
+  cudaError_t e = launch_pool_only(bk, h_in, B, pooled, ld, (cudaStream_t)stream);
+  return e == cudaSuccess ? LLMCACHE_OK : cuda_fail(e, __func__);
+}
+
+int llmcache_fingerprint_pooled(llmcache_bank_t* bk, const float* pooled, uint32_t ld, uint32_t B,
+                                void* fp, float* rq, void* stream) {
+  if (!bk || (B && (!pooled || !fp || !rq))) return LLMCACHE_ERR_ARG;
+  if (B > bk->desc.max_batch || ld < bk->desc.d_model) return LLMCACHE_ERR_SHAPE;
+  if (!aligned16(fp) || ((uintptr_t)pooled & 3u)) return LLMCACHE_ERR_ARG;
+  DeviceGuard guard(bk->desc.device);
+  if (!guard.ok) return LLMCACHE_ERR_CUDA;
+  cudaError_t e = launch_fingerprint_pooled(bk, pooled, ld, B, (__nv_bfloat16*)fp, rq, (cudaStream_t)stream);
+  return e == cudaSuccess ? LLMCACHE_OK : cuda_fail(e, __func__);
+}
+
+int llmcache_bank_pool_out(llmcache_bank_t* bk, float* pooled_out, uint32_t ld) {
+  if (!bk) return LLMCACHE_ERR_ARG;
+  if (bk->probe_open && bk->last_B) return LLMCACHE_ERR_STATE;      // not between a probe and its commit
+  if (!pooled_out) { bk->pool_out = nullptr; bk->pool_out_ld = 0; return LLMCACHE_OK; }
+  if (!bk->a.move_partial || !bk->a.act) return LLMCACHE_ERR_UNSUPPORTED;
+  if (ld < bk->desc.d_model) return LLMCACHE_ERR_SHAPE;
+  if ((uintptr_t)pooled_out & 3u) return LLMCACHE_ERR_ARG;
+  bk->pool_out = pooled_out;
+  bk->pool_out_ld = ld;
+  return LLMCACHE_OK;
+}
+
 // Largest Hamming distance that still matches: the SimHash angle estimate is pi * ham / k and a match
 // needs cos(angle) > tau, i.e. ham < k * acos(tau) / pi.
 static int32_t hamming_threshold(float tau, uint32_t k) {
@@ -287,13 +324,16 @@ static int32_t hamming_threshold(float tau, uint32_t k) {
 }
 
 static int probe_common(llmcache_bank_t* bk, const void* h_in, bool compute_fp, uint32_t B, float tau,
-                        void* h_out, llmcache_probe_io* io, void* stream, bool simhash = false) {
+                        void* h_out, llmcache_probe_io* io, void* stream, bool simhash = false,
+                        const float* pooled = nullptr, uint32_t pooled_ld = 0) {
   if (!bk) return LLMCACHE_ERR_ARG;
   if (B > bk->desc.max_batch) return LLMCACHE_ERR_SHAPE;
   if (B) {
     int rc = check_io(io);
     if (rc != LLMCACHE_OK) return rc;
-    if (compute_fp && !h_in) return LLMCACHE_ERR_ARG;
+    if (compute_fp && !h_in && !pooled) return LLMCACHE_ERR_ARG;
+    if (pooled && (pooled_ld < bk->desc.d_model || ((uintptr_t)pooled & 3u))) return LLMCACHE_ERR_SHAPE;
+    if (bk->pool_out && !h_out) return LLMCACHE_ERR_ARG;             // every row of h_out must pass through
     if (!aligned16(h_in) || !aligned16(h_out)) return LLMCACHE_ERR_ARG;
   } else if (!io) {
     return LLMCACHE_ERR_ARG;
@@ -318,8 +358,9 @@ static int probe_common(llmcache_bank_t* bk, const void* h_in, bool compute_fp, 
   if (B == 0) {
     if (io->counts) e = cudaMemsetAsync(io->counts, 0, 2 * sizeof(uint32_t), st);
   } else {
-    if (compute_fp) e = launch_fingerprint(bk, h_in, B, (__nv_bfloat16*)io->fp, io->rq, st);
-    else            e = launch_rownorm(bk, (const __nv_bfloat16*)io->fp, B, bk->desc.fp_dim, io->rq, st);
+    if (pooled)          e = launch_fingerprint_pooled(bk, pooled, pooled_ld, B, (__nv_bfloat16*)io->fp, io->rq, st);
+    else if (compute_fp) e = launch_fingerprint(bk, h_in, B, (__nv_bfloat16*)io->fp, io->rq, st);
+    else                 e = launch_rownorm(bk, (const __nv_bfloat16*)io->fp, B, bk->desc.fp_dim, io->rq, st);
     if (simhash) {
       if (e == cudaSuccess) e = launch_simhash_scan(bk, (const __nv_bfloat16*)io->fp, B, st);
       if (e == cudaSuccess) e = launch_decide(bk, B, tau, io->rq, io, st, bk->desc.fp_dim, hamming_threshold(tau, bk->desc.fp_dim));
@@ -339,7 +380,15 @@ static int probe_common(llmcache_bank_t* bk, const void* h_in, bool compute_fp, 
       if (e == cudaSuccess) e = cudaEventRecord(bk->ev_join, bk->side);
       if (e == cudaSuccess) bk->join_pending = true;
     }
-    if (e == cudaSuccess) e = launch_gather(bk, h_in, h_out, io, B, st);
+    bk->moved[0] = bk->moved[1] = false;
+    if (bk->pool_out) {
+      // the reused rows are summed while they are copied; the miss inputs (if wanted) go the plain way
+      if (e == cudaSuccess) e = launch_move_pool(bk, 0, nullptr, h_out, io, B, st);
+      if (e == cudaSuccess) bk->moved[0] = true;
+      if (e == cudaSuccess && h_in && io->h_miss) e = launch_gather(bk, h_in, nullptr, io, B, st);
+    } else {
+      if (e == cudaSuccess) e = launch_gather(bk, h_in, h_out, io, B, st);
+    }
   }
   if (e == cudaSuccess && io->counts_host && io->counts)
     e = cudaMemcpyAsync(io->counts_host, io->counts, 2 * sizeof(uint32_t), cudaMemcpyDeviceToHost, st);
@@ -362,6 +411,12 @@ int llmcache_probe_fp(llmcache_bank_t* bk, const void* h_in, uint32_t B, float t
   return probe_common(bk, h_in, false, B, tau, h_out, io, stream);
 }
 
+int llmcache_probe_pooled(llmcache_bank_t* bk, const float* pooled, uint32_t ld, const void* h_in, uint32_t B,
+                          float tau, void* h_out, llmcache_probe_io* io, void* stream) {
+  if (B && !pooled) return LLMCACHE_ERR_ARG;
+  return probe_common(bk, h_in, true, B, tau, h_out, io, stream, false, pooled, ld);
+}
+
 int llmcache_commit(llmcache_bank_t* bk, const void* miss_out, const llmcache_probe_io* io, void* h_out,
                     int32_t* new_slot, void* stream) {
   if (!bk || !io) return LLMCACHE_ERR_ARG;
@@ -373,6 +428,7 @@ int llmcache_commit(llmcache_bank_t* bk, const void* miss_out, const llmcache_pr
     if (rc != LLMCACHE_OK) return rc;
     if (!aligned16(miss_out) || !aligned16(h_out)) return LLMCACHE_ERR_ARG;
     if (bk->a.act && !miss_out) return LLMCACHE_ERR_ARG;
+    if (bk->pool_out && !miss_out) return LLMCACHE_ERR_ARG;
   }
   DeviceGuard guard(bk->desc.device);
   if (!guard.ok) return LLMCACHE_ERR_CUDA;
@@ -388,7 +444,15 @@ int llmcache_commit(llmcache_bank_t* bk, const void* miss_out, const llmcache_pr
   bk->bits_dirty = true;
   if (e == cudaSuccess && bk->select_deferred) e = launch_select_victims(bk, io, B, st);
   bk->select_deferred = false;
-  if (e == cudaSuccess) e = launch_scatter_insert(bk, miss_out, io, h_out, new_slot, B, st);
+  if (bk->pool_out && bk->moved[0]) {
+    // keys and metadata of the new entries, then the rows (summed while they move), then the means
+    if (e == cudaSuccess) e = launch_scatter_insert(bk, nullptr, io, nullptr, new_slot, B, st);
+    if (e == cudaSuccess) e = launch_move_pool(bk, 1, miss_out, h_out, io, B, st);
+    if (e == cudaSuccess) e = launch_pool_finish_moved(bk, io, B, bk->pool_out, bk->pool_out_ld, st);
+    bk->moved[0] = bk->moved[1] = false;
+  } else {
+    if (e == cudaSuccess) e = launch_scatter_insert(bk, miss_out, io, h_out, new_slot, B, st);
+  }
   if (e != cudaSuccess) return cuda_fail(e, __func__);
   return LLMCACHE_OK;
 }

@@ -175,7 +175,8 @@ __device__ __forceinline__ float group_sum(float v, float* red, int group) {
 __global__ void __launch_bounds__(PROJ_THREADS)
 k_project(const float* __restrict__ partial, const __nv_bfloat16* __restrict__ proj,
           const float* __restrict__ center, __nv_bfloat16* __restrict__ fp, float* __restrict__ rq,
-          uint32_t B, uint32_t n, uint32_t d, uint32_t k, uint32_t L, uint32_t Jmax) {
+          uint32_t B, uint32_t n, uint32_t d, uint32_t k, uint32_t L, uint32_t Jmax,
+          const float* __restrict__ pooled, uint32_t ld) {
   griddep_sync();
   extern __shared__ float sm[];
   float* p = sm;                               // [G][d]
@@ -191,7 +192,14 @@ k_project(const float* __restrict__ partial, const __nv_bfloat16* __restrict__ p
   {
     // pool blocks whose span overlaps rows [b*n, (b+1)*n), in block order
     float* pg = p + (size_t)grp * d;
-    if (bq < B) {
+    if (bq < B && pooled) {
+      // the position means were taken elsewhere (while the rows were written)
+      for (uint32_t i = gt; i < d; i += PROJ_TPS) {
+        float v = pooled[(size_t)bq * ld + i];
+        if (center) v -= center[i];
+        pg[i] = v;
+      }
+    } else if (bq < B) {
       const unsigned long long first = (unsigned long long)bq * n, last = first + n - 1;
       const uint32_t c_lo = (uint32_t)(first / L), c_hi = (uint32_t)(last / L);
       const uint32_t j_lo = bq - (uint32_t)(((unsigned long long)c_lo * L) / n);
@@ -369,7 +377,8 @@ static cudaError_t launch_project(const PoolPlan& P, const float* partial, const
                                   const float* center, __nv_bfloat16* fp, float* rq,
                                   uint32_t B, uint32_t n, uint32_t d, uint32_t k, cudaStream_t st) {
   return launch_k(k_project, dim3((B + PROJ_G - 1) / PROJ_G), dim3(PROJ_THREADS),
-                  project_smem_bytes(d, k, proj != nullptr), st, partial, proj, center, fp, rq, B, n, d, k, P.L, P.Jmax);
+                  project_smem_bytes(d, k, proj != nullptr), st, partial, proj, center, fp, rq, B, n, d, k, P.L, P.Jmax,
+                  (const float*)nullptr, 0u);
 }
 
 cudaError_t launch_fingerprint(llmcache_bank* bk, const void* h_in, uint32_t B,
@@ -386,6 +395,33 @@ cudaError_t launch_fingerprint(llmcache_bank* bk, const void* h_in, uint32_t B,
   if (e != cudaSuccess) return e;
   ProfScope prof(bk, LLMCACHE_K_PROJECT, st);
   return launch_project(P, bk->a.pool_partial, bk->a.proj, bk->a.center, fp, rq, B, D.seq_len, D.d_model, D.fp_dim, st);
+}
+
+// Step 1a alone: position means of h_in -> pooled[b * ld + c].
+cudaError_t launch_pool_only(llmcache_bank* bk, const void* h_in, uint32_t B, float* pooled, uint32_t ld, cudaStream_t st) {
+  if (B == 0) return cudaSuccess;
+  const llmcache_bank_desc& D = bk->desc;
+  const bool bf16 = D.hidden_dtype == LLMCACHE_BF16;
+  const PoolPlan P = pool_plan(B, D.seq_len, D.d_model, bf16, bk->sm_count);
+  cudaError_t e;
+  {
+    ProfScope prof(bk, LLMCACHE_K_POOL, st);
+    e = launch_pool(P, bf16, h_in, bk->a.pool_partial, bk->a.status, B, D.seq_len, D.d_model, st);
+  }
+  if (e != cudaSuccess) return e;
+  return launch_pool_finish_plain(bk, P, B, pooled, ld, st);
+}
+
+// Step 1b alone: fingerprints from given position means pooled[b * ld + c], c < d.
+cudaError_t launch_fingerprint_pooled(llmcache_bank* bk, const float* pooled, uint32_t ld, uint32_t B,
+                                      __nv_bfloat16* fp, float* rq, cudaStream_t st) {
+  if (B == 0) return cudaSuccess;
+  const llmcache_bank_desc& D = bk->desc;
+  ProfScope prof(bk, LLMCACHE_K_PROJECT, st);
+  return launch_k(k_project, dim3((B + PROJ_G - 1) / PROJ_G), dim3(PROJ_THREADS),
+                  project_smem_bytes(D.d_model, D.fp_dim, bk->a.proj != nullptr), st, (const float*)nullptr,
+                  (const __nv_bfloat16*)bk->a.proj, (const float*)bk->a.center, fp, rq, B, D.seq_len, D.d_model,
+                  D.fp_dim, 1u, 1u, pooled, ld);
 }
 
 cudaError_t launch_rownorm(llmcache_bank* bk, const __nv_bfloat16* fp, uint32_t B, uint32_t k, float* rq, cudaStream_t st) {

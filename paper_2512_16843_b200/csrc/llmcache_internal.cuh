@@ -13,6 +13,8 @@ namespace llmc {
 constexpr uint32_t M_CAP = (1u << 30) - 1u;   // ceiling of the decayed match rate (Q8)
 constexpr uint32_t HIT_Q8 = 256u;             // one match in Q8
 constexpr uint32_t POOL_MAX_GRID = 640;       // most blocks the pooling pass ever launches
+// floats of one set of partial sums of a pooling (or moving) pass
+inline size_t move_partial_floats(uint32_t max_batch, uint32_t d) { return ((size_t)max_batch + 3 * POOL_MAX_GRID) * d; }
 
 // Counters kept on the device (index into Bank::d_stats).
 enum { ST_SEQ = 0, ST_HIT, ST_MISS, ST_DEGEN, ST_INSERT, ST_EVICT, ST_DROP, ST_FLUSH, ST_COUNT };
@@ -36,6 +38,7 @@ struct BankArrays {
   float*    center;         // [d] or nullptr
   // scratch
   float*    pool_partial;   // [(max_batch + 3 * POOL_MAX_GRID), d] partial sums of the pooling pass
+  float*    move_partial;   // 2 x the same: partial sums of the rows moved for hits / for misses (or nullptr)
   unsigned long long* best; // [max_batch] packed (orderable score << 32 | ~slot); 0 = none
   uint32_t* hitcnt;         // [N] matches per slot within the current probe (zero between calls)
   int32_t*  victims;        // [min(max_batch,N)]
@@ -74,6 +77,12 @@ struct llmcache_bank {
   bool     join_pending = false;
   bool     select_deferred = false;   // large bank: the victim selection runs at commit instead
   bool     bits_dirty = true;    // stored fingerprints changed since the SimHash codes were packed
+  // fingerprint-on-write: where the position means of the rows written in a tick go (nullptr: off)
+  float*   pool_out = nullptr;
+  uint32_t pool_out_ld = 0;
+  uint32_t move_grid[2] = {0, 0};   // launch shapes of the two moving passes of the current tick
+  uint32_t move_jmax = 0;
+  bool     moved[2] = {false, false};
   // instrumentation
   uint64_t n_launches = 0;
   bool     prof_on = false;
@@ -109,6 +118,16 @@ PoolPlan pool_plan(uint32_t B, uint32_t n, uint32_t d, bool bf16, int sm_count);
 cudaError_t launch_fingerprint(llmcache_bank* bk, const void* h_in, uint32_t B,
                                __nv_bfloat16* fp, float* rq, cudaStream_t st);
 cudaError_t launch_rownorm(llmcache_bank* bk, const __nv_bfloat16* fp, uint32_t B, uint32_t k, float* rq, cudaStream_t st);
+cudaError_t launch_pool_only(llmcache_bank* bk, const void* h_in, uint32_t B, float* pooled, uint32_t ld, cudaStream_t st);
+cudaError_t launch_fingerprint_pooled(llmcache_bank* bk, const float* pooled, uint32_t ld, uint32_t B,
+                                      __nv_bfloat16* fp, float* rq, cudaStream_t st);
+cudaError_t setup_move_kernels();
+cudaError_t launch_move_pool(llmcache_bank* bk, int which, const void* miss_out, void* h_out,
+                             const llmcache_probe_io* io, uint32_t B, cudaStream_t st);
+cudaError_t launch_pool_finish_moved(llmcache_bank* bk, const llmcache_probe_io* io, uint32_t B,
+                                     float* pooled, uint32_t ld, cudaStream_t st);
+cudaError_t launch_pool_finish_plain(llmcache_bank* bk, const PoolPlan& P, uint32_t B, float* pooled, uint32_t ld,
+                                     cudaStream_t st);
 cudaError_t launch_scan(llmcache_bank* bk, const __nv_bfloat16* q, uint32_t B, cudaStream_t st);
 cudaError_t launch_decide(llmcache_bank* bk, uint32_t B, float tau, const float* rq,
                           const llmcache_probe_io* io, cudaStream_t st, uint32_t sim_k = 0, int32_t ham_max = -1);

@@ -134,9 +134,22 @@ def gpu_probe_result(bufs: L.ProbeBuffers, B, tick) -> O.ProbeResult:
                          miss_idx=bufs.miss_idx[:M].cpu().numpy(), tick=tick)
 
 
+def assert_position_means(pooled_gpu: np.ndarray, h_bits: np.ndarray, n: int, d: int, where=""):
+    """pooled_gpu [B, d] f32 against the exact means of the bf16 rows h_bits [B, n*d].  An fp32 sum of n
+    terms in any order is off by at most (n - 1) * 2^-24 * sum|x|; the division adds one rounding."""
+    x = O.bf16_to_f32(h_bits).astype(np.float64).reshape(h_bits.shape[0], n, d)
+    want = x.mean(axis=1)
+    bound = 2.0 * n * 2.0 ** -24 * np.abs(x).mean(axis=1) + 1e-30
+    err = np.abs(pooled_gpu.astype(np.float64) - want)
+    assert np.all(err <= bound), f"{where} position means off by {np.max(err / bound):.2f} x the bound"
+
+
 def lockstep_step(gb: L.Bank, ob: O.Bank, bufs: L.ProbeBuffers, h_dev: torch.Tensor, dtype: str,
-                  miss_out_dev: torch.Tensor, tau=None, with_act=True, fp_only=False, do_commit=True):
-    """One probe (+ commit) on both sides from the same state.  Returns dict of counters."""
+                  miss_out_dev: torch.Tensor, tau=None, with_act=True, fp_only=False, do_commit=True,
+                  pooled_dev: torch.Tensor = None):
+    """One probe (+ commit) on both sides from the same state.  Returns dict of counters.
+    pooled_dev: the GPU side probes from these position means instead of pooling h_dev itself (the
+    oracle always starts from the hidden states: the result is defined to be the same)."""
     B = h_dev.shape[0]
     pull_state(gb, ob, with_act)
     n, d = gb.n, gb.d
@@ -146,6 +159,8 @@ def lockstep_step(gb: L.Bank, ob: O.Bank, bufs: L.ProbeBuffers, h_dev: torch.Ten
     if fp_only:
         bufs.fp[:B].copy_(h_dev)
         gb.probe_fp(bufs, B, h_out=h_out, tau=tau)
+    elif pooled_dev is not None:
+        gb.probe_pooled(pooled_dev, bufs, B, h_out=h_out, tau=tau, h_in=h_dev)
     else:
         gb.probe(h_dev, bufs, h_out=h_out, tau=tau)
     torch.cuda.synchronize()
@@ -196,4 +211,5 @@ def lockstep_step(gb: L.Bank, ob: O.Bank, bufs: L.ProbeBuffers, h_dev: torch.Ten
         assert np.array_equal(bits(h_out2), ho), "scattered outputs"
     assert_state_equal(gb, ob, with_act=with_act, where="after commit")
     res["inserted"] = int((new_or >= 0).sum())
+    res["h_out"] = h_out2
     return res

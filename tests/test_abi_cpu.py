@@ -27,7 +27,7 @@ def test_library_exports_every_declared_symbol():
 
 
 def test_abi_version_and_strerror():
-    assert L.llmcache_abi_version() == 1
+    assert L.llmcache_abi_version() == 2
     assert L.strerror(0) == "ok" and "argument" in L.strerror(L.ERR_ARG)
 
 

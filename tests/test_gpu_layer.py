@@ -136,6 +136,59 @@ def test_infer_algorithm1_matches_oracle_and_chain_property(pre_ln):
         o.close()
 
 
+def test_infer_with_fingerprint_on_write_equals_plain_loop():
+    """Same batches through llmcache_infer and llmcache_infer_pooled (own banks each): same hits per layer,
+    same output bits.  (The two differ only in where the position means of h_1..h_{L-1} are taken.)"""
+    n, d, heads, ffn, B, Lyr, N, k = 40, 128, 2, 256, 14, 4, 64, 64
+    ws = [synth.layer_weights(d, ffn, 400 + 20 * l, DEV) for l in range(Lyr)]
+    for w in ws:
+        for key in ("w_qkv", "w_o", "w_1", "w_2"):
+            w[key] = (w[key].float() * 3.0).to(torch.bfloat16)
+    proj = synth.projection(d, k, 19, DEV)
+    layers = [L.Layer(w, heads=heads, seq_len=n, max_seqs=B) for w in ws]
+    mkb = lambda fused: [L.Bank(capacity=N, seq_len=n, d_model=d, fp_dim=k, max_batch=B, proj=proj, tau=0.9,
+                                fused_pool=fused) for _ in range(Lyr)]
+    banks_a, banks_b = mkb(0), mkb(1)
+    bufs = L.ProbeBuffers(B, k, DEV)
+    mk = lambda: torch.zeros((B, n, d), dtype=torch.bfloat16, device=DEV)
+    buf_a, buf_b, h_miss, miss_out = mk(), mk(), mk(), mk()
+    pooled = torch.zeros((B, d), dtype=torch.float32, device=DEV)
+    hl = [l.handle for l in layers]
+
+    def run(h0, fused):
+        if fused:
+            ptr = L.llmcache_infer_pooled([b.handle for b in banks_b], hl, h0, B, None, buf_a, buf_b, h_miss, miss_out,
+                                          bufs.io, pooled)
+        else:
+            ptr = L.llmcache_infer([b.handle for b in banks_a], hl, h0, B, None, buf_a, buf_b, h_miss, miss_out, bufs.io)
+        torch.cuda.synchronize()
+        return (buf_a if ptr == buf_a.data_ptr() else buf_b).clone()
+
+    h0 = synth.randn((B, n, d), 3, DEV, torch.bfloat16)
+    batches = [h0]
+    mixed = h0.clone()
+    mixed[1] = (h0[0].float() + 0.02 * synth.randn((n, d), 4, DEV)).to(torch.bfloat16)
+    mixed[5:9] = synth.randn((4, n, d), 5, DEV, torch.bfloat16)
+    batches += [h0, mixed, synth.randn((B, n, d), 6, DEV, torch.bfloat16), mixed]
+    prev_a, prev_b = [0] * Lyr, [0] * Lyr
+    total = 0
+    for i, hb in enumerate(batches):
+        oa, ob = run(hb, False), run(hb, True)
+        ha = [b.stats()["hits"] for b in banks_a]
+        hb_ = [b.stats()["hits"] for b in banks_b]
+        assert [x - y for x, y in zip(ha, prev_a)] == [x - y for x, y in zip(hb_, prev_b)], f"batch {i}"
+        total += ha[0] - prev_a[0]
+        prev_a, prev_b = ha, hb_
+        assert torch.equal(oa.view(torch.int16), ob.view(torch.int16)), f"batch {i}"
+    assert total >= B + (B - 4)
+    launches_a = sum(b.stats()["kernel_launches"] for b in banks_a)
+    launches_b = sum(b.stats()["kernel_launches"] for b in banks_b)
+    assert launches_b != launches_a                      # the pooled loop really took the other path
+    assert all(l.status() == L.OK for l in layers) and all(b.status() == L.OK for b in banks_a + banks_b)
+    for o in layers + banks_a + banks_b:
+        o.close()
+
+
 def test_divergence_monitor_matches_oracle():
     """Stored outputs that no longer match what the layer produces are found and invalidated; the relative
     differences agree with the oracle's within the layer tolerance (absolute 1e-2 on a quantity of order
