@@ -137,9 +137,8 @@ enum {
   LLMCACHE_K_SELECT = 7,    /* Sec. IV-D victim selection (side stream, during GATHER) */
   LLMCACHE_K_SCATTER = 8,   /* Algorithm 1 insert: write-back + store              */
   LLMCACHE_K_EVICT = 9,     /* Sec. III-E flushes                                  */
-  LLMCACHE_K_INSERT = 10,   /* keys + metadata of new entries (when the rows move in a pooling pass) */
-  LLMCACHE_K_POOL_FINISH = 11, /* partial column sums -> position means               */
-  LLMCACHE_K_COUNT = 12
+  LLMCACHE_K_POOL_FINISH = 10, /* partial column sums -> position means               */
+  LLMCACHE_K_COUNT = 11
 };
 
 uint32_t    llmcache_abi_version(void);

@@ -39,7 +39,7 @@ EXPORTS = [
 ]
 FINGERPRINT_STATIC_MAX_FLOATS = 2 * 1024 * 1024
 KERNEL_NAMES = ["pool", "project", "rownorm", "scan", "decide", "touch", "gather", "select", "scatter", "evict",
-                "insert", "pool_finish"]
+                "pool_finish"]
 
 
 class BankDesc(C.Structure):

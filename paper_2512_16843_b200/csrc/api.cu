@@ -383,7 +383,7 @@ static int probe_common(llmcache_bank_t* bk, const void* h_in, bool compute_fp, 
     bk->moved[0] = bk->moved[1] = false;
     if (bk->pool_out) {
       // the reused rows are summed while they are copied; the miss inputs (if wanted) go the plain way
-      if (e == cudaSuccess) e = launch_move_pool(bk, 0, nullptr, h_out, io, B, st);
+      if (e == cudaSuccess) e = launch_move_pool(bk, 0, nullptr, h_out, io, nullptr, B, st);
       if (e == cudaSuccess) bk->moved[0] = true;
       if (e == cudaSuccess && h_in && io->h_miss) e = launch_gather(bk, h_in, nullptr, io, B, st);
     } else {
@@ -445,9 +445,8 @@ int llmcache_commit(llmcache_bank_t* bk, const void* miss_out, const llmcache_pr
   if (e == cudaSuccess && bk->select_deferred) e = launch_select_victims(bk, io, B, st);
   bk->select_deferred = false;
   if (bk->pool_out && bk->moved[0]) {
-    // keys and metadata of the new entries, then the rows (summed while they move), then the means
-    if (e == cudaSuccess) e = launch_scatter_insert(bk, nullptr, io, nullptr, new_slot, B, st);
-    if (e == cudaSuccess) e = launch_move_pool(bk, 1, miss_out, h_out, io, B, st);
+    // the rows (summed while they move) with the keys and metadata of the new entries, then the means
+    if (e == cudaSuccess) e = launch_move_pool(bk, 1, miss_out, h_out, io, new_slot, B, st);
     if (e == cudaSuccess) e = launch_pool_finish_moved(bk, io, B, bk->pool_out, bk->pool_out_ld, st);
     bk->moved[0] = bk->moved[1] = false;
   } else {

@@ -123,7 +123,7 @@ cudaError_t launch_fingerprint_pooled(llmcache_bank* bk, const float* pooled, ui
                                       __nv_bfloat16* fp, float* rq, cudaStream_t st);
 cudaError_t setup_move_kernels();
 cudaError_t launch_move_pool(llmcache_bank* bk, int which, const void* miss_out, void* h_out,
-                             const llmcache_probe_io* io, uint32_t B, cudaStream_t st);
+                             const llmcache_probe_io* io, int32_t* new_slot_out, uint32_t B, cudaStream_t st);
 cudaError_t launch_pool_finish_moved(llmcache_bank* bk, const llmcache_probe_io* io, uint32_t B,
                                      float* pooled, uint32_t ld, cudaStream_t st);
 cudaError_t launch_pool_finish_plain(llmcache_bank* bk, const PoolPlan& P, uint32_t B, float* pooled, uint32_t ld,

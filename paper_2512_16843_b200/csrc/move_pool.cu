@@ -41,6 +41,13 @@ struct MoveArgs {
   float* partial;            // [gridDim.x * Jmax, d]
   uint32_t* status;
   uint32_t act_rows, n, d, V, R, Jmax, stage_rows, stages, cons_threads;
+  // scatter only: the new entries' keys and metadata (Algorithm 1 "C_l[f_X] <- h_l"), written by the block
+  // that moves the first row of a sequence; block 0 also reports the slots and adds up the counters
+  const uint4* q_fp; const float* rq; uint32_t kv;                  // query fingerprints, 16-byte vectors per row
+  uint4* bank_fp; float* rb; uint8_t* valid;
+  uint32_t* last_use; uint32_t* insert_tick; uint32_t* hits; uint32_t* rate; uint32_t* rate_epoch;
+  uint32_t tick, epoch;
+  int32_t* new_slot_out; const uint32_t* tally; unsigned long long* stats;
 };
 
 // Addresses of the i-th sequence of the list.
@@ -76,7 +83,17 @@ k_move_pool(const MoveArgs a) {
   auto full_bar = [&](uint32_t s) { return bar0 + 8 * s; };
   auto empty_bar = [&](uint32_t s) { return bar0 + 8 * (stages + s); };
 
-  const unsigned long long total = (unsigned long long)(*a.count) * n;
+  const uint32_t count = *a.count;
+  if (blockIdx.x == 0 && a.bank_fp) {
+    if (a.new_slot_out)
+      for (uint32_t m = threadIdx.x; m < count; m += blockDim.x) a.new_slot_out[m] = a.new_slot[m];
+    if (threadIdx.x == 0) {
+      a.stats[ST_INSERT] += a.tally[0];
+      a.stats[ST_EVICT] += a.tally[1];
+      a.stats[ST_DROP] += a.tally[2];
+    }
+  }
+  const unsigned long long total = (unsigned long long)count * n;
   const unsigned long long L = (total + gridDim.x - 1) / gridDim.x;
   unsigned long long r = (unsigned long long)blockIdx.x * L;
   unsigned long long r1 = r + L;
@@ -160,6 +177,23 @@ k_move_pool(const MoveArgs a) {
     while (r < r1) {
       unsigned long long seg_end = (unsigned long long)(i + 1) * n;
       if (seg_end > r1) seg_end = r1;
+      if (a.bank_fp && r == (unsigned long long)i * n) {              // this block moves the sequence's first row
+        const int32_t v = a.new_slot[i];
+        if (v >= 0) {
+          const int32_t b = a.idx[i];
+          for (uint32_t c = threadIdx.x; c < a.kv; c += cons_threads)
+            a.bank_fp[(size_t)v * a.kv + c] = a.q_fp[(size_t)b * a.kv + c];
+          if (threadIdx.x == 0) {
+            a.rb[v] = a.rq[b];
+            a.valid[v] = 1;
+            a.last_use[v] = a.tick;
+            a.insert_tick[v] = a.tick;
+            a.hits[v] = 0;
+            a.rate[v] = HIT_Q8;
+            a.rate_epoch[v] = a.epoch;
+          }
+        }
+      }
       float acc[8];
 #pragma unroll
       for (int e = 0; e < 8; ++e) acc[e] = 0.f;
@@ -250,7 +284,7 @@ cudaError_t setup_move_kernels() {
 
 // which: 0 = hits (bank rows -> h_out), 1 = misses (miss_out -> h_out and the bank)
 cudaError_t launch_move_pool(llmcache_bank* bk, int which, const void* miss_out, void* h_out,
-                             const llmcache_probe_io* io, uint32_t B, cudaStream_t st) {
+                             const llmcache_probe_io* io, int32_t* new_slot_out, uint32_t B, cudaStream_t st) {
   if (B == 0) return cudaSuccess;
   const llmcache_bank_desc& D = bk->desc;
   const PoolPlan P = pool_plan(B, D.seq_len, D.d_model, true, bk->sm_count);
@@ -267,6 +301,14 @@ cudaError_t launch_move_pool(llmcache_bank* bk, int which, const void* miss_out,
   a.act_rows = D.act_rows;
   a.n = D.seq_len; a.d = D.d_model; a.V = P.V; a.R = P.R; a.Jmax = P.Jmax;
   a.stage_rows = P.stage_rows; a.stages = P.stages; a.cons_threads = P.cons_threads;
+  if (which == 1) {
+    a.q_fp = (const uint4*)io->fp; a.rq = (const float*)io->rq; a.kv = D.fp_dim / 8;
+    a.bank_fp = (uint4*)bk->a.fp; a.rb = bk->a.rb; a.valid = bk->a.valid;
+    a.last_use = bk->a.last_use; a.insert_tick = bk->a.insert_tick; a.hits = bk->a.hits;
+    a.rate = bk->a.rate; a.rate_epoch = bk->a.rate_epoch;
+    a.tick = (uint32_t)bk->tick; a.epoch = (uint32_t)(bk->tick / bk->pol.half_life);
+    a.new_slot_out = new_slot_out; a.tally = (const uint32_t*)bk->a.misc; a.stats = bk->a.stats;
+  }
   bk->move_grid[which] = P.grid;
   bk->move_jmax = P.Jmax;
   ProfScope prof(bk, which == 0 ? LLMCACHE_K_GATHER : LLMCACHE_K_SCATTER, st);

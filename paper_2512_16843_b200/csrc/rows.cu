@@ -183,8 +183,7 @@ cudaError_t launch_scatter_insert(llmcache_bank* bk, const void* miss_out, const
   const llmcache_bank_desc& D = bk->desc;
   const size_t row_bytes = (size_t)D.seq_len * D.d_model * 2;
   const uint32_t epoch = (uint32_t)(bk->tick / bk->pol.half_life);
-  // without rows to move only the keys and the metadata of the new entries are written
-  ProfScope prof(bk, miss_out ? LLMCACHE_K_SCATTER : LLMCACHE_K_INSERT, st);
+  ProfScope prof(bk, LLMCACHE_K_SCATTER, st);
   return launch_k(k_scatter_insert, dim3(copy_grid(bk, B, row_bytes, g_scatter_occ)), dim3(COPY_THREADS), 0, st,
                   (const char*)miss_out, (char*)h_out, (char*)bk->a.act, row_bytes, (const int32_t*)io->miss_idx,
                   (const int32_t*)bk->a.new_slot, (const uint32_t*)io->counts, (const uint4*)io->fp,
