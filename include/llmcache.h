@@ -176,7 +176,8 @@ int llmcache_fingerprint_pooled(llmcache_bank_t* bank, const float* pooled, uint
                                 void* fp, float* rq, void* stream);
 
 /* Fingerprint for callers that must not allocate device memory.  (The paper has no counterpart:
- * this is a packaging variant of llmcache_fingerprint, same kernels, same result.)
+ * this is a packaging variant of llmcache_fingerprint: the same arithmetic, run as two kernels whose
+ * fp32 sums may be taken in another order, so results agree to rounding, not bit for bit.)
  *
  * Who needs it: code that runs after its host application has handed all device memory to its own
  * pool (an inference server that reserves the GPU at start-up, say), or inside a latency-critical

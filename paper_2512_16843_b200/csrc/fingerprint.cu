@@ -1,303 +1,104 @@
 // Fingerprint kernels (Sec. IV-B): pooled reduction over the sequence
 // positions, centring + projection, unit-length scaling, bf16 rounding.
+//
+//   k_pool          the pooling pass
+//   k_project       projection + rounding (from the pooling pass's partial sums or from given position
+//                   means) on the tensor cores, one thread-block cluster per group of 8 sequences
+//   k_normalise     the same without a projection matrix
+//   k_rownorm       inverse norms of caller-supplied fingerprints
 #include "llmcache_internal.cuh"
 #include "ptx.cuh"
+#include "fp_phases.cuh"
 
 namespace llmc {
 
-// ---------------------------------------------------------------------------
-// Pool.  The B*n rows of the batch are one flat list that is cut into equal
-// spans, one per block (one block per SM), so every block streams the same
-// number of bytes.  A span may cross sequence boundaries: a block writes one
-// vector of partial sums per sequence it touches,
-//     partial[(block * Jmax + j), :] = sum of its rows of the j-th sequence it touches.
-//
-// The rows of a span are contiguous in memory.  One producer thread moves them
-// into a ring of shared-memory stages with bulk asynchronous copies (completion
-// counted on an mbarrier per stage), which keeps well over 100 KB of reads in
-// flight per SM without holding them in registers.  The consumer threads form a
-// V x R grid: V = 16-byte vectors per row, R = rows taken per pass; every thread
-// always owns the same E columns, so the running sums live in registers.  At the
-// end of a sequence's rows the R row groups are combined through shared memory
-// in a fixed order (deterministic).  A stage never crosses a sequence boundary.
-// All waits are bounded; on expiry the status word is set and the block drains
-// its copies and leaves.
-// ---------------------------------------------------------------------------
 template <bool BF16>
 __global__ void __launch_bounds__(1024, 1)
-k_pool(const uint4* __restrict__ h, float* __restrict__ partial, uint32_t* __restrict__ status,
-       uint32_t B, uint32_t n, uint32_t d, uint32_t V, uint32_t R, uint32_t L, uint32_t Jmax,
-       uint32_t stage_rows, uint32_t stages, uint32_t cons_threads) {
+k_pool(const uint4* __restrict__ h, float* __restrict__ partial, uint32_t* __restrict__ status, PoolShape S) {
   griddep_sync();
-  constexpr int E = BF16 ? 8 : 4;
   extern __shared__ __align__(128) uint8_t sm_raw[];
-  const uint32_t row_bytes = V * 16;
-  const uint32_t stage_bytes = stage_rows * row_bytes;
-  const uint32_t ring = smem_u32(sm_raw);
-  float* red = reinterpret_cast<float*>(sm_raw + (size_t)stages * stage_bytes);          // [R][d]
-  uint8_t* tail = reinterpret_cast<uint8_t*>(red + (size_t)R * d);
-  const uint32_t bar0 = smem_u32(tail);                                                  // full[stages], empty[stages]
-  volatile uint32_t* flags = reinterpret_cast<volatile uint32_t*>(tail + 16 * stages);   // [0] abort, [1] go
-  auto full_bar = [&](uint32_t s) { return bar0 + 8 * s; };
-  auto empty_bar = [&](uint32_t s) { return bar0 + 8 * (stages + s); };
+  pool_phase<BF16>(sm_raw, h, partial, status, S);
+}
 
-  if (threadIdx.x == 0) {
-    for (uint32_t s = 0; s < stages; ++s) { mbar_init(full_bar(s), 1); mbar_init(empty_bar(s), cons_threads / 32); }
-    flags[0] = 0; flags[1] = 0;
-    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
-    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
-  }
+// ---------------------------------------------------------------------------
+// Projection + rounding as a kernel of its own.  One thread-block cluster of S blocks serves G
+// sequences: the d rows of P are split over the S blocks, the S partial results meet in block 0's
+// shared memory (distributed shared memory) and are added there in block order.  The producer thread
+// starts before the preceding grid has finished: P never changes.  Every block of a cluster reaches
+// both cluster barriers whatever happens.
+// ---------------------------------------------------------------------------
+__device__ __forceinline__ uint32_t cluster_rank() { uint32_t r; asm volatile("mov.u32 %0, %%cluster_ctarank;" : "=r"(r)); return r; }
+__device__ __forceinline__ uint32_t cluster_size() { uint32_t r; asm volatile("mov.u32 %0, %%cluster_nctarank;" : "=r"(r)); return r; }
+__device__ __forceinline__ void cluster_sync_all() {
+  asm volatile("barrier.cluster.arrive.release.aligned;" ::: "memory");
+  asm volatile("barrier.cluster.wait.acquire.aligned;" ::: "memory");
+}
+// address of the same shared-memory location in block `rank` of the cluster
+__device__ __forceinline__ uint32_t cluster_map(uint32_t saddr, uint32_t rank) {
+  uint32_t r;
+  asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(r) : "r"(saddr), "r"(rank));
+  return r;
+}
+__device__ __forceinline__ void st_cluster_f32(uint32_t addr, float v) {
+  asm volatile("st.shared::cluster.f32 [%0], %1;" ::"r"(addr), "f"(v) : "memory");
+}
+
+template <int NT>
+__global__ void __launch_bounds__(PROJ_THREADS, 1)
+k_project(const __grid_constant__ CUtensorMap map_p, MeanSrc src, __nv_bfloat16* __restrict__ fp, float* __restrict__ rq,
+          uint32_t* __restrict__ status, uint32_t B, ProjShape S, uint32_t rows_per) {
+  extern __shared__ __align__(128) uint8_t sm_raw[];
+  const uint32_t CS = cluster_size(), rank = cluster_rank();
+  const uint32_t b0 = (blockIdx.x / CS) * PROJ_G, k = S.k, d = src.d;
+  const uint32_t r0 = min(d, rank * rows_per), nrows = min(d, r0 + rows_per) - r0;
+  const ProjSmem m = proj_smem(sm_raw, S);
+  if (threadIdx.x == 0) proj_init(m, S, true);
   __syncthreads();
 
-  const unsigned long long total = (unsigned long long)B * n;
-  unsigned long long r = (unsigned long long)blockIdx.x * L;
-  unsigned long long r1 = r + L;
-  if (r1 > total) r1 = total;
-  uint32_t b = (uint32_t)(r / n);
-  uint32_t it = 0;
-
-  if (threadIdx.x >= cons_threads) {
-    // ---------------------------------------------------------------- producer (one thread)
-    if (threadIdx.x == cons_threads) {
-      bool ok = true;
-      while (r < r1 && ok) {
-        unsigned long long seg_end = (unsigned long long)(b + 1) * n;
-        if (seg_end > r1) seg_end = r1;
-        while (r < seg_end) {
-          const uint32_t rows = (uint32_t)min((unsigned long long)stage_rows, seg_end - r);
-          const uint32_t s = it % stages, ph = (it / stages) & 1u;
-          if (!mbar_wait(empty_bar(s), ph ^ 1u, flags)) { ok = false; break; }
-          mbar_expect_tx(full_bar(s), rows * row_bytes);
-          bulk_load_1d(ring + s * stage_bytes, h + r * V, rows * row_bytes, full_bar(s));
-          r += rows;
-          ++it;
-        }
-        ++b;
-      }
-      if (!ok) {
-        flags[0] = 1;
-        atomicExch(status, 1u);
-        // copies that were started must land before the block's shared memory is released
-        const uint32_t back = it < stages ? it : stages;
-        volatile uint32_t never = 0;
-        for (uint32_t i = 0; i < back; ++i) {
-          const uint32_t itx = it - 1 - i;
-          mbar_wait(full_bar(itx % stages), (itx / stages) & 1u, &never, 200000000ull);
-        }
-      }
+  float vals[2 * NT];
+#pragma unroll
+  for (int i = 0; i < 2 * NT; ++i) vals[i] = 0.f;
+  if (threadIdx.x >= PROJ_CONS) {
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+    if (threadIdx.x == PROJ_CONS) {
+      uint32_t it = 0;
+      if (!proj_produce(m, S, &map_p, r0, nrows, blockIdx.x * 5u, it)) proj_drain(m, S, it, status);
     }
+    __syncwarp();
   } else {
-    // ---------------------------------------------------------------- consumers
-    const bool active = threadIdx.x < V * R;
-    const uint32_t col = threadIdx.x % V, rg = threadIdx.x / V;
-    float* out = partial + (size_t)blockIdx.x * Jmax * d;
-    while (r < r1) {
-      unsigned long long seg_end = (unsigned long long)(b + 1) * n;
-      if (seg_end > r1) seg_end = r1;
-      float acc[E];
-#pragma unroll
-      for (int e = 0; e < E; ++e) acc[e] = 0.f;
-      while (r < seg_end) {
-        const uint32_t rows = (uint32_t)min((unsigned long long)stage_rows, seg_end - r);
-        const uint32_t s = it % stages, ph = (it / stages) & 1u;
-        if (!mbar_wait(full_bar(s), ph, flags)) { flags[0] = 1; atomicExch(status, 1u); }
-        if (active) {
-          const uint32_t src = ring + s * stage_bytes + col * 16;
-          for (uint32_t rr = rg; rr < rows; rr += R) {
-            const uint4 v = lds16(src + rr * row_bytes);
-            if (BF16) {
-              const uint32_t w[4] = {v.x, v.y, v.z, v.w};
-#pragma unroll
-              for (int i = 0; i < 4; ++i) {
-                acc[2 * i]     += __uint_as_float(w[i] << 16);
-                acc[2 * i + 1] += __uint_as_float(w[i] & 0xFFFF0000u);
-              }
-            } else {
-              acc[0] += __uint_as_float(v.x); acc[1] += __uint_as_float(v.y);
-              acc[2] += __uint_as_float(v.z); acc[3] += __uint_as_float(v.w);
-            }
-          }
-        }
-        __syncwarp();
-        if ((threadIdx.x & 31) == 0) mbar_arrive(empty_bar(s));      // this warp is done with the stage
-        r += rows;
-        ++it;
-      }
-      // combine the row groups of this sequence piece (consumer threads only)
-      if (active) {
-#pragma unroll
-        for (int e = 0; e < E; ++e) red[(size_t)rg * d + col * E + e] = acc[e];
-      }
-      if (threadIdx.x == 0) flags[1] = flags[0];
-      asm volatile("bar.sync 1, %0;" ::"r"(cons_threads) : "memory");
-      if (flags[1]) break;                                           // uniform over the consumers
-      for (uint32_t i = threadIdx.x; i < d; i += cons_threads) {
-        float sum = 0.f;
-        for (uint32_t q = 0; q < R; ++q) sum += red[(size_t)q * d + i];
-        out[i] = sum;
-      }
-      asm volatile("bar.sync 1, %0;" ::"r"(cons_threads) : "memory");
-      out += d;
-      ++b;
-    }
+    proj_prepare(m, src, b0);
+    griddep_sync();
+    uint32_t it = 0;
+    proj_consume<NT>(m, S, src, B, b0, r0, nrows, blockIdx.x * 5u, it, status, vals);
   }
-  __syncthreads();
+  // every block of the cluster is done with its own ring: block 0's may now receive the CS partial results
+  cluster_sync_all();
+  if (threadIdx.x < PROJ_CONS) {
+    const uint32_t dst0 = cluster_map(m.ring, 0) + rank * (PROJ_G * k * 4);
+#pragma unroll
+    for (int t = 0; t < NT; ++t)
+#pragma unroll
+      for (int e = 0; e < 2; ++e) {
+        const uint32_t idx = proj_val_index<NT>(k, t, e);
+        if (idx != 0xFFFFFFFFu) st_cluster_f32(dst0 + idx * 4, vals[2 * t + e]);
+      }
+  }
+  cluster_sync_all();
+  if (rank != 0 || threadIdx.x >= PROJ_CONS) return;
+  for (uint32_t idx = threadIdx.x; idx < PROJ_G * k; idx += PROJ_CONS) {
+    float v = m.part[idx];
+    for (uint32_t r = 1; r < CS; ++r) v += m.part[(size_t)r * PROJ_G * k + idx];
+    m.part[idx] = v;
+  }
+  asm volatile("bar.sync 1, %0;" ::"n"(PROJ_CONS) : "memory");
+  finish_group(m.part, k, B, b0, fp, rq);
 }
 
-// ---------------------------------------------------------------------------
-// Project + normalise: G sequences per block, 128 threads per sequence in the
-// element-wise phases.
-//   p = (sum of the sequence's partial vectors) / n - mu ;  g = p . P  (or p when no projection)
-//   q = bf16(g / ||g||) ; rq = 1 / ||q||
-// P is read with 16-byte loads: a thread owns 8 adjacent output columns and
-// every `slices`-th row; the row slices are combined through shared memory in a
-// fixed order.
-// ---------------------------------------------------------------------------
-constexpr int PROJ_G = 2;
-constexpr int PROJ_THREADS = 1024;
-constexpr int PROJ_TPS = PROJ_THREADS / PROJ_G;      // threads per sequence
-
-// Sum over the TPS threads that serve one sequence (fixed order).  red: [PROJ_THREADS / 32] floats.
-__device__ __forceinline__ float group_sum(float v, float* red, int group) {
-#pragma unroll
-  for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xFFFFFFFFu, v, o);
-  const int w = threadIdx.x >> 5, l = threadIdx.x & 31;
-  __syncthreads();
-  if (l == 0) red[w] = v;
-  __syncthreads();
-  float tot = 0.f;
-  constexpr int WPG = PROJ_TPS / 32;
-#pragma unroll
-  for (int i = 0; i < WPG; ++i) tot += red[group * WPG + i];
-  return tot;
-}
-
-__global__ void __launch_bounds__(PROJ_THREADS)
-k_project(const float* __restrict__ partial, const __nv_bfloat16* __restrict__ proj,
-          const float* __restrict__ center, __nv_bfloat16* __restrict__ fp, float* __restrict__ rq,
-          uint32_t B, uint32_t n, uint32_t d, uint32_t k, uint32_t L, uint32_t Jmax,
-          const float* __restrict__ pooled, uint32_t ld) {
+__global__ void __launch_bounds__(NRM_THREADS)
+k_normalise(MeanSrc src, __nv_bfloat16* __restrict__ fp, float* __restrict__ rq) {
   griddep_sync();
-  extern __shared__ float sm[];
-  float* p = sm;                               // [G][d]
-  float* g = p + (size_t)PROJ_G * d;           // [G][k]            (only with projection)
-  float* part = g + (size_t)PROJ_G * k;        // [slices][G][k]    (only with projection)
-  __shared__ float red[PROJ_THREADS / 32];
-  const uint32_t b0 = blockIdx.x * PROJ_G;
-  const float fn = (float)n;
-  const int grp = threadIdx.x / PROJ_TPS;      // sequence served in the element-wise phases
-  const uint32_t gt = threadIdx.x % PROJ_TPS;
-  const uint32_t bq = b0 + grp;
-
-  {
-    // pool blocks whose span overlaps rows [b*n, (b+1)*n), in block order
-    float* pg = p + (size_t)grp * d;
-    if (bq < B && pooled) {
-      // the position means were taken elsewhere (while the rows were written)
-      for (uint32_t i = gt; i < d; i += PROJ_TPS) {
-        float v = pooled[(size_t)bq * ld + i];
-        if (center) v -= center[i];
-        pg[i] = v;
-      }
-    } else if (bq < B) {
-      const unsigned long long first = (unsigned long long)bq * n, last = first + n - 1;
-      const uint32_t c_lo = (uint32_t)(first / L), c_hi = (uint32_t)(last / L);
-      const uint32_t j_lo = bq - (uint32_t)(((unsigned long long)c_lo * L) / n);
-      for (uint32_t i = gt; i < d; i += PROJ_TPS) {
-        // the first block may have touched earlier sequences (index j_lo); later blocks start inside bq
-        float v = partial[((size_t)c_lo * Jmax + j_lo) * d + i];
-        for (uint32_t c = c_lo + 1; c <= c_hi; ++c) v += partial[(size_t)c * Jmax * d + i];
-        v = v / fn;
-        if (center) v -= center[i];
-        pg[i] = v;
-      }
-    } else {
-      for (uint32_t i = gt; i < d; i += PROJ_TPS) pg[i] = 0.f;
-    }
-  }
-  __syncthreads();
-
-  if (proj) {
-    const uint32_t ncg = k >> 3;                                   // groups of 8 columns
-    const uint32_t slices = ncg >= blockDim.x ? 1u : blockDim.x / ncg;
-    const uint4* P4 = reinterpret_cast<const uint4*>(proj);
-    for (uint32_t cg0 = 0; cg0 < ncg; cg0 += blockDim.x) {         // one trip unless k > 8 * threads
-      const uint32_t cg = cg0 + (ncg >= blockDim.x ? threadIdx.x : threadIdx.x % ncg);
-      const uint32_t sl = ncg >= blockDim.x ? 0u : threadIdx.x / ncg;
-      if (cg < ncg && sl < slices) {
-        float acc[PROJ_G][8];
-#pragma unroll
-        for (int gi = 0; gi < PROJ_G; ++gi)
-#pragma unroll
-          for (int e = 0; e < 8; ++e) acc[gi][e] = 0.f;
-        auto fma_row = [&](const uint4& w, uint32_t i) {
-          const uint32_t ww[4] = {w.x, w.y, w.z, w.w};
-          float x[PROJ_G];
-#pragma unroll
-          for (int gi = 0; gi < PROJ_G; ++gi) x[gi] = p[gi * d + i];
-#pragma unroll
-          for (int u = 0; u < 4; ++u) {
-            const float w0 = __uint_as_float(ww[u] << 16), w1 = __uint_as_float(ww[u] & 0xFFFF0000u);
-#pragma unroll
-            for (int gi = 0; gi < PROJ_G; ++gi) {
-              acc[gi][2 * u]     = fmaf(x[gi], w0, acc[gi][2 * u]);
-              acc[gi][2 * u + 1] = fmaf(x[gi], w1, acc[gi][2 * u + 1]);
-            }
-          }
-        };
-        constexpr int INFL = 8;                                    // rows in flight
-        // This thread's rows are sl, sl + slices, ...  Every block reads the same matrix, so each block
-        // starts at a different one of them (and wraps): the blocks then ask for different lines at any
-        // moment instead of all hitting one L2 line together.
-        const uint32_t nrow = sl < d ? (d - sl + slices - 1) / slices : 0u;
-        const uint32_t rot = nrow ? (blockIdx.x * 5u) % nrow : 0u;
-        auto row_of = [&](uint32_t t) { uint32_t tt = t + rot; if (tt >= nrow) tt -= nrow; return sl + tt * slices; };
-        uint32_t t = 0;
-        for (; t + INFL <= nrow; t += INFL) {
-          uint4 w[INFL];
-          uint32_t ri[INFL];
-#pragma unroll
-          for (int u = 0; u < INFL; ++u) { ri[u] = row_of(t + u); w[u] = ld_nc16(P4 + (size_t)ri[u] * ncg + cg); }
-#pragma unroll
-          for (int u = 0; u < INFL; ++u) fma_row(w[u], ri[u]);
-        }
-        for (; t < nrow; ++t) { const uint32_t i = row_of(t); fma_row(ld_nc16(P4 + (size_t)i * ncg + cg), i); }
-#pragma unroll
-        for (int gi = 0; gi < PROJ_G; ++gi)
-#pragma unroll
-          for (int e = 0; e < 8; ++e) part[((size_t)sl * PROJ_G + gi) * k + cg * 8 + e] = acc[gi][e];
-      }
-    }
-    __syncthreads();
-    for (uint32_t idx = threadIdx.x; idx < PROJ_G * k; idx += blockDim.x) {
-      float v = 0.f;
-      for (uint32_t sl = 0; sl < slices; ++sl) v += part[(size_t)sl * PROJ_G * k + idx];
-      g[idx] = v;
-    }
-    __syncthreads();
-  } else {
-    g = p;                                      // identity: k == d
-  }
-
-  // unit length + rounding: the G sequences side by side, 128 threads each
-  const float* gv = g + (size_t)grp * k;
-  float ss = 0.f;
-  for (uint32_t c = gt; c < k; c += PROJ_TPS) ss = fmaf(gv[c], gv[c], ss);
-  ss = group_sum(ss, red, grp);
-  const float nrm = sqrtf(ss);
-  const bool ok = isfinite(ss) && nrm >= 1e-20f;
-  float qs = 0.f;
-  if (bq < B) {
-    __nv_bfloat16* dst = fp + (size_t)bq * k;
-    for (uint32_t c = gt; c < k; c += PROJ_TPS) {
-      __nv_bfloat16 q = __float2bfloat16_rn(ok ? gv[c] / nrm : 0.f);
-      dst[c] = q;
-      const float qf = __bfloat162float(q);
-      qs = fmaf(qf, qf, qs);
-    }
-  }
-  qs = group_sum(qs, red, grp);
-  if (gt == 0 && bq < B) rq[bq] = (ok && qs > 0.f) ? 1.0f / sqrtf(qs) : 0.f;
+  extern __shared__ float nrm_sm[];              // [d] + [32]
+  normalise_seq(src, blockIdx.x, nrm_sm, nrm_sm + src.d, threadIdx.x, 1, fp, rq);
 }
 
 // rq[b] = 1/||fp[b]|| for fingerprints supplied by the caller; one warp per row.
@@ -323,16 +124,72 @@ __global__ void k_rownorm(const __nv_bfloat16* __restrict__ fp, uint32_t B, uint
 }
 
 // ---------------------------------------------------------------------------
+// Launch shapes.
+// ---------------------------------------------------------------------------
+constexpr uint32_t PROJ_RING_BYTES = 128 * 1024;
+constexpr uint32_t PROJ_STAGE_BYTES = 32 * 1024;
+constexpr uint32_t PROJ_A_ROWS = 1024;            // most rows of P per refill of the A operand
+
+// NT: 8-column tiles per consumer warp; split: blocks (of one cluster) that share the rows of P of a group.
+struct ProjPlan { int NT; uint32_t split, groups, rows_per; ProjShape shape; size_t smem; };
+
+// max_blocks: number of blocks the groups may be spread over by splitting the rows of P (1: no splitting).
+static ProjPlan proj_plan(uint32_t B, uint32_t d, uint32_t k, uint32_t max_blocks) {
+  ProjPlan P;
+  const uint32_t tiles = k / 8, warps = PROJ_CONS / 32;
+  P.NT = 1;
+  while ((uint32_t)P.NT * warps < tiles) P.NT *= 2;
+  P.groups = (B + PROJ_G - 1) / PROJ_G;
+  ProjShape& sh = P.shape;
+  sh.k = k;
+  const uint32_t row_bytes = k * 2;
+  sh.stage_rows = (PROJ_STAGE_BYTES / row_bytes) / PROJ_KSTEP * PROJ_KSTEP;
+  if (sh.stage_rows < PROJ_KSTEP) sh.stage_rows = PROJ_KSTEP;
+  if (sh.stage_rows > 256) sh.stage_rows = 256;                                // most rows of a TMA box
+  const uint32_t stage_bytes = sh.stage_rows * row_bytes;
+  sh.stages = PROJ_RING_BYTES / stage_bytes;
+  if (sh.stages < 2) sh.stages = 2;
+  if (sh.stages > 8) sh.stages = 8;
+  size_t ring = (size_t)sh.stages * stage_bytes;
+  if (ring < (size_t)PROJ_G * k * 4) ring = (size_t)PROJ_G * k * 4;            // the ring is reused for the group's result
+  sh.ring_bytes = (uint32_t)((ring + 127) / 128 * 128);
+  sh.a_rows = PROJ_A_ROWS / sh.stage_rows * sh.stage_rows;
+  if (sh.a_rows < sh.stage_rows) sh.a_rows = sh.stage_rows;
+  sh.a_stride = (sh.a_rows * 2 + 127) / 128 * 128 + 16;
+  // spread the rows of P over the blocks of a cluster while SMs are idle, an item keeps at least 128 rows and
+  // block 0's ring can take the partial results
+  uint32_t S = 1;
+  while (S < 8 && (unsigned long long)P.groups * S * 2 <= (unsigned long long)max_blocks && (d + 2 * S - 1) / (2 * S) >= 128 &&
+         (size_t)2 * S * PROJ_G * k * 4 <= sh.ring_bytes)
+    S *= 2;
+  P.split = S;
+  P.rows_per = (d + S - 1) / S;
+  P.smem = (size_t)SMEM_HEAD + sh.ring_bytes + (size_t)3 * PROJ_G * sh.a_stride;
+  return P;
+}
+
+// Dynamic shared memory of the fingerprint's second kernel.
 size_t project_smem_bytes(uint32_t d, uint32_t k, bool has_proj) {
-  const uint32_t ncg = k / 8;
-  const uint32_t slices = (has_proj && ncg < (uint32_t)PROJ_THREADS) ? PROJ_THREADS / ncg : 1;
-  return ((size_t)PROJ_G * d + (has_proj ? (size_t)PROJ_G * k + (size_t)slices * PROJ_G * k : 0)) * sizeof(float);
+  if (!has_proj) return (size_t)d * sizeof(float) + 128;
+  return proj_plan(1, d, k, 1).smem;
+}
+
+template <int NT>
+static cudaError_t set_smem_limit_nt() {
+  const int lim = 220 * 1024;
+  return cudaFuncSetAttribute(k_project<NT>, cudaFuncAttributeMaxDynamicSharedMemorySize, lim);
 }
 
 cudaError_t setup_fingerprint_kernels() {
-  cudaError_t e = cudaFuncSetAttribute(k_project, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024);
-  if (e == cudaSuccess) e = cudaFuncSetAttribute(k_pool<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, 220 * 1024);
-  if (e == cudaSuccess) e = cudaFuncSetAttribute(k_pool<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, 220 * 1024);
+  const int lim = 220 * 1024;
+  cudaError_t e = tensor_map_setup();
+  if (e == cudaSuccess) e = set_smem_limit_nt<1>();
+  if (e == cudaSuccess) e = set_smem_limit_nt<2>();
+  if (e == cudaSuccess) e = set_smem_limit_nt<4>();
+  if (e == cudaSuccess) e = set_smem_limit_nt<8>();
+  if (e == cudaSuccess) e = set_smem_limit_nt<16>();
+  if (e == cudaSuccess) e = cudaFuncSetAttribute(k_pool<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, lim);
+  if (e == cudaSuccess) e = cudaFuncSetAttribute(k_pool<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, lim);
   return e;
 }
 
@@ -362,23 +219,48 @@ PoolPlan pool_plan(uint32_t B, uint32_t n, uint32_t d, bool bf16, int sm_count) 
   P.L = (uint32_t)((rows + grid - 1) / grid);
   P.grid = (uint32_t)((rows + P.L - 1) / P.L);
   P.Jmax = (P.L + n - 1) / n + 1;
-  P.smem = (size_t)P.stages * stage_bytes + (size_t)P.R * d * sizeof(float) + 16 * P.stages + 16;
+  P.smem = (size_t)SMEM_HEAD + (size_t)P.stages * stage_bytes + (size_t)P.R * d * sizeof(float);
   return P;
+}
+
+static PoolShape pool_shape(const PoolPlan& P, uint32_t B, uint32_t n, uint32_t d) {
+  return PoolShape{B, n, d, P.V, P.R, P.L, P.Jmax, P.stage_rows, P.stages, P.cons_threads};
 }
 
 static cudaError_t launch_pool(const PoolPlan& P, bool bf16, const void* h_in, float* partial, uint32_t* status,
                                uint32_t B, uint32_t n, uint32_t d, cudaStream_t st) {
   return launch_k(bf16 ? k_pool<true> : k_pool<false>, dim3(P.grid), dim3(P.threads), P.smem, st,
-                  (const uint4*)h_in, partial, status, B, n, d, P.V, P.R, P.L, P.Jmax, P.stage_rows, P.stages,
-                  P.cons_threads);
+                  (const uint4*)h_in, partial, status, pool_shape(P, B, n, d));
 }
 
-static cudaError_t launch_project(const PoolPlan& P, const float* partial, const __nv_bfloat16* proj,
-                                  const float* center, __nv_bfloat16* fp, float* rq,
-                                  uint32_t B, uint32_t n, uint32_t d, uint32_t k, cudaStream_t st) {
-  return launch_k(k_project, dim3((B + PROJ_G - 1) / PROJ_G), dim3(PROJ_THREADS),
-                  project_smem_bytes(d, k, proj != nullptr), st, partial, proj, center, fp, rq, B, n, d, k, P.L, P.Jmax,
-                  (const float*)nullptr, 0u);
+// Second kernel of the fingerprint: from the pooling pass's partial sums (pooled == nullptr) or from given
+// position means.  L, Jmax: shape of the pooling pass that wrote `partial`.
+static cudaError_t launch_project(uint32_t L, uint32_t Jmax, const float* partial, const float* pooled, uint32_t ld,
+                                  const __nv_bfloat16* proj, const float* center, __nv_bfloat16* fp, float* rq,
+                                  uint32_t* status, uint32_t B, uint32_t n, uint32_t d, uint32_t k, int sm_count,
+                                  cudaStream_t st) {
+  const MeanSrc src{partial, pooled, center, ld, n, d, L, Jmax};
+  if (!proj)
+    return launch_k(k_normalise, dim3(B), dim3(NRM_THREADS), (size_t)d * sizeof(float) + 128, st, src, fp, rq);
+  const ProjPlan P = proj_plan(B, d, k, (uint32_t)sm_count);
+  alignas(64) CUtensorMap map_p;
+  if (!make_tensor_map_bf16(&map_p, proj, d, k, P.shape.stage_rows)) return cudaErrorInvalidValue;
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = dim3(P.groups * P.split);
+  cfg.blockDim = dim3(PROJ_THREADS);
+  cfg.dynamicSmemBytes = P.smem;
+  cfg.stream = st;
+  cudaLaunchAttribute attr[2];
+  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[0].val.programmaticStreamSerializationAllowed = 1;
+  attr[1].id = cudaLaunchAttributeClusterDimension;
+  attr[1].val.clusterDim.x = P.split;
+  attr[1].val.clusterDim.y = 1;
+  attr[1].val.clusterDim.z = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = 2;
+  auto kern = P.NT == 1 ? k_project<1> : P.NT == 2 ? k_project<2> : P.NT == 4 ? k_project<4> : P.NT == 8 ? k_project<8> : k_project<16>;
+  return cudaLaunchKernelEx(&cfg, kern, map_p, src, fp, rq, status, B, P.shape, P.rows_per);
 }
 
 cudaError_t launch_fingerprint(llmcache_bank* bk, const void* h_in, uint32_t B,
@@ -394,7 +276,8 @@ cudaError_t launch_fingerprint(llmcache_bank* bk, const void* h_in, uint32_t B,
   }
   if (e != cudaSuccess) return e;
   ProfScope prof(bk, LLMCACHE_K_PROJECT, st);
-  return launch_project(P, bk->a.pool_partial, bk->a.proj, bk->a.center, fp, rq, B, D.seq_len, D.d_model, D.fp_dim, st);
+  return launch_project(P.L, P.Jmax, bk->a.pool_partial, nullptr, 0, bk->a.proj, bk->a.center, fp, rq, bk->a.status, B,
+                        D.seq_len, D.d_model, D.fp_dim, bk->sm_count, st);
 }
 
 // Step 1a alone: position means of h_in -> pooled[b * ld + c].
@@ -418,10 +301,8 @@ cudaError_t launch_fingerprint_pooled(llmcache_bank* bk, const float* pooled, ui
   if (B == 0) return cudaSuccess;
   const llmcache_bank_desc& D = bk->desc;
   ProfScope prof(bk, LLMCACHE_K_PROJECT, st);
-  return launch_k(k_project, dim3((B + PROJ_G - 1) / PROJ_G), dim3(PROJ_THREADS),
-                  project_smem_bytes(D.d_model, D.fp_dim, bk->a.proj != nullptr), st, (const float*)nullptr,
-                  (const __nv_bfloat16*)bk->a.proj, (const float*)bk->a.center, fp, rq, B, D.seq_len, D.d_model,
-                  D.fp_dim, 1u, 1u, pooled, ld);
+  return launch_project(1, 1, nullptr, pooled, ld, bk->a.proj, bk->a.center, fp, rq, bk->a.status, B, D.seq_len,
+                        D.d_model, D.fp_dim, bk->sm_count, st);
 }
 
 cudaError_t launch_rownorm(llmcache_bank* bk, const __nv_bfloat16* fp, uint32_t B, uint32_t k, float* rq, cudaStream_t st) {
@@ -523,7 +404,8 @@ extern "C" int llmcache_fingerprint_static(const void* h_in, uint32_t hidden_dty
   // nothing in the shared array has to start at zero
   e = launch_pool(P, bf16, h_in, sd->scratch, sd->status, B, n, d, st);
   if (e == cudaSuccess)
-    e = launch_project(P, sd->scratch, (const __nv_bfloat16*)proj, center, (__nv_bfloat16*)fp, rq, B, n, d, k, st);
+    e = launch_project(P.L, P.Jmax, sd->scratch, nullptr, 0, (const __nv_bfloat16*)proj, center, (__nv_bfloat16*)fp, rq,
+                       sd->status, B, n, d, k, sd->sm_count, st);
   if (e != cudaSuccess) return fail(LLMCACHE_ERR_CUDA, cudaGetErrorString(e));
   return LLMCACHE_OK;
 }

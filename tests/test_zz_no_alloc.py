@@ -31,11 +31,11 @@ def _both(bank, h, dtype_code, n, d, k, proj, center):
     L.llmcache_fingerprint(bank.handle, h, B, fp_a, rq_a)
     L.llmcache_fingerprint_static(h, dtype_code, B, n, d, k, proj, center, fp_b, rq_b)
     torch.cuda.synchronize()
-    # same tolerance as the parity tests use for fingerprints (1e-3 relative over the vector,
-    # one bf16 rounding step per element); the two paths run the same kernels, so they also agree exactly
-    U.compare_fingerprints(U.bits(fp_b), rq_b.cpu().numpy(), U.bits(fp_a), rq_a.cpu().numpy())
-    assert torch.equal(fp_a.view(torch.int16), fp_b.view(torch.int16))
-    assert torch.equal(rq_a, rq_b)
+    # same tolerance as the parity tests use for fingerprints (1e-3 relative over the vector, one bf16
+    # rounding step per element): the two entry points add the same fp32 terms, but not in the same order
+    # (the bank's runs as one persistent kernel, this one as two kernels that split the projection's rows)
+    flipped = U.compare_fingerprints(U.bits(fp_b), rq_b.cpu().numpy(), U.bits(fp_a), rq_a.cpu().numpy())
+    assert flipped < 0.01
 
 
 @pytest.mark.parametrize("dtype,n,d,k,use_proj", [("bf16", 384, 768, 256, True), ("f32", 128, 768, 768, False)])
