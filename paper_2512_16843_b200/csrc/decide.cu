@@ -41,6 +41,8 @@ k_decide_compact(unsigned long long* __restrict__ best, const float* __restrict_
   griddep_sync();
   __shared__ uint32_t warp_tot[32];
   uint32_t hbase = 0, mbase = 0, ndegen = 0;
+  const uint32_t n_chunks = (B + DEC_THREADS - 1) / DEC_THREADS;
+  int32_t my_slot = -1;                                  // this thread's slot when the batch fits one chunk
   for (uint32_t base = 0; base < B; base += DEC_THREADS) {
     const uint32_t b = base + threadIdx.x;
     bool is_hit = false, in_range = b < B;
@@ -71,6 +73,7 @@ k_decide_compact(unsigned long long* __restrict__ best, const float* __restrict_
       hit[b] = is_hit ? 1 : 0;
       slot[b] = sl;
       score[b] = sc;
+      my_slot = sl;
       if (is_hit) atomicAdd(hitcnt + sl, 1u);
     }
     uint32_t nh;
@@ -86,20 +89,22 @@ k_decide_compact(unsigned long long* __restrict__ best, const float* __restrict_
   // Metadata refresh of matched slots (Sec. III-E / IV-D).  All matches of the batch are counted by
   // now; for each matched slot exactly one thread (the one whose exchange returns the count) applies
   // "one decay step, + 256 per match", so the result does not depend on the order of the batch, and
-  // the counter is back at zero for the next probe.
+  // the counter is back at zero for the next probe.  The slot's metadata is fetched next to the
+  // exchange, not after it.
   __syncthreads();
   for (uint32_t base = 0; base < B; base += DEC_THREADS) {
     const uint32_t b = base + threadIdx.x;
     if (b >= B) continue;
-    const int32_t j = slot[b];
+    const int32_t j = n_chunks == 1 ? my_slot : slot[b];
     if (j < 0) continue;
     const uint32_t c = atomicExch(hitcnt + j, 0u);
+    const uint32_t old_rate = rate[j], old_epoch = rate_epoch[j], old_hits = hits_total[j];
     if (c == 0) continue;
-    const unsigned long long m = (unsigned long long)rate_now(rate[j], rate_epoch[j], epoch) + (unsigned long long)HIT_Q8 * c;
+    const unsigned long long m = (unsigned long long)rate_now(old_rate, old_epoch, epoch) + (unsigned long long)HIT_Q8 * c;
     rate[j] = m > M_CAP ? M_CAP : (uint32_t)m;
     rate_epoch[j] = epoch;
     last_use[j] = tick;
-    const unsigned long long h = (unsigned long long)hits_total[j] + c;
+    const unsigned long long h = (unsigned long long)old_hits + c;
     hits_total[j] = h > 0xFFFFFFFFull ? 0xFFFFFFFFu : (uint32_t)h;
   }
   // degenerate count: block reduction by atomics on shared memory
