@@ -164,7 +164,7 @@ __device__ __forceinline__ void pool_phase(uint8_t* sm, const uint4* __restrict_
 // ---------------------------------------------------------------------------
 // Position means of sequence bq, column i, centred: either given (pooled) or the sum of the pooling
 // pass's partial vectors of the blocks whose span overlaps rows [bq*n, (bq+1)*n), in block order.
-// The partial sums may have been written by other blocks of the same grid: they are read past L1.
+// The sums were written by the grid before this one; they are read past L1.
 // ---------------------------------------------------------------------------
 struct MeanSrc { const float* partial; const float* pooled; const float* center; uint32_t ld, n, d, L, Jmax; };
 
@@ -201,10 +201,10 @@ __device__ __forceinline__ float centred_mean(const MeanSrc& m, const SeqBlocks&
 // carries the 8 sequences' centred means as three bf16 rows each: head in rows 0..7 and middle in rows
 // 8..15 of one mma, tail in rows 0..7 of a second mma into the same accumulator; rows g and g + 8 of the
 // accumulator are added at the end.  Nothing of the fp32 means is lost; only the order of the sums
-// differs from a plain fp32 dot product.  The item's rows of P are
-// streamed once through a ring of shared-memory stages by TMA (issued by thread PROJ_CONS): a stage is
-// k / 64 boxes of stage_rows x 64 columns with the 128-byte swizzle, so that ldmatrix finds its eight rows
-// in different banks; rows beyond the end of P arrive as zeros.  Warp w of the PROJ_CONS / 32 consumer warps owns the output columns
+// differs from a plain fp32 dot product.  The item's rows of P are streamed once through a ring of
+// shared-memory stages by TMA (issued by thread PROJ_CONS): a stage is k / 64 boxes of stage_rows x 64
+// columns with the 128-byte swizzle, so that ldmatrix finds its eight rows in different banks; rows beyond
+// the end of P arrive as zeros.  Warp w of the PROJ_CONS / 32 consumer warps owns the output columns
 // [w * NT * 8, (w + 1) * NT * 8) over all the item's rows, so nothing has to be combined across warps.
 // Shared memory after the head: ring | A [24][a_rows] bf16 (the item's rows are taken a_rows at a time).
 // The ring's memory is reused for the group's [8][k] result once the item's rows are consumed.
