@@ -352,3 +352,28 @@ def test_maximum_widths(dtype, d, k):
                    proj=synth.projection(bad, 2048, 1, DEV))
         assert e.value.status == L.ERR_SHAPE
     gb.close()
+
+
+def test_large_batch_many_queries_per_slot_lockstep():
+    """A batch that the decision kernel walks in several passes (more than 1,024 sequences), in which a few
+    stored entries are matched by hundreds of queries each: the per-slot match counts, the decayed rates and
+    the recency stamps must come out exactly as the oracle's, whichever thread applies them."""
+    N, n, d, B = 1200, 2, 64, 2500               # the 1,000 misses of a step leave the 40 hot entries in the bank
+    gb, ob = make_pair(N, n, d, d, B, "bf16", policy=L.LRU_STALENESS)
+    bufs = L.ProbeBuffers(B, d, DEV)
+    seeds = rand_h(40, n, d, 71, "bf16")
+    g = torch.Generator().manual_seed(72)
+    for step in range(3):
+        h = rand_h(B, n, d, 80 + step, "bf16")
+        if step:
+            # 60% of the batch repeats one of 40 sequences that are in the bank after the first step
+            rep = torch.randperm(B, generator=g)[: (B * 6) // 10].to(DEV)
+            pick = torch.randint(0, 40, (rep.numel(),), generator=g).to(DEV)
+            h[rep] = seeds[pick]
+        else:
+            h[:40] = seeds
+        r = U.lockstep_step(gb, ob, bufs, h, "bf16", synth.activations(B, n, d, 90 + step, DEV))
+        if step:
+            assert r["H"] >= (B * 6) // 10
+    assert int(ob.hits.max()) > 30
+    gb.close()
