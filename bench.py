@@ -1,5 +1,5 @@
 #!/usr/bin/env python
-"""Benchmark of the per-layer cache probe on the BERT-base-shaped workload.
+"""Benchmark of the per-layer cache probe on the BERT-base-shaped workload (other shapes: --workload).
 
 One step = one pass of the whole hot path over one batch at every layer: for each
 of the 12 per-layer banks, llmcache_probe (fingerprint, bank scan, threshold +
@@ -135,9 +135,10 @@ def parse():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--e2e-steps", type=int, default=3)
     ap.add_argument("--no-cpu-baseline", action="store_true")
-    ap.add_argument("--workload", default="bert_base", choices=["bert_base", "gpt2_small", "bert_large_churn", "scan_stress", "e2e_bert_base"])
+    ap.add_argument("--workload", default="bert_base", choices=["bert_base", "gpt2_small", "bert_large_churn", "scan_stress", "gather_stress", "e2e_bert_base"])
     ap.add_argument("--bank", type=int, default=65536, help="scan_stress: number of bank entries")
-    ap.add_argument("--queries", type=int, default=65536, help="scan_stress: queries per batch")
+    ap.add_argument("--queries", type=int, default=65536, help="scan_stress: queries per batch (gather_stress: 8192 per probe)")
+    ap.add_argument("--act-rows", type=int, default=16384, help="gather_stress: rows of the activation store (1 MiB each)")
     ap.add_argument("--layers", type=int, default=0, help="bert_base: number of per-layer banks (default 12; fewer only for profiler captures)")
     ap.add_argument("--pool-batches", type=int, default=0, help="bert_base: distinct input batches in rotation (default 24)")
     return ap.parse_args()
@@ -468,6 +469,92 @@ def run_scan_stress(args):
     bank.close()
 
 
+def run_gather_stress(args):
+    """Second half of the bank-scan stress configuration: the gather of hit rows of 512 x 1024 bf16 activations
+    (1 MiB each).  65,536 keys share an activation store of `--act-rows` rows (slot j uses row j mod act_rows:
+    65,536 rows of 1 MiB would be 69 GB), and the 65,536 queries are probed 8,192 at a time."""
+    from paper_2512_16843_b200 import binding as L
+    from paper_2512_16843_b200 import synth
+    L.lib()
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device (there is no CPU fallback)")
+    dev = torch.device("cuda", 0)
+    N, k, n, act_rows = 65536, 1024, 512, args.act_rows
+    Bq, chunk = 65536, 8192
+    keys, q, src = synth.scan_stress(N, Bq, k, n_clusters=4096, spread=0.1, near_fraction=0.3, q_sigma=0.05,
+                                     seed=synth.BASE_SEED + 4000, device=dev)
+    # inverse norms of the keys from the library itself (the row-norm kernel of a keys-only bank)
+    tmp = L.Bank(capacity=N, seq_len=1, d_model=k, fp_dim=k, max_batch=N, store_act=0, tau=2.0)
+    tb = L.ProbeBuffers(N, k, dev)
+    tb.fp.copy_(keys)
+    tmp.probe_fp(tb, N)
+    torch.cuda.synchronize()
+    rb = tb.rq.clone()
+    tmp.close()
+    del tb
+    bank = L.Bank(capacity=N, seq_len=n, d_model=k, fp_dim=k, max_batch=chunk, act_rows=act_rows, tau=0.9)
+    bank.import_(L.WHAT_FP, keys)
+    bank.import_(L.WHAT_RB, rb)
+    bank.import_(L.WHAT_VALID, torch.ones(N, dtype=torch.uint8))
+    act = torch.empty((act_rows, n * k), dtype=torch.bfloat16, device=dev)
+    for f in range(0, act_rows, 1024):
+        c = min(1024, act_rows - f)
+        act[f:f + c] = synth.activations(c, n, k, synth.BASE_SEED + 4200 + f, dev)
+    bank.import_(L.WHAT_ACT, act)
+    del act
+    bufs = L.ProbeBuffers(chunk, k, dev)
+    h_out = torch.empty((chunk, n * k), dtype=torch.bfloat16, device=dev)
+    chunks = [q[i:i + chunk].contiguous() for i in range(0, Bq, chunk)]
+    exp_hits = int((src >= 0).sum())
+
+    def one_step():
+        hits = 0
+        for c in chunks:
+            bufs.fp.copy_(c)
+            bank.probe_fp(bufs, chunk, h_out=h_out)
+        return hits
+
+    for _ in range(max(1, args.warmup // 3)):
+        one_step()
+    torch.cuda.synchronize()
+    steps = max(1, min(args.steps, 10))
+    sampler = ClockSampler(0)
+    sampler.start()
+    bank.profile(True)
+    h0 = bank.stats()["hits"]
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record()
+    for _ in range(steps):
+        one_step()
+    e1.record()
+    torch.cuda.synchronize()
+    clocks = sampler.stop()
+    ms = e0.elapsed_time(e1)
+    prof = bank.profile_read()
+    hits = (bank.stats()["hits"] - h0) / steps
+    g_ms = prof["gather"][0] / prof["gather"][1]
+    row = n * k * 2
+    algo = hits / len(chunks) * row * 2                  # per launch: every hit row read once and written once
+    peaks, kind = measured_peaks()
+    ach = algo / (g_ms * 1e-3) / 1e9
+    out = {"metric": METRIC, "value": Bq * steps / (ms * 1e-3), "unit": UNIT, "n_gpus": 1, "steps": steps,
+           "warmup": args.warmup, "ms_per_step": ms / steps, "higher_is_better": True, "scaling": "weak",
+           "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
+           "config": {"workload": f"bank-scan stress, gather half: {N} keys x fp_dim 1024, activation store of {act_rows} rows "
+                                  f"of 512 x 1024 bf16 (1 MiB, slot mod {act_rows}), {Bq} queries probed {chunk} at a time, "
+                                  f"30% near-duplicates, tau 0.9",
+                      "hits": int(round(hits)), "expected_hits": exp_hits,
+                      "l2": "%.1f GB of hit rows per probe call" % (algo / 2e9)},
+           "gpu_launches": sum(v[1] for v in prof.values()),
+           "roofline": {"kernel": "gather", "bound": "hbm", "achieved": ach, "peak": peaks["hbm_gbs"], "unit": "GB/s",
+                        "frac": ach / peaks["hbm_gbs"], "peak_kind": "of " + kind, "traffic": None,
+                        "ms_per_launch": g_ms, "algorithmic_bytes_per_launch": algo,
+                        "all_kernels": {n_: {"ms_per_launch": v[0] / v[1], "launches": v[1]} for n_, v in prof.items() if v[1]}},
+           "clocks": clocks}
+    print(json.dumps(out))
+    bank.close()
+
+
 def run_e2e(args):
     """End-to-end Algorithm 1 on a BERT-base-shaped random-init encoder: the same batches with and without
     the per-layer banks (the paper's NoCache vs LLMCache comparison, Table I, on synthetic data)."""
@@ -700,6 +787,8 @@ if __name__ == "__main__":
         run_reference(a)
     elif a.workload == "scan_stress":
         run_scan_stress(a)
+    elif a.workload == "gather_stress":
+        run_gather_stress(a)
     elif a.workload == "e2e_bert_base":
         run_e2e(a)
     else:
