@@ -35,42 +35,118 @@ struct MetaView {
 };
 
 // Order in which slots are taken: free slots first (key 0), then occupied slots by ascending eviction
-// key (bit 63 set, which no eviction key has); ties go to the lower slot.  All loads are issued
-// unconditionally so that they overlap.
-__device__ __forceinline__ unsigned long long take_key(const MetaView& mv, const PolicyParams& p,
-                                                       uint32_t j, uint32_t tick, uint32_t epoch) {
-  const uint8_t v = mv.valid[j];
-  const uint32_t r = mv.rate[j], re = mv.rate_epoch[j], it = mv.insert_tick[j], lu = mv.last_use[j];
-  return v ? (evict_key(p, tick, epoch, r, re, it, lu) | (1ull << 63)) : 0ull;
+// key (bit 63 set, which no eviction key has); ties go to the lower slot.
+// Keys of SEL_U consecutive slots starting at j0 (slots >= N: all ones, which sorts after every real key).
+// All loads are issued before the first key is formed, so that a thread has them in flight together.
+constexpr int SEL_U = 8;
+__device__ __forceinline__ void take_keys(const MetaView& mv, const PolicyParams& p, uint32_t j0, uint32_t N,
+                                          uint32_t tick, uint32_t epoch, unsigned long long (&key)[SEL_U]) {
+  uint8_t v[SEL_U];
+  uint32_t r[SEL_U], re[SEL_U], it[SEL_U], lu[SEL_U];
+#pragma unroll
+  for (int u = 0; u < SEL_U; ++u) {
+    const uint32_t j = min(j0 + u, N - 1);
+    v[u] = mv.valid[j]; r[u] = mv.rate[j]; re[u] = mv.rate_epoch[j]; it[u] = mv.insert_tick[j]; lu[u] = mv.last_use[j];
+  }
+#pragma unroll
+  for (int u = 0; u < SEL_U; ++u)
+    key[u] = j0 + u >= N ? ~0ull : (v[u] ? (evict_key(p, tick, epoch, r[u], re[u], it[u], lu[u]) | (1ull << 63)) : 0ull);
+}
+
+// Exclusive prefix sum of `v` over the threads of the block (in thread order) and the block total.
+__device__ __forceinline__ uint32_t sel_scan(uint32_t v, uint32_t* warp_tot, uint32_t& total) {
+  const uint32_t lane = threadIdx.x & 31, w = threadIdx.x >> 5;
+  uint32_t incl = v;
+#pragma unroll
+  for (int o = 1; o < 32; o <<= 1) {
+    const uint32_t t = __shfl_up_sync(0xFFFFFFFFu, incl, o);
+    if (lane >= (uint32_t)o) incl += t;
+  }
+  __syncthreads();
+  if (lane == 31) warp_tot[w] = incl;
+  __syncthreads();
+  uint32_t before = 0, tot = 0;
+#pragma unroll
+  for (uint32_t i = 0; i < (SEL_THREADS >> 5); ++i) {
+    const uint32_t c = warp_tot[i];
+    if (i < w) before += c;
+    tot += c;
+  }
+  total = tot;
+  return before + incl - v;
 }
 
 // In-place bitonic sort of (key, slot) pairs, ascending by key then slot.  len is a power of two;
 // the arrays may live in shared or global memory.  Thread t handles the pair (i, i + stride) with
 // i = (t / stride) * 2 * stride + t % stride, so for stride <= 32 a warp only touches elements that
 // no other warp touches in that step and a warp-level sync is enough.
+__device__ __forceinline__ void bitonic_steps(unsigned long long* key, uint32_t* val, uint32_t len, uint32_t g0,
+                                              uint32_t size, uint32_t first_stride) {
+  // the steps of merge size `size` with strides first_stride, first_stride / 2, ..., 1 on `len` elements whose
+  // first one has index g0 in the whole sequence (the direction of a pair depends on that index)
+  for (uint32_t stride = first_stride, lg = 31 - __clz(stride);; stride >>= 1, --lg) {
+    for (uint32_t t = threadIdx.x; t < (len >> 1); t += SEL_THREADS) {
+      const uint32_t i = ((t >> lg) << (lg + 1)) | (t & (stride - 1)), l = i + stride;
+      const unsigned long long ka = key[i], kb = key[l];
+      const uint32_t va = val[i], vb = val[l];
+      const bool a_gt_b = (ka > kb) || (ka == kb && va > vb);
+      const bool ascending = ((g0 + i) & size) == 0;
+      if (a_gt_b == ascending) {
+        key[i] = kb; key[l] = ka;
+        val[i] = vb; val[l] = va;
+      }
+    }
+    // a step with stride <= 32 stays inside the warp's own 64 elements; a block-level sync is only
+    // needed when this step or the next one reaches further
+    const uint32_t next = stride > 1 ? (stride >> 1) : size;
+    if (stride > 32 || next > 32) __syncthreads(); else __syncwarp();
+    if (stride == 1) break;
+  }
+}
+
 __device__ __forceinline__ void bitonic_sort(unsigned long long* key, uint32_t* val, uint32_t len) {
   __syncthreads();
-  for (uint32_t size = 2; size <= len; size <<= 1) {
-    for (uint32_t stride = size >> 1, lg = 31 - __clz(stride);; stride >>= 1, --lg) {
+  for (uint32_t size = 2; size <= len; size <<= 1) bitonic_steps(key, val, len, 0, size, size >> 1);
+  __syncthreads();
+}
+
+// The same sort for a sequence in global memory that is longer than the shared-memory buffers (cap elements,
+// a power of two; len a larger power of two).  Every step whose stride is below cap stays inside aligned
+// pieces of cap elements, so those steps run on one piece at a time in shared memory; only the steps with
+// strides of cap and more (log2(len / cap) * (log2(len / cap) + 1) / 2 of them) work on global memory.
+__device__ __forceinline__ void bitonic_sort_large(unsigned long long* gkey, uint32_t* gval, uint32_t len,
+                                                   unsigned long long* skey, uint32_t* sval, uint32_t cap) {
+  __syncthreads();
+  auto pieces = [&](uint32_t size_lo, uint32_t size_hi) {
+    // on every piece: the steps with strides < cap of the merge sizes size_lo .. size_hi
+    for (uint32_t g0 = 0; g0 < len; g0 += cap) {
+      for (uint32_t i = threadIdx.x; i < cap; i += SEL_THREADS) { skey[i] = gkey[g0 + i]; sval[i] = gval[g0 + i]; }
+      __syncthreads();
+      for (uint32_t size = size_lo; size <= size_hi; size <<= 1)
+        bitonic_steps(skey, sval, cap, g0, size, min(size >> 1, cap >> 1));
+      __syncthreads();
+      for (uint32_t i = threadIdx.x; i < cap; i += SEL_THREADS) { gkey[g0 + i] = skey[i]; gval[g0 + i] = sval[i]; }
+      __syncthreads();
+    }
+  };
+  pieces(2, cap);                                                    // sorted pieces, directions alternating
+  for (uint32_t size = cap << 1; size <= len; size <<= 1) {
+    for (uint32_t stride = size >> 1, lg = 31 - __clz(stride); stride >= cap; stride >>= 1, --lg) {
       for (uint32_t t = threadIdx.x; t < (len >> 1); t += SEL_THREADS) {
         const uint32_t i = ((t >> lg) << (lg + 1)) | (t & (stride - 1)), l = i + stride;
-        const unsigned long long ka = key[i], kb = key[l];
-        const uint32_t va = val[i], vb = val[l];
+        const unsigned long long ka = gkey[i], kb = gkey[l];
+        const uint32_t va = gval[i], vb = gval[l];
         const bool a_gt_b = (ka > kb) || (ka == kb && va > vb);
         const bool ascending = (i & size) == 0;
         if (a_gt_b == ascending) {
-          key[i] = kb; key[l] = ka;
-          val[i] = vb; val[l] = va;
+          gkey[i] = kb; gkey[l] = ka;
+          gval[i] = vb; gval[l] = va;
         }
       }
-      // a step with stride <= 32 stays inside the warp's own 64 elements; a block-level sync is only
-      // needed when this step or the next one reaches further
-      const uint32_t next = stride > 1 ? (stride >> 1) : size;
-      if (stride > 32 || next > 32) __syncthreads(); else __syncwarp();
-      if (stride == 1) break;
+      __syncthreads();
     }
+    pieces(size, size);
   }
-  __syncthreads();
 }
 
 // One block.  Output: new_slot[m] for every miss m (in miss order): the slot it is stored in, or -1
@@ -115,8 +191,13 @@ __device__ __forceinline__ void select_victims_block(const SelectArgs& A) {
 
   const uint32_t M = counts[1];
   const bool cached = N <= SEL_SMEM;
-  auto key_at = [&](uint32_t j) -> unsigned long long {
-    return cached ? s_cache[j] : take_key(mv, pol, j, tick, epoch);
+  auto keys_at = [&](uint32_t j0, unsigned long long (&key)[SEL_U]) {
+    if (cached) {
+#pragma unroll
+      for (int u = 0; u < SEL_U; ++u) key[u] = j0 + u < N ? s_cache[j0 + u] : ~0ull;
+    } else {
+      take_keys(mv, pol, j0, N, tick, epoch, key);
+    }
   };
   if (threadIdx.x == 0) { s_and = ~0ull; s_or = 0ull; s_evict = 0; }
   __syncthreads();
@@ -124,10 +205,18 @@ __device__ __forceinline__ void select_victims_block(const SelectArgs& A) {
   // keys of all slots; bitwise AND / OR over them tells which bytes differ at all
   {
     unsigned long long a = ~0ull, o = 0ull;
-    for (uint32_t j = threadIdx.x; j < N; j += SEL_THREADS) {
-      const unsigned long long key = take_key(mv, pol, j, tick, epoch);
-      if (cached) s_cache[j] = key;
-      a &= key; o |= key;
+    for (uint32_t base = 0; base < N; base += SEL_THREADS * SEL_U) {
+      const uint32_t j0 = base + threadIdx.x * SEL_U;
+      if (j0 >= N) break;
+      unsigned long long key[SEL_U];
+      take_keys(mv, pol, j0, N, tick, epoch, key);
+#pragma unroll
+      for (int u = 0; u < SEL_U; ++u) {
+        if (j0 + u < N) {
+          if (cached) s_cache[j0 + u] = key[u];
+          a &= key[u]; o |= key[u];
+        }
+      }
     }
 #pragma unroll
     for (int off = 16; off > 0; off >>= 1) {
@@ -159,9 +248,14 @@ __device__ __forceinline__ void select_victims_block(const SelectArgs& A) {
       for (uint32_t i = threadIdx.x; i < 256; i += SEL_THREADS) hist[i] = 0;
       __syncthreads();
       const unsigned long long hi_mask = shift == 56 ? 0ull : (~0ull << (shift + 8));
-      for (uint32_t j = threadIdx.x; j < N; j += SEL_THREADS) {
-        const unsigned long long key = key_at(j);
-        if ((key & hi_mask) == prefix) atomicAdd(&hist[(uint32_t)(key >> shift) & 255u], 1u);
+      for (uint32_t base = 0; base < N; base += SEL_THREADS * SEL_U) {
+        const uint32_t j0 = base + threadIdx.x * SEL_U;
+        if (j0 >= N) break;
+        unsigned long long key[SEL_U];
+        keys_at(j0, key);
+#pragma unroll
+        for (int u = 0; u < SEL_U; ++u)
+          if (j0 + u < N && (key[u] & hi_mask) == prefix) atomicAdd(&hist[(uint32_t)(key[u] >> shift) & 255u], 1u);
       }
       __syncthreads();
       if (threadIdx.x < 32) {
@@ -201,19 +295,40 @@ __device__ __forceinline__ void select_victims_block(const SelectArgs& A) {
     uint32_t* sval = in_smem ? s_val : g_val;
     if (!in_smem && pow2 > sort_cap) pow2 = sort_cap;   // cannot happen: sort_cap >= pow2(min(B, N))
     uint32_t n_eq_seen = 0, n_out = 0, n_occ = 0;
-    for (uint32_t base = 0; base < N; base += SEL_THREADS) {
-      const uint32_t j = base + threadIdx.x;
-      const unsigned long long key = j < N ? key_at(j) : ~0ull;
-      const bool eq = j < N && key == T;
+    for (uint32_t base = 0; base < N; base += SEL_THREADS * SEL_U) {
+      // every thread takes SEL_U consecutive slots, so thread order is slot order
+      const uint32_t j0 = base + threadIdx.x * SEL_U;
+      unsigned long long key[SEL_U];
+      if (j0 < N) {
+        keys_at(j0, key);
+      } else {
+#pragma unroll
+        for (int u = 0; u < SEL_U; ++u) key[u] = ~0ull;
+      }
+      uint32_t c_eq = 0;
+#pragma unroll
+      for (int u = 0; u < SEL_U; ++u) c_eq += (j0 + u < N && key[u] == T) ? 1u : 0u;
       uint32_t tot_eq;
-      const uint32_t r_eq = sel_rank(eq, warp_tot, tot_eq);
-      const bool chosen = j < N && (key < T || (eq && n_eq_seen + r_eq < need));
+      uint32_t eq_before = n_eq_seen + sel_scan(c_eq, warp_tot, tot_eq);
+      uint32_t chosen = 0, c_ch = 0;                                 // bit u: slot j0 + u is taken
+#pragma unroll
+      for (int u = 0; u < SEL_U; ++u) {
+        const bool in = j0 + u < N, eq = in && key[u] == T;
+        if (in && (key[u] < T || (eq && eq_before < need))) { chosen |= 1u << u; ++c_ch; }
+        if (eq) ++eq_before;
+      }
       uint32_t tot_ch;
-      const uint32_t r_ch = sel_rank(chosen, warp_tot, tot_ch);
-      if (chosen && n_out + r_ch < pow2) {
-        skey[n_out + r_ch] = key;
-        sval[n_out + r_ch] = j;
-        if (key >> 63) ++n_occ;
+      uint32_t pos = n_out + sel_scan(c_ch, warp_tot, tot_ch);
+#pragma unroll
+      for (int u = 0; u < SEL_U; ++u) {
+        if (chosen & (1u << u)) {
+          if (pos < pow2) {
+            skey[pos] = key[u];
+            sval[pos] = j0 + u;
+            if (key[u] >> 63) ++n_occ;
+          }
+          ++pos;
+        }
       }
       n_eq_seen += tot_eq;
       n_out += tot_ch;
@@ -223,7 +338,8 @@ __device__ __forceinline__ void select_victims_block(const SelectArgs& A) {
       skey[i] = ~0ull;
       sval[i] = 0xFFFFFFFFu;
     }
-    bitonic_sort(skey, sval, pow2);
+    if (in_smem) bitonic_sort(skey, sval, pow2);
+    else         bitonic_sort_large(skey, sval, pow2, s_key, s_val, SEL_SMEM);
     for (uint32_t i = threadIdx.x; i < take; i += SEL_THREADS) victims[i] = (int32_t)sval[i];
   }
   __syncthreads();

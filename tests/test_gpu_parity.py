@@ -377,3 +377,21 @@ def test_large_batch_many_queries_per_slot_lockstep():
             assert r["H"] >= (B * 6) // 10
     assert int(ob.hits.max()) > 30
     gb.close()
+
+
+@pytest.mark.parametrize("policy", [L.LRU, L.LRU_STALENESS])
+def test_more_victims_than_the_shared_memory_sort_holds(policy):
+    """Thousands of misses at once into a bank of thousands of slots: the chosen slots are sorted in pieces in
+    shared memory and merged through global memory; which miss gets which slot must still be the oracle's."""
+    N, n, d, B = 8000, 1, 64, 6000              # 6,000 inserts fill free slots first; later steps also evict thousands
+    gb, ob = make_pair(N, n, d, d, B, "bf16", policy=policy)
+    bufs = L.ProbeBuffers(B, d, DEV)
+    keep = rand_h(700, n, d, 171, "bf16")
+    for step in range(3):
+        h = rand_h(B, n, d, 180 + step, "bf16")
+        h[100:800] = keep                          # 700 sequences come back every step: their entries are hit and survive
+        r = U.lockstep_step(gb, ob, bufs, h, "bf16", synth.activations(B, n, d, 190 + step, DEV))
+        assert r["inserted"] == r["M"] > 2048
+        if step:
+            assert r["H"] >= 700
+    gb.close()
