@@ -38,7 +38,7 @@ struct MetaView {
 // key (bit 63 set, which no eviction key has); ties go to the lower slot.
 // Keys of SEL_U consecutive slots starting at j0 (slots >= N: all ones, which sorts after every real key).
 // All loads are issued before the first key is formed, so that a thread has them in flight together.
-constexpr int SEL_U = 8;
+constexpr int SEL_U = 4;
 __device__ __forceinline__ void take_keys(const MetaView& mv, const PolicyParams& p, uint32_t j0, uint32_t N,
                                           uint32_t tick, uint32_t epoch, unsigned long long (&key)[SEL_U]) {
   uint8_t v[SEL_U];
