@@ -139,6 +139,8 @@ def parse():
     ap.add_argument("--bank", type=int, default=65536, help="scan_stress: number of bank entries")
     ap.add_argument("--queries", type=int, default=65536, help="scan_stress: queries per batch (gather_stress: 8192 per probe)")
     ap.add_argument("--act-rows", type=int, default=16384, help="gather_stress: rows of the activation store (1 MiB each)")
+    ap.add_argument("--batch", type=int, default=0, help="e2e_bert_base: sequences per batch (default 256)")
+    ap.add_argument("--seq-len", type=int, default=0, help="e2e_bert_base: sequence length (default 384)")
     ap.add_argument("--layers", type=int, default=0, help="bert_base: number of per-layer banks (default 12; fewer only for profiler captures)")
     ap.add_argument("--pool-batches", type=int, default=0, help="bert_base: distinct input batches in rotation (default 24)")
     return ap.parse_args()
@@ -222,13 +224,17 @@ def aggregate(ms_local, seqs_local, dist=None, device="cpu"):
     return ms, seqs, seqs / (ms * 1e-3)
 
 
-def build_batches(wl, seeds_tok, count, seed, device):
-    """`count` batches of hidden states: 60% edits of the seeds, 40% fresh, shuffled."""
+def build_batches(wl, seeds_tok, count, seed, device, B=None):
+    """`count` batches of hidden states: 60% edits of the seeds, 40% fresh, shuffled.  A batch too small to be
+    split 60/40 is, as a whole, an edit or fresh with those probabilities (seeded)."""
     from paper_2512_16843_b200 import synth
-    B = CFG["batch"]
+    B = B or CFG["batch"]
     n_edit = int(round(B * CFG["edit_fraction"]))
+    g = torch.Generator().manual_seed(seed + 77)
     out = []
     for i in range(count):
+        if B < 8:
+            n_edit = int((torch.rand(B, generator=g) < CFG["edit_fraction"]).sum())
         ed, _ = wl.edited(seeds_tok, n_edit, CFG["edit_positions"], seed + 10 * i + 1)
         fr = wl.tokens(B - n_edit, seed + 10 * i + 2)
         tok = torch.cat([ed, fr])[synth.shuffled(B, seed + 10 * i + 3, device)]
@@ -566,28 +572,30 @@ def run_e2e(args):
     dev = torch.device("cuda", 0)
     Lyr = args.layers or CFG["layers"]
     d, n, B, N, k = (CFG[x] for x in ("d_model", "seq_len", "batch", "bank", "fp_dim"))
+    B, n = args.batch or B, args.seq_len or n          # e.g. --batch 1 --seq-len 128: the setting the paper measures in
     heads, ffn = 12, 3072
     seed = synth.BASE_SEED + 6000
     wl = synth.TokenWorkload(CFG["vocab"], n, d, seed, dev)
     seeds_tok = wl.tokens(CFG["n_seeds"], seed + 5)
     proj = synth.projection(d, k, seed + 6, dev)
     ws = [synth.layer_weights(d, ffn, seed + 100 * (l + 1), dev) for l in range(Lyr)]
-    probe = L.Layer(ws[0], heads=heads, seq_len=n, max_seqs=B)
+    CAL = 64                                           # sequences of the calibration batch
+    probe = L.Layer(ws[0], heads=heads, seq_len=n, max_seqs=max(B, CAL))
     need = L.llmcache_layer_bytes(probe.desc)
     probe.close()
     workspace = torch.empty(need + 256, dtype=torch.uint8, device=dev)
     off = (-workspace.data_ptr()) % 256
-    layers = [L.Layer(w, heads=heads, seq_len=n, max_seqs=B, workspace=workspace[off:]) for w in ws]
-    mk = lambda: torch.empty((B, n, d), dtype=torch.bfloat16, device=dev)
+    layers = [L.Layer(w, heads=heads, seq_len=n, max_seqs=max(B, CAL), workspace=workspace[off:]) for w in ws]
+    mk = lambda: torch.empty((max(B, CAL), n, d), dtype=torch.bfloat16, device=dev)
     buf_a, buf_b, h_miss, miss_out = mk(), mk(), mk(), mk()
     # centring vectors (an input of the library): mean pooled layer input of a seeded calibration batch;
     # without them the pooled outputs of random-init layers are all alike and every sequence would match
     tau = 0.85
-    centers, h = [], wl.hidden(wl.tokens(64, seed + 9))
+    centers, h = [], wl.hidden(wl.tokens(CAL, seed + 9))
     for l in range(Lyr):
         centers.append(h.float().mean(dim=(0, 1)).contiguous())
-        layers[l].forward(h, buf_a[:64])
-        h = buf_a[:64].clone()
+        layers[l].forward(h, buf_a[:CAL])
+        h = buf_a[:CAL].clone()
     mkbanks = lambda fused: [L.Bank(capacity=N, seq_len=n, d_model=d, fp_dim=k, max_batch=B, hidden_dtype=L.BF16,
                                     proj=proj, center=centers[l], tau=tau, fused_pool=fused) for l in range(Lyr)]
     banks = mkbanks(0)
@@ -597,9 +605,11 @@ def run_e2e(args):
     hb, hbf, hl = [b.handle for b in banks], [b.handle for b in banks_f], [l.handle for l in layers]
     # enough distinct batches that none comes round again within an arm (a repeated batch would hit in full)
     P = args.pool_batches or min(160, args.warmup + args.steps + 10)
-    pool = build_batches(wl, seeds_tok, P, seed + 1000, dev)
-    warm = [wl.hidden(torch.cat([seeds_tok, wl.tokens(B - CFG["n_seeds"], seed + 7)]))]
-    warm += [wl.hidden(wl.tokens(B, seed + 20 + i)) for i in range(1, N // B)]
+    pool = build_batches(wl, seeds_tok, P, seed + 1000, dev, B)
+    # the banks are filled with fresh sequences and then the seeds (so that these are not the first to be evicted),
+    # B at a time
+    warm_tok = torch.cat([wl.tokens(N - CFG["n_seeds"], seed + 7), seeds_tok])
+    warm = [wl.hidden(warm_tok[i:i + B]) for i in range(0, N - B + 1, B)]
 
     def infer(h, cached):
         if cached == 2:
