@@ -78,3 +78,37 @@ def test_no_cpu_fallback_without_a_device():
     with pytest.raises(L.LLMCacheError) as e:
         L.llmcache_bank_create(L.make_desc(capacity=16, seq_len=8, d_model=64, fp_dim=64, max_batch=4))
     assert e.value.status == L.ERR_CUDA
+
+
+def test_header_is_plain_c(tmp_path):
+    """The boundary is a C ABI: the header must compile as C99 on its own, and a C program must link against the
+    library using nothing but that header."""
+    import shutil
+    import subprocess
+    gcc = shutil.which("gcc")
+    if gcc is None:
+        pytest.skip("no C compiler")
+    root = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+    src = tmp_path / "use_header.c"
+    src.write_text(
+        '#include "llmcache.h"\n'
+        "#include <stdio.h>\n"
+        "int main(void) {\n"
+        "  llmcache_bank_desc d = {0};\n"
+        "  size_t bytes = 0;\n"
+        "  d.struct_size = (uint32_t)sizeof d; d.capacity = 4; d.seq_len = 2; d.d_model = 64; d.fp_dim = 64;\n"
+        "  d.max_batch = 2; d.hidden_dtype = LLMCACHE_BF16; d.store_act = 1; d.tau = 0.9f;\n"
+        "  if (llmcache_abi_version() != LLMCACHE_ABI_VERSION) return 2;\n"
+        "  if (llmcache_bank_bytes(&d, &bytes) != LLMCACHE_OK || bytes == 0) return 3;\n"
+        '  printf("%s %zu\\n", llmcache_strerror(LLMCACHE_ERR_SHAPE), bytes);\n'
+        "  return 0;\n"
+        "}\n")
+    exe = tmp_path / "use_header"
+    lib_dir = os.path.dirname(L.LIB_PATH)
+    r = subprocess.run([gcc, "-std=c99", "-Wall", "-Werror", "-pedantic", "-I", os.path.join(root, "include"), str(src),
+                        "-o", str(exe), "-L", lib_dir, "-l:libllmcache.so", "-Wl,-rpath," + lib_dir],
+                       capture_output=True, text=True)
+    assert r.returncode == 0, r.stderr
+    r = subprocess.run([str(exe)], capture_output=True, text=True)
+    assert r.returncode == 0, (r.returncode, r.stdout, r.stderr)
+    assert "shape" in r.stdout
