@@ -17,7 +17,7 @@ inline uint32_t pow2_ceil(uint32_t x) { uint32_t p = 1; while (p < x) p <<= 1; r
 
 struct Layout {
   size_t fp, rb, valid, last_use, insert_tick, hits, rate, rate_epoch, act, proj, center;
-  size_t pool_partial, move_partial, best, hitcnt, victims, new_slot, bits, qbits, sort_key, sort_slot, stats, status, misc, total;
+  size_t pool_partial, move_partial, best, hitcnt, victims, new_slot, bits, qbits, sort_key, sort_slot, stats, status, misc, blk_cnt, sel_keys, sel_state, sel_blk, sel_mcnt, total;
   uint32_t sort_len;
 };
 
@@ -86,6 +86,11 @@ Layout make_layout(const llmcache_bank_desc& d) {
   L.stats = take(ST_COUNT * 8);
   L.status = take(4);
   L.misc = take(64);
+  L.blk_cnt = take(((size_t)d.max_batch + 1023) / 1024 * 8);
+  L.sel_keys = take(N * 8);
+  L.sel_state = take((size_t)SEL_STATE_WORDS * 4);
+  L.sel_blk = take((N + 1023) / 1024 * 8);
+  L.sel_mcnt = take(((size_t)d.max_batch + 1023) / 1024 * 4);
   L.total = o;
   return L;
 }
@@ -223,6 +228,11 @@ int llmcache_bank_create(const llmcache_bank_desc* desc, llmcache_bank_t** bank_
   a.stats = (unsigned long long*)(base + L.stats);
   a.status = (uint32_t*)(base + L.status);
   a.misc = (uint32_t*)(base + L.misc);
+  a.blk_cnt = (uint32_t*)(base + L.blk_cnt);
+  a.sel_keys = (unsigned long long*)(base + L.sel_keys);
+  a.sel_state = (uint32_t*)(base + L.sel_state);
+  a.sel_blk = (uint32_t*)(base + L.sel_blk);
+  a.sel_mcnt = (uint32_t*)(base + L.sel_mcnt);
   bk->sort_len = L.sort_len;
 
   cudaError_t e = cudaSuccess;
@@ -235,6 +245,7 @@ int llmcache_bank_create(const llmcache_bank_desc* desc, llmcache_bank_t** bank_
   if (e == cudaSuccess) e = setup_scan_kernels();
   if (e == cudaSuccess) e = setup_rows_kernels();
   if (e == cudaSuccess) e = setup_move_kernels();
+  if (e == cudaSuccess) e = setup_select_kernels();
   if (e == cudaSuccess) e = cudaStreamCreateWithFlags(&bk->side, cudaStreamNonBlocking);
   if (e == cudaSuccess) e = cudaEventCreateWithFlags(&bk->ev_fork, cudaEventDisableTiming);
   if (e == cudaSuccess) e = cudaEventCreateWithFlags(&bk->ev_join, cudaEventDisableTiming);
@@ -370,9 +381,10 @@ static int probe_common(llmcache_bank_t* bk, const void* h_in, bool compute_fp, 
     }
     // The slots for this batch's misses are chosen now, on the side stream, while the gather runs:
     // the choice depends only on the metadata after this probe's refresh, which the gather does not touch.
-    // (A one-block pass over a very large bank takes milliseconds; there it is left to the commit, so that
-    // probes that are never committed do not pay for it.)
-    bk->select_deferred = bk->desc.capacity > 65536u;
+    // (A bank that stores keys only has no gather to hide the selection behind, and over a very large bank it
+    // takes a few dozen launches; there it is left to the commit, so that probes that are never committed do
+    // not pay for it.)
+    bk->select_deferred = !bk->a.act || bk->desc.capacity > 65536u;
     if (!bk->select_deferred) {
       if (e == cudaSuccess) e = cudaEventRecord(bk->ev_fork, st);
       if (e == cudaSuccess) e = cudaStreamWaitEvent(bk->side, bk->ev_fork, 0);

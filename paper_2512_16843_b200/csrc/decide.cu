@@ -6,6 +6,7 @@
 namespace llmc {
 
 constexpr int DEC_THREADS = 1024;
+constexpr uint32_t DEC_SINGLE_BLOCK_MAX = 2048;   // batches up to this size are decided by one block
 
 // Exclusive rank of `pred` among the threads of the block (in thread order) and
 // the block total.  warp_tot is a 32-word shared array.
@@ -123,13 +124,146 @@ k_decide_compact(unsigned long long* __restrict__ best, const float* __restrict_
   }
 }
 
+// ---------------------------------------------------------------------------
+// The same step for large batches, as two grids of DEC_THREADS sequences per block.
+//   k_decide_flags    decision per sequence, matches per slot, hits and degenerate inputs per block
+//   k_compact_touch   every block adds up the hit counts of the blocks before it (so the index lists come out
+//                     ascending over the whole batch), writes its part of hit_idx / miss_idx and refreshes
+//                     the metadata of the slots its sequences matched
+// No block waits for another: the second grid starts when the first has finished.
+// ---------------------------------------------------------------------------
+__global__ void __launch_bounds__(DEC_THREADS)
+k_decide_flags(unsigned long long* __restrict__ best, const float* __restrict__ rq, uint32_t B, float tau, int cmp_ge,
+               uint8_t* __restrict__ hit, int32_t* __restrict__ slot, float* __restrict__ score,
+               uint32_t* __restrict__ hitcnt, uint32_t* __restrict__ blk_cnt, uint32_t sim_k, int32_t ham_max) {
+  griddep_sync();
+  __shared__ uint32_t warp_tot[32];
+  __shared__ uint32_t sdeg;
+  if (threadIdx.x == 0) sdeg = 0;
+  const uint32_t b = blockIdx.x * DEC_THREADS + threadIdx.x;
+  bool is_hit = false, degen = false;
+  if (b < B) {
+    const unsigned long long pk = best[b];
+    best[b] = 0ull;
+    const float r = rq[b];
+    float sc;
+    int32_t sl = -1;
+    if (!(r > 0.f)) {
+      sc = 0.f;
+      degen = true;
+    } else if (pk == 0ull) {
+      sc = -INFINITY;
+    } else {
+      sl = (int32_t)(0xFFFFFFFFu - (uint32_t)pk);
+      if (sim_k) {
+        const uint32_t ham = 0xFFFFFFFFu - (uint32_t)(pk >> 32);
+        sc = cospif((float)ham / (float)sim_k);
+        is_hit = (int32_t)ham <= ham_max;
+      } else {
+        sc = orderable_float((uint32_t)(pk >> 32)) * r;
+        is_hit = cmp_ge ? (sc >= tau) : (sc > tau);
+      }
+    }
+    if (!is_hit) sl = -1;
+    hit[b] = is_hit ? 1 : 0;
+    slot[b] = sl;
+    score[b] = sc;
+    if (is_hit) atomicAdd(hitcnt + sl, 1u);
+  }
+  uint32_t nh;
+  block_rank(is_hit, warp_tot, nh);
+  const uint32_t bal = __ballot_sync(0xFFFFFFFFu, degen);
+  if ((threadIdx.x & 31) == 0 && bal) atomicAdd(&sdeg, __popc(bal));
+  __syncthreads();
+  if (threadIdx.x == 0) {
+    blk_cnt[2 * blockIdx.x] = nh;
+    blk_cnt[2 * blockIdx.x + 1] = sdeg;
+  }
+}
+
+// Sum of v over the threads of the block (every thread receives it).  red: 32 words of shared memory.
+__device__ __forceinline__ uint32_t block_sum(uint32_t v, uint32_t* red) {
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xFFFFFFFFu, v, o);
+  __syncthreads();
+  if ((threadIdx.x & 31) == 0) red[threadIdx.x >> 5] = v;
+  __syncthreads();
+  uint32_t tot = 0;
+  const uint32_t nw = blockDim.x >> 5;
+  for (uint32_t i = 0; i < nw; ++i) tot += red[i];
+  return tot;
+}
+
+__global__ void __launch_bounds__(DEC_THREADS)
+k_compact_touch(const uint8_t* __restrict__ hit, const int32_t* __restrict__ slot, uint32_t B,
+                const uint32_t* __restrict__ blk_cnt, int32_t* __restrict__ hit_idx, int32_t* __restrict__ miss_idx,
+                uint32_t* __restrict__ counts, uint32_t* __restrict__ hitcnt, unsigned long long* __restrict__ stats,
+                uint32_t* __restrict__ last_use, uint32_t* __restrict__ hits_total, uint32_t* __restrict__ rate,
+                uint32_t* __restrict__ rate_epoch, uint32_t tick, uint32_t epoch) {
+  griddep_sync();
+  __shared__ uint32_t warp_tot[32];
+  __shared__ uint32_t red[32];
+  const uint32_t b = blockIdx.x * DEC_THREADS + threadIdx.x;
+  const bool in_range = b < B;
+  const bool is_hit = in_range && hit[b] != 0;
+  const int32_t j = is_hit ? slot[b] : -1;
+  // hits in the blocks before this one
+  uint32_t part = 0;
+  for (uint32_t i = threadIdx.x; i < blockIdx.x; i += DEC_THREADS) part += blk_cnt[2 * i];
+  const uint32_t hbase = block_sum(part, red);
+  uint32_t nh;
+  const uint32_t r = block_rank(is_hit, warp_tot, nh);
+  if (in_range) {
+    if (is_hit) hit_idx[hbase + r] = (int32_t)b;
+    else        miss_idx[(blockIdx.x * DEC_THREADS - hbase) + (threadIdx.x - r)] = (int32_t)b;
+  }
+  if (j >= 0) {
+    const uint32_t c = atomicExch(hitcnt + j, 0u);
+    const uint32_t old_rate = rate[j], old_epoch = rate_epoch[j], old_hits = hits_total[j];
+    if (c) {
+      const unsigned long long m = (unsigned long long)rate_now(old_rate, old_epoch, epoch) + (unsigned long long)HIT_Q8 * c;
+      rate[j] = m > M_CAP ? M_CAP : (uint32_t)m;
+      rate_epoch[j] = epoch;
+      last_use[j] = tick;
+      const unsigned long long h = (unsigned long long)old_hits + c;
+      hits_total[j] = h > 0xFFFFFFFFull ? 0xFFFFFFFFu : (uint32_t)h;
+    }
+  }
+  if (blockIdx.x == gridDim.x - 1) {
+    // the last block knows the batch's totals: hits before it + its own; degenerate inputs summed over all blocks
+    uint32_t dpart = 0;
+    for (uint32_t i = threadIdx.x; i < gridDim.x; i += DEC_THREADS) dpart += blk_cnt[2 * i + 1];
+    const uint32_t ndeg = block_sum(dpart, red);
+    if (threadIdx.x == 0) {
+      const uint32_t H = hbase + nh;
+      counts[0] = H;
+      counts[1] = B - H;
+      stats[ST_SEQ] += B;
+      stats[ST_HIT] += H;
+      stats[ST_MISS] += B - H;
+      stats[ST_DEGEN] += ndeg;
+    }
+  }
+}
+
 cudaError_t launch_decide(llmcache_bank* bk, uint32_t B, float tau, const float* rq,
                           const llmcache_probe_io* io, cudaStream_t st, uint32_t sim_k, int32_t ham_max) {
   ProfScope prof(bk, LLMCACHE_K_DECIDE, st);
-  return launch_k(k_decide_compact, dim3(1), dim3(DEC_THREADS), 0, st, bk->a.best, rq, B, tau,
-                  (int)(bk->desc.cmp == LLMCACHE_GE), io->hit, io->slot, io->score, io->hit_idx, io->miss_idx,
-                  io->counts, bk->a.hitcnt, bk->a.stats, bk->a.last_use, bk->a.hits, bk->a.rate, bk->a.rate_epoch,
-                  (uint32_t)bk->tick, (uint32_t)(bk->tick / bk->pol.half_life), sim_k, ham_max);
+  const uint32_t tick = (uint32_t)bk->tick, epoch = (uint32_t)(bk->tick / bk->pol.half_life);
+  if (B <= DEC_SINGLE_BLOCK_MAX)
+    return launch_k(k_decide_compact, dim3(1), dim3(DEC_THREADS), 0, st, bk->a.best, rq, B, tau,
+                    (int)(bk->desc.cmp == LLMCACHE_GE), io->hit, io->slot, io->score, io->hit_idx, io->miss_idx,
+                    io->counts, bk->a.hitcnt, bk->a.stats, bk->a.last_use, bk->a.hits, bk->a.rate, bk->a.rate_epoch,
+                    tick, epoch, sim_k, ham_max);
+  const uint32_t nblk = (B + DEC_THREADS - 1) / DEC_THREADS;
+  cudaError_t e = launch_k(k_decide_flags, dim3(nblk), dim3(DEC_THREADS), 0, st, bk->a.best, rq, B, tau,
+                           (int)(bk->desc.cmp == LLMCACHE_GE), io->hit, io->slot, io->score, bk->a.hitcnt,
+                           bk->a.blk_cnt, sim_k, ham_max);
+  if (e != cudaSuccess) return e;
+  bk->n_launches += 1;
+  return launch_k(k_compact_touch, dim3(nblk), dim3(DEC_THREADS), 0, st, (const uint8_t*)io->hit,
+                  (const int32_t*)io->slot, B, (const uint32_t*)bk->a.blk_cnt, io->hit_idx, io->miss_idx, io->counts,
+                  bk->a.hitcnt, bk->a.stats, bk->a.last_use, bk->a.hits, bk->a.rate, bk->a.rate_epoch, tick, epoch);
 }
 
 }  // namespace llmc

@@ -40,11 +40,16 @@ __global__ void k_evict(uint8_t* __restrict__ valid, const uint32_t* __restrict_
   }
 }
 
+constexpr uint32_t SEL_ONE_BLOCK_MAX = 4096;
+
 // One block.  Runs on the bank's side stream, next to the gather of the same probe.
 __global__ void __launch_bounds__(SEL_THREADS) k_select_victims(SelectArgs A) { select_victims_block(A); }
 
 cudaError_t launch_select_victims(llmcache_bank* bk, const llmcache_probe_io* io, uint32_t B, cudaStream_t st) {
   if (B == 0) return cudaSuccess;
+  // one block is quickest while the bank's keys and the batch's misses are a few thousand; beyond that the
+  // selection runs as a sequence of grids over all SMs
+  if (bk->desc.capacity > SEL_ONE_BLOCK_MAX || B > SEL_ONE_BLOCK_MAX) return launch_select_victims_mb(bk, io, B, st);
   SelectArgs sel;
   sel.mv = MetaView{bk->a.valid, bk->a.last_use, bk->a.insert_tick, bk->a.rate, bk->a.rate_epoch};
   sel.pol = bk->pol;

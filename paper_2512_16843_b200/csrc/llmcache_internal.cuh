@@ -50,7 +50,14 @@ struct BankArrays {
   unsigned long long* stats;      // [ST_COUNT]
   uint32_t* status;         // [1] sticky device status
   uint32_t* misc;           // [8] small per-call words
+  // scratch of the multi-block decision and victim selection (large batches / large banks)
+  uint32_t* blk_cnt;        // [2 * ceil(max_batch / 1024)] hits and degenerate inputs per block of the decision
+  unsigned long long* sel_keys;   // [N] taking-order key of every slot
+  uint32_t* sel_state;      // [SEL_STATE_WORDS] radix-select state and digit histograms (zeroed per selection)
+  uint32_t* sel_blk;        // [2 * ceil(N / 1024)] keys below / equal to the threshold per block
+  uint32_t* sel_mcnt;       // [ceil(max_batch / 1024)] insertable misses per block
 };
+constexpr uint32_t SEL_STATE_WORDS = 64 + 8 * 256;
 
 }  // namespace llmc
 
@@ -135,6 +142,8 @@ cudaError_t launch_simhash_scan(llmcache_bank* bk, const __nv_bfloat16* q, uint3
 cudaError_t launch_gather(llmcache_bank* bk, const void* h_in, void* h_out,
                           const llmcache_probe_io* io, uint32_t B, cudaStream_t st);
 cudaError_t launch_select_victims(llmcache_bank* bk, const llmcache_probe_io* io, uint32_t B, cudaStream_t st);
+cudaError_t setup_select_kernels();
+cudaError_t launch_select_victims_mb(llmcache_bank* bk, const llmcache_probe_io* io, uint32_t B, cudaStream_t st);
 cudaError_t launch_scatter_insert(llmcache_bank* bk, const void* miss_out, const llmcache_probe_io* io,
                                   void* h_out, int32_t* new_slot_out, uint32_t B, cudaStream_t st);
 cudaError_t launch_evict(llmcache_bank* bk, uint32_t mode, const int32_t* slots, uint32_t n,

@@ -80,12 +80,13 @@ __device__ __forceinline__ uint32_t sel_scan(uint32_t v, uint32_t* warp_tot, uin
 // the arrays may live in shared or global memory.  Thread t handles the pair (i, i + stride) with
 // i = (t / stride) * 2 * stride + t % stride, so for stride <= 32 a warp only touches elements that
 // no other warp touches in that step and a warp-level sync is enough.
+template <int THREADS = SEL_THREADS>
 __device__ __forceinline__ void bitonic_steps(unsigned long long* key, uint32_t* val, uint32_t len, uint32_t g0,
                                               uint32_t size, uint32_t first_stride) {
   // the steps of merge size `size` with strides first_stride, first_stride / 2, ..., 1 on `len` elements whose
   // first one has index g0 in the whole sequence (the direction of a pair depends on that index)
   for (uint32_t stride = first_stride, lg = 31 - __clz(stride);; stride >>= 1, --lg) {
-    for (uint32_t t = threadIdx.x; t < (len >> 1); t += SEL_THREADS) {
+    for (uint32_t t = threadIdx.x; t < (len >> 1); t += THREADS) {
       const uint32_t i = ((t >> lg) << (lg + 1)) | (t & (stride - 1)), l = i + stride;
       const unsigned long long ka = key[i], kb = key[l];
       const uint32_t va = val[i], vb = val[l];

@@ -213,3 +213,65 @@ def lockstep_step(gb: L.Bank, ob: O.Bank, bufs: L.ProbeBuffers, h_dev: torch.Ten
     res["inserted"] = int((new_or >= 0).sum())
     res["h_out"] = h_out2
     return res
+
+
+def lockstep_step_sampled(gb: L.Bank, ob: O.Bank, bufs: L.ProbeBuffers, q_dev: torch.Tensor, n_sample: int, seed: int,
+                          tau=None, do_commit=True):
+    """One probe_fp (+ commit) of a keys-only bank that is too large for the oracle to score in full.
+    The oracle scores a seeded sample of the queries against the whole bank (scores, decisions, slots);
+    the compaction is checked in full against the GPU's own flags; the metadata refresh and the whole commit
+    (which slots the misses take, every array of the bank afterwards) are the oracle's, computed from the
+    GPU's decisions, and compared in full."""
+    B = q_dev.shape[0]
+    pull_state(gb, ob, with_act=False)
+    bufs.fp[:B].copy_(q_dev)
+    gb.probe_fp(bufs, B, tau=tau)
+    torch.cuda.synchronize()
+    assert gb.status() == L.OK
+    tau_eff = float(gb.desc.tau) if tau is None else tau
+    hit = bufs.hit[:B].cpu().numpy()
+    slot = bufs.slot[:B].cpu().numpy()
+    score = bufs.score[:B].cpu().numpy()
+    H, M = [int(x) for x in bufs.counts.cpu()]
+    assert H + M == B and H == int(hit.sum())
+    idx = np.arange(B, dtype=np.int32)
+    assert np.array_equal(bufs.hit_idx[:H].cpu().numpy(), idx[hit != 0])
+    assert np.array_equal(bufs.miss_idx[:M].cpu().numpy(), idx[hit == 0])
+    assert np.all(slot[hit == 0] == -1)
+    # the oracle on a sample of the queries
+    sample = np.sort(np.random.Generator(np.random.Philox(key=seed)).choice(B, min(n_sample, B), replace=False))
+    qs = bits(q_dev[torch.from_numpy(sample).to(q_dev.device)])
+    rqs = O.inv_norm_of_stored(qs)
+    s = O.scores(qs, rqs, ob.fp, ob.rb, ob.valid)
+    best, bslot, _ = O.best_match(s)
+    ohit, oslot = O.decide(best, bslot, rqs, tau_eff, ob.cmp_ge)
+    near = 0
+    for i, b in enumerate(sample):
+        so, sg = float(best[i]), float(score[b])
+        if np.isinf(so) or np.isinf(sg):
+            assert so == sg
+        else:
+            assert abs(sg - so) <= REL * max(abs(so), 1e-6) + 1e-6, f"score[{b}] {sg} vs {so}"
+        if hit[b] != ohit[i]:
+            assert abs(so - tau_eff) <= REL * abs(tau_eff) + 1e-6
+            near += 1
+        elif hit[b] and slot[b] != oslot[i]:
+            assert abs(float(s[i, slot[b]]) - so) <= REL * abs(so)
+            near += 1
+    # metadata refresh from the GPU's decisions
+    ob.tick += 1
+    O.touch(ob, slot[hit != 0])
+    assert_state_equal(gb, ob, with_act=False, where="after probe")
+    res = dict(H=H, M=M, near=near)
+    if not do_commit:
+        return res
+    gp = gpu_probe_result(bufs, B, ob.tick)
+    gb.commit(None, bufs)
+    torch.cuda.synchronize()
+    assert gb.status() == L.OK
+    new_or = O.commit(ob, gp, None, None)
+    new_gpu = bufs.new_slot[:M].cpu().numpy()
+    assert np.array_equal(new_gpu, new_or), "new_slot differs from the oracle's"
+    assert_state_equal(gb, ob, with_act=False, where="after commit")
+    res["inserted"] = int((new_or >= 0).sum())
+    return res

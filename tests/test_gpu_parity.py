@@ -395,3 +395,43 @@ def test_more_victims_than_the_shared_memory_sort_holds(policy):
         if step:
             assert r["H"] >= 700
     gb.close()
+
+
+@pytest.mark.parametrize("N,B,steps", [(5000, 20000, 3), (40000, 20000, 5), (262144, 65536, 7)])
+def test_large_bank_large_batch_commit_lockstep(N, B, steps):
+    """Banks and batches for which the decision and the victim selection run as several grids: tens of
+    thousands of misses per step take free slots first and then evict by (stale, decayed rate, last use, slot);
+    the repeated keys are matched by several queries each.  Keys-only banks; the oracle scores a sample of
+    the queries and replays the metadata refresh and the whole commit from the GPU's decisions."""
+    k = 64
+    gb = L.Bank(capacity=N, seq_len=1, d_model=k, fp_dim=k, max_batch=B, store_act=0, tau=0.9,
+                policy=L.LRU_STALENESS, half_life_ticks=2, min_age_ticks=1, stale_floor_q8=200)
+    ob = U.oracle_bank_like(gb, store_act=False)
+    bufs = L.ProbeBuffers(B, k, DEV)
+    g = torch.Generator().manual_seed(4242 + N)
+    tot = dict(H=0, inserted=0)
+    for step in range(steps):
+        q = rand_h(B, 1, k, 9000 + 17 * step + N, "bf16").view(B, k)
+        q = (q.float() / q.float().norm(dim=1, keepdim=True)).to(torch.bfloat16)
+        resident = int(ob.valid.sum()) if step else 0
+        if resident:
+            # 40% of the batch repeats keys that are in the bank, drawn from a tenth of the occupied slots so
+            # that many are matched several times
+            occ = np.flatnonzero(ob.valid)
+            pool_slots = occ[torch.randperm(len(occ), generator=g)[: max(1, len(occ) // 10)].numpy()]
+            n_rep = (B * 4) // 10
+            pick = pool_slots[torch.randint(0, len(pool_slots), (n_rep,), generator=g).numpy()]
+            rows = torch.randperm(B, generator=g)[:n_rep].to(DEV)
+            q[rows] = U.to_dev_bf16(ob.fp[pick], DEV)
+        r = U.lockstep_step_sampled(gb, ob, bufs, q.contiguous(), 48, 77 + step)
+        tot["H"] += r["H"]
+        tot["inserted"] += r["inserted"]
+        if resident:
+            assert r["H"] >= (B * 4) // 10
+    st = gb.stats()
+    assert st["resident"] == min(N, tot["inserted"])
+    if tot["inserted"] > N:
+        assert st["evictions"] == tot["inserted"] - N
+    if B > N:
+        assert st["dropped"] > 0
+    gb.close()
