@@ -1,16 +1,18 @@
 #!/usr/bin/env python
-"""Benchmark of the per-layer cache probe on the BERT-base-shaped workload (other shapes: --workload).
+"""Benchmark of the per-layer cache probe.
 
-One step = one pass of the whole hot path over one batch at every layer: for each
-of the 12 per-layer banks, llmcache_probe (fingerprint, bank scan, threshold +
-compaction, gather of hits, metadata refresh) followed by llmcache_commit (victim
-selection, scatter of miss outputs, insertion).  Metric: probed sequences per
+One step = one pass of the whole hot path over one batch at every layer: for each per-layer bank,
+llmcache_probe (fingerprint, bank scan, threshold + compaction, gather of hits, metadata refresh) followed
+by llmcache_commit (victim selection, scatter of miss outputs, insertion).  Metric: probed sequences per
 second per layer = (sequences x layers) / time.
 
-    python bench.py --gpus 1 --steps 20 --warmup 5
-    python bench.py --impl reference ...       # the CPU oracle, timed as it stands
+    python bench.py --gpus 1 --steps 20 --warmup 5      # headline + sub-records, one JSON line
+    python bench.py --workload bert_base ...            # one workload only
+    python bench.py --impl reference ...                # the CPU oracle, timed as it stands
 
-Prints one JSON line on rank 0.
+The default run times the largest single-GPU configuration (BERT-large-shaped encoder under churn) as the
+headline and adds, in the same JSON line, the bank-scan stress (tensor roofline), the gather of 1 MiB rows
+(HBM roofline) and the smaller configurations as sub-records.  Prints one JSON line on rank 0.
 """
 import argparse
 import hashlib
@@ -30,6 +32,7 @@ import torch
 
 METRIC = "probed sequences/sec per layer (fingerprint+scan+gather)"
 UNIT = "sequences/s"
+NOMINAL_HBM_GBS = 8000.0                                 # the ~8 TB/s the targets are quoted against
 
 # BERT-base-shaped workload: 12 layers, d_model 768, batch 256 x seq_len 384, vocabulary 30,522,
 # 60% of the sequences are token-level edits (10% of positions) of 64 seed sequences, per-layer bank of
@@ -37,29 +40,48 @@ UNIT = "sequences/s"
 CFG = dict(layers=12, d_model=768, seq_len=384, batch=256, vocab=30522, n_seeds=64, edit_fraction=0.60,
            edit_positions=0.10, bank=2048, fp_dim=256, tau=0.90, pool_batches=24)
 
-# Other shapes of the same step (parity-test configurations; `--workload`): not the headline line.
+HEADLINE = "bert_large_churn"
 WORKLOADS = {
     "bert_base": CFG,
     # GPT-2-small-shaped decoder: batch 32 x seq_len 1024, half of each batch are repeats of 64 hot documents
     # (512-token prefix of one of 8 seed documents + fixed suffix), half have fresh random suffixes
     "gpt2_small": dict(layers=12, d_model=768, seq_len=1024, batch=32, vocab=50257, n_seeds=8, bank=1024, fp_dim=256,
-                       tau=0.90, pool_batches=24, kind="prefix", hot=64, prefix=512, repeat_fraction=0.5),
+                       tau=0.90, pool_batches=72, kind="prefix", hot=64, prefix=512, repeat_fraction=0.5),
     # BERT-large-shaped encoder under churn: batch 512 x seq_len 512, 75% near one of 256 drifting centres
     # (shift 0.02 per batch, noise 0.05), 25% junk that never repeats, LRU + staleness eviction
     "bert_large_churn": dict(layers=24, d_model=1024, seq_len=512, batch=512, bank=1024, fp_dim=256, tau=0.90,
                              pool_batches=10, kind="cluster", centres=256, near_fraction=0.75, drift=0.02, noise=0.05),
+    # Single-layer probe of fp32 hidden states (the batch-1-to-64 / seq_len-128 regime): 1,024 entries from 16
+    # centres, 64 queries (half near an entry, half fresh).  Eight independent banks and 72 input batches rotate,
+    # so that neither the inputs nor the stored rows of a probe are still in L2 from the previous one and no
+    # batch comes round again (its misses would then hit) within a default run.
+    "single_layer_fp32": dict(layers=8, d_model=768, seq_len=128, batch=64, bank=1024, fp_dim=256, tau=0.90,
+                              pool_batches=72, kind="cluster1", centres=16, hidden="f32"),
 }
 
 
 def describe(name, cfg):
     head = {"bert_base": "BERT-base-shaped encoder", "gpt2_small": "GPT-2-small-shaped decoder",
-            "bert_large_churn": "BERT-large-shaped encoder under churn"}[name]
+            "bert_large_churn": "BERT-large-shaped encoder under churn",
+            "single_layer_fp32": "single-layer probe, fp32 hidden states"}[name]
     tail = {"bert_base": "60% token-level edits of 64 seeds",
             "gpt2_small": "half repeats of 64 hot documents (512-token shared prefixes), half fresh suffixes",
-            "bert_large_churn": "75% near 256 drifting centres (shift 0.02 per batch), 25% junk, LRU + staleness eviction"}[name]
+            "bert_large_churn": "75% near 256 drifting centres (shift 0.02 per batch), 25% junk, LRU + staleness eviction",
+            "single_layer_fp32": "entries from 16 centres (noise 0.05), half of the queries near an entry, half fresh; "
+                                 "8 independent banks in rotation"}[name]
     return (f"{head}: {cfg['layers']} per-layer banks x {cfg['bank']} entries (bf16 {cfg['seq_len']}x{cfg['d_model']}), "
             f"batch {cfg['batch']} x seq_len {cfg['seq_len']}, d_model {cfg['d_model']}, fp_dim {cfg['fp_dim']} (projected), "
             f"tau {cfg['tau']:.2f}, {tail}")
+
+
+def config_of(name, cfg, world=1):
+    """The `config` object of the JSON line: the same for the GPU arm and for the oracle arm."""
+    B, n, d, N, P = cfg["batch"], cfg["seq_len"], cfg["d_model"], cfg["bank"], cfg["pool_batches"]
+    s_in = 4 if cfg.get("hidden") == "f32" else 2
+    return {"workload": describe(name, cfg), "step": f"probe + commit on each of {cfg['layers']} layers",
+            "l2": f"inputs larger than L2: every layer of a step reads a different {B * n * d * s_in / 1e6:.0f} MB "
+                  f"batch out of a pool of {P}, plus {N * n * d * 2 / 1e9:.2f} GB of bank rows per layer",
+            "parallelism": "independent replicas per GPU, no collective" if world > 1 else "single GPU"}
 
 
 def make_inputs(cfg, seed, dev):
@@ -90,6 +112,11 @@ def make_inputs(cfg, seed, dev):
         warm += [wl.hidden(wl.with_shared_prefix(seeds_tok, B, cfg["prefix"], seed + 300 + i)[0])
                  for i in range((N - cfg["hot"]) // B)]
         return warm, pool
+    if kind == "cluster1":
+        wl = synth.ClusterWorkload(cfg["centres"], n, d, seed, dev, dtype=torch.float32)
+        warm = [wl.entries(first, B) for first in range(0, N, B)]
+        pool = [wl.queries(B, N, seed + 300 + i)[0] for i in range(P)]
+        return warm, pool
     # cluster: drifting centres in hidden-state space
     C = cfg["centres"]
     centres = synth.randn((C, n, d), seed + 1, dev, torch.bfloat16)
@@ -117,32 +144,38 @@ def make_inputs(cfg, seed, dev):
     return warm, pool
 
 
-# DRAM traffic per launch from an ncu capture of the named kernel on this workload, valid only while the
-# kernel's source file is unchanged (sha256 prefix of the file at capture time).
+# DRAM traffic per launch (dram__bytes_read.sum + dram__bytes_write.sum of one launch) from an ncu capture of
+# the named kernel on the named workload; valid only while the kernel's source file is unchanged (sha256
+# prefix of the file at capture time), otherwise the bench prints null.
 NCU_TRAFFIC = {
-    # profiles/bert_base_one_layer_kernels.md (dram__bytes_read.sum + dram__bytes_write.sum of one launch)
-    "pool": {"file": "fp_phases.cuh", "sha": "bbd8f33e3017", "bytes_per_launch": 155089664},
-    "gather": {"file": "rows.cu", "sha": "40053a7cf26b", "bytes_per_launch": 82544896},
-    "scatter": {"file": "rows.cu", "sha": "40053a7cf26b", "bytes_per_launch": 124241152},
+    "bert_base": {
+        "pool": {"file": "fp_phases.cuh", "sha": "bbd8f33e3017", "bytes_per_launch": 155089664},
+        "gather": {"file": "rows.cu", "sha": "40053a7cf26b", "bytes_per_launch": 82544896},
+        "scatter": {"file": "rows.cu", "sha": "40053a7cf26b", "bytes_per_launch": 124241152},
+    },
 }
+
+SUB_WORKLOADS = ["bert_base", "gpt2_small", "single_layer_fp32"]
 
 
 def parse():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=200)
+    ap.add_argument("--steps", type=int, default=50)
     ap.add_argument("--warmup", type=int, default=10)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--e2e-steps", type=int, default=3)
     ap.add_argument("--no-cpu-baseline", action="store_true")
-    ap.add_argument("--workload", default="bert_base", choices=["bert_base", "gpt2_small", "bert_large_churn", "scan_stress", "gather_stress", "e2e_bert_base"])
+    ap.add_argument("--workload", default="all",
+                    choices=["all"] + list(WORKLOADS) + ["scan_stress", "gather_stress", "e2e_bert_base"],
+                    help="all: the headline workload plus every sub-record (default)")
     ap.add_argument("--bank", type=int, default=65536, help="scan_stress: number of bank entries")
     ap.add_argument("--queries", type=int, default=65536, help="scan_stress: queries per batch (gather_stress: 8192 per probe)")
     ap.add_argument("--act-rows", type=int, default=16384, help="gather_stress: rows of the activation store (1 MiB each)")
     ap.add_argument("--batch", type=int, default=0, help="e2e_bert_base: sequences per batch (default 256)")
     ap.add_argument("--seq-len", type=int, default=0, help="e2e_bert_base: sequence length (default 384)")
-    ap.add_argument("--layers", type=int, default=0, help="bert_base: number of per-layer banks (default 12; fewer only for profiler captures)")
-    ap.add_argument("--pool-batches", type=int, default=0, help="bert_base: distinct input batches in rotation (default 24)")
+    ap.add_argument("--layers", type=int, default=0, help="number of per-layer banks (default: the workload's; fewer only for profiler captures)")
+    ap.add_argument("--pool-batches", type=int, default=0, help="distinct input batches in rotation (default: the workload's)")
     return ap.parse_args()
 
 
@@ -178,6 +211,12 @@ class ClockSampler:
     def _read(self):
         for ln in self.proc.stdout:
             self.lines.append(ln.strip())
+
+    def wait_ready(self, timeout_s=2.0):
+        """Blocks until nvidia-smi has delivered its first sample (it takes a moment to start)."""
+        t0 = time.time()
+        while self.proc and not self.lines and time.time() - t0 < timeout_s:
+            time.sleep(0.01)
 
     def mark(self):
         """Start of the timed region: samples taken before it are only used if the region gets none."""
@@ -249,10 +288,25 @@ def build_batches(wl, seeds_tok, count, seed, device, B=None):
     return out
 
 
-def run_ours(args):
-    from paper_2512_16843_b200 import binding as L
-    from paper_2512_16843_b200 import synth
-    L.lib()                                              # fail loudly if the CUDA library is missing
+def median_min(xs):
+    xs = sorted(xs)
+    return (float(np.median(xs)) if xs else None), (float(xs[0]) if xs else None)
+
+
+def timed_steps(fn, steps, barrier):
+    """Runs fn() `steps` times with an event before every step and one after the last (on the current stream).
+    Returns (total ms of exactly these steps, [ms of each step])."""
+    ev = [torch.cuda.Event(enable_timing=True) for _ in range(steps + 1)]
+    barrier()
+    for i in range(steps):
+        ev[i].record()
+        fn()
+    ev[steps].record()
+    barrier()
+    return ev[0].elapsed_time(ev[steps]), [ev[i].elapsed_time(ev[i + 1]) for i in range(steps)]
+
+
+def init_dist():
     rank = int(os.environ.get("RANK", "0"))
     local = int(os.environ.get("LOCAL_RANK", "0"))
     world = int(os.environ.get("WORLD_SIZE", "1"))
@@ -264,32 +318,51 @@ def run_ours(args):
     if world > 1:
         import torch.distributed as dist
         dist.init_process_group("nccl", device_id=dev)
-    cfg = dict(WORKLOADS[args.workload])
+    return rank, local, world, dev, dist
+
+
+def run_probe_workload(name, args, env, steps, warmup, e2e_steps, with_cpu, tau_sweep=()):
+    """One workload of per-layer banks: timed steps, per-kernel device times, end-to-end steps from host
+    memory, the CPU oracle on a sample.  Returns the record (a dict); the caller prints it."""
+    from paper_2512_16843_b200 import binding as L
+    from paper_2512_16843_b200 import synth
+    rank, local, world, dev, dist = env
+    cfg = dict(WORKLOADS[name])
     if args.layers:
         cfg["layers"] = args.layers
     if args.pool_batches:
         cfg["pool_batches"] = args.pool_batches
     Lyr, d, n, B, N, k = (cfg[x] for x in ("layers", "d_model", "seq_len", "batch", "bank", "fp_dim"))
+    f32_in = cfg.get("hidden") == "f32"
+    s_in = 4 if f32_in else 2
     seed = rank_seed(rank)
     proj = synth.projection(d, k, seed + 6, dev)
-    banks = [L.Bank(device=local, capacity=N, seq_len=n, d_model=d, fp_dim=k, max_batch=B, hidden_dtype=L.BF16,
-                    proj=proj, tau=cfg["tau"], policy=L.LRU_STALENESS) for _ in range(Lyr)]
+    banks = [L.Bank(device=local, capacity=N, seq_len=n, d_model=d, fp_dim=k, max_batch=B,
+                    hidden_dtype=L.F32 if f32_in else L.BF16, proj=proj, tau=cfg["tau"], policy=L.LRU_STALENESS)
+             for _ in range(Lyr)]
     bufs = [L.ProbeBuffers(B, k, dev) for _ in range(Lyr)]
     P = cfg["pool_batches"]
     warm, pool = make_inputs(cfg, seed, dev)
     miss_out = [synth.activations(B, n, d, seed + 50 + i, dev) for i in range(2)]
     h_out = [torch.empty((B, n * d), dtype=torch.bfloat16, device=dev) for _ in range(3)]
-    # warm every bank to capacity through the library
+    # warm every bank to capacity through the library; the very first probe + commit on this shape is timed
+    # by the host's clock as the cold call (call to completion, first-use costs of the kernels included)
+    torch.cuda.synchronize()
+    cold_ms = None
     for l in range(Lyr):
         for i, hb in enumerate(warm):
+            t0 = time.perf_counter()
             banks[l].probe(hb, bufs[l], h_out=h_out[0])
             banks[l].commit(miss_out[i % 2], bufs[l], h_out=h_out[0])
+            if cold_ms is None:
+                torch.cuda.synchronize()
+                cold_ms = (time.perf_counter() - t0) * 1e3
     del warm
     torch.cuda.synchronize()
 
     counter = [0]
 
-    def one_step(host_pool=None, stage=None, results=None):
+    def one_step(host_pool=None, stage=None, results=None, tau=None):
         s = counter[0]
         counter[0] += 1
         for l in range(Lyr):
@@ -297,10 +370,10 @@ def run_ours(args):
             if host_pool is None:
                 h = pool[i]
             else:
-                stage[l % 2].copy_(host_pool[i], non_blocking=True)
+                stage[l % 2].copy_(host_pool[i % len(host_pool)], non_blocking=True)
                 h = stage[l % 2]
             ho = h_out[(s + l) % 3]
-            banks[l].probe(h, bufs[l], h_out=ho)
+            banks[l].probe(h, bufs[l], h_out=ho, tau=tau)
             banks[l].commit(miss_out[(s + l) % 2], bufs[l], h_out=ho)
             if results is not None:
                 r = results[l]
@@ -316,24 +389,21 @@ def run_ours(args):
     sampler = ClockSampler(local)
     if rank == 0:
         sampler.start()                                  # already sampling when the timed region begins
-    for _ in range(args.warmup):
+    for _ in range(warmup):
         one_step()
+    if rank == 0:
+        sampler.wait_ready()
     barrier()
     launches0 = sum(b.stats()["kernel_launches"] for b in banks)
     hits0 = sum(b.stats()["hits"] for b in banks)
-    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-    barrier()
     sampler.mark()
-    e0.record()
-    for _ in range(args.steps):
-        one_step()
-    e1.record()
-    barrier()
+    total_ms, per_step = timed_steps(one_step, steps, barrier)
     clocks = sampler.stop() if rank == 0 else None
-    seqs = B * Lyr * args.steps
-    ms, _, value = aggregate(e0.elapsed_time(e1), seqs, dist, dev)
+    seqs = B * Lyr * steps
+    ms, _, value = aggregate(total_ms, seqs, dist, dev)
     launches = sum(b.stats()["kernel_launches"] for b in banks) - launches0
     hits = sum(b.stats()["hits"] for b in banks) - hits0
+    med, mn = median_min(per_step)
 
     # ---- per-kernel device time over the same loop (events around every launch) -------------------
     # The GPU is held back by a ~2 ms spin before every step so that the host has the whole step enqueued
@@ -341,7 +411,7 @@ def run_ours(args):
     for b in banks:
         b.profile(True)
     st0 = [b.stats() for b in banks]
-    prof_steps = min(args.steps, 50)
+    prof_steps = min(steps, 50)
     for _ in range(prof_steps):
         torch.cuda._sleep(4000000)
         one_step()
@@ -349,8 +419,8 @@ def run_ours(args):
     prof = {}
     for b in banks:
         b.profile(False)
-        for name, (tms, cnt) in b.profile_read().items():
-            a = prof.setdefault(name, [0.0, 0])
+        for kname, (tms, cnt) in b.profile_read().items():
+            a = prof.setdefault(kname, [0.0, 0])
             a[0] += tms
             a[1] += cnt
     st1 = [b.stats() for b in banks]
@@ -358,103 +428,159 @@ def run_ours(args):
     M_avg = B - H_avg
     row = n * d * 2
     algo_bytes = {                                       # algorithmic bytes per launch
-        "pool": B * n * d * 2 + B * k * 2,
+        "pool": B * n * d * s_in + B * k * 2,
         "gather": H_avg * row * 2,
         "scatter": M_avg * row * 3 + M_avg * k * 2,
     }
     # the victim selection runs on a side stream next to the gather: it is not on the critical path
-    total_ms = sum(v[0] for name, v in prof.items() if name != "select") or 1.0
-    kernels = {name: {"ms_per_launch": v[0] / v[1], "launches": v[1], "share": v[0] / total_ms}
-               for name, v in prof.items() if v[1]}
+    total_k = sum(v[0] for kname, v in prof.items() if kname != "select") or 1.0
+    kernels = {kname: {"ms_per_launch": v[0] / v[1], "launches": v[1], "share": v[0] / total_k}
+               for kname, v in prof.items() if v[1]}
     dom = max((k_ for k_ in kernels if k_ in algo_bytes), key=lambda k_: kernels[k_]["share"])
     peaks, peak_kind = measured_peaks()
     achieved = algo_bytes[dom] / (kernels[dom]["ms_per_launch"] * 1e-3) / 1e9
     roof = {"kernel": dom, "bound": "hbm", "achieved": achieved, "peak": peaks["hbm_gbs"], "unit": "GB/s",
-            "frac": achieved / peaks["hbm_gbs"], "peak_kind": "of " + peak_kind, "traffic": ncu_traffic(dom) if args.workload == "bert_base" else None,
+            "frac": achieved / peaks["hbm_gbs"], "frac_of_nominal_8tbs": achieved / NOMINAL_HBM_GBS,
+            "peak_kind": "of " + peak_kind, "traffic": ncu_traffic(name, dom),
             "algorithmic_bytes_per_launch": algo_bytes[dom], "all_kernels": {}}
-    for name in kernels:
-        ent = dict(kernels[name])
-        if name in algo_bytes:
-            ent["achieved_GBps"] = algo_bytes[name] / (ent["ms_per_launch"] * 1e-3) / 1e9
+    for kname in kernels:
+        ent = dict(kernels[kname])
+        if kname in algo_bytes:
+            ent["algorithmic_bytes_per_launch"] = algo_bytes[kname]
+            ent["achieved_GBps"] = algo_bytes[kname] / (ent["ms_per_launch"] * 1e-3) / 1e9
             ent["frac_of_hbm_peak"] = ent["achieved_GBps"] / peaks["hbm_gbs"]
-        roof["all_kernels"][name] = ent
+            ent["frac_of_nominal_8tbs"] = ent["achieved_GBps"] / NOMINAL_HBM_GBS
+        roof["all_kernels"][kname] = ent
+    # all HBM kernels of a step together, against the step itself (no event brackets involved)
+    step_bytes = Lyr * sum(algo_bytes.values())
+    roof["step_aggregate"] = {"algorithmic_bytes_per_step": step_bytes,
+                              "achieved_GBps": step_bytes / (med * 1e-3) / 1e9,
+                              "frac_of_hbm_peak": step_bytes / (med * 1e-3) / 1e9 / peaks["hbm_gbs"],
+                              "what": "pool + gather + scatter bytes of all layers / median step time (small kernels included in the time)"}
+
+    # ---- threshold sweep (the paper's threshold ablation, Sec. V-F): same batches, other tau --------
+    sweep = None
+    if tau_sweep:
+        sweep = {}
+        for tau in tau_sweep:
+            h0s = sum(b.stats()["hits"] for b in banks)
+            t_ms, t_steps = timed_steps(lambda: one_step(tau=tau), 5, barrier)
+            h1s = sum(b.stats()["hits"] for b in banks)
+            t_med, t_min = median_min(t_steps)
+            sweep["%.2f" % tau] = {"ms_per_step_median": t_med, "ms_per_step_min": t_min,
+                                   "hit_fraction": (h1s - h0s) / float(B * Lyr * 5)}
 
     # ---- end to end: inputs come from pinned host memory, decisions go back to the host ------------
     e2e = None
-    if args.e2e_steps > 0:
-        host_pool = [p.cpu().pin_memory() for p in pool]
+    if e2e_steps > 0:
+        n_host = min(P, 4)                               # distinct batches kept in pinned host memory
+        host_pool = [pool[i].cpu().pin_memory() for i in range(n_host)]
         stage = [torch.empty_like(pool[0]) for _ in range(2)]
         results = [(torch.empty(B, dtype=torch.uint8).pin_memory(), torch.empty(B, dtype=torch.int32).pin_memory(),
                     torch.empty(B, dtype=torch.float32).pin_memory()) for _ in range(Lyr)]
         one_step(host_pool, stage, results)
-        barrier()
-        e0.record()
-        for _ in range(args.e2e_steps):
-            one_step(host_pool, stage, results)
-        e1.record()
-        barrier()
-        ems, _, e2e_value = aggregate(e0.elapsed_time(e1), B * Lyr * args.e2e_steps, dist, dev)
+        e_ms, e_steps = timed_steps(lambda: one_step(host_pool, stage, results), e2e_steps, barrier)
+        ems, _, e2e_value = aggregate(e_ms, B * Lyr * e2e_steps, dist, dev)
         e2e = {"value": e2e_value, "unit": UNIT,
-               "h2d_bytes_per_step": Lyr * B * n * d * 2, "d2h_bytes_per_step": Lyr * B * 9 + Lyr * 8,
-               "steps": args.e2e_steps}
+               "h2d_bytes_per_step": Lyr * B * n * d * s_in, "d2h_bytes_per_step": Lyr * B * 9 + Lyr * 8,
+               "steps": e2e_steps, "ms_per_step": ems / e2e_steps}
         del host_pool
 
     cpu = None
-    if rank == 0 and world == 1 and not args.no_cpu_baseline:
+    if with_cpu and rank == 0 and world == 1:
         cpu = cpu_baseline_from_gpu_state(banks, pool, proj, counter[0], cfg)
 
-    if rank == 0:
-        out = {"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
-               "warmup": args.warmup, "ms_per_step": ms / args.steps, "higher_is_better": True, "scaling": "weak",
-               "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
-               "config": {"workload": describe(args.workload, cfg),
-                          "step": f"probe + commit on each of {Lyr} layers", "hit_fraction": hits / float(seqs),
-                          "l2": f"inputs larger than L2: every layer of a step reads a different {B * n * d * 2 / 1e6:.0f} MB "
-                                f"batch out of a pool of {P}, plus {N * n * d * 2 / 1e9:.2f} GB of bank rows per layer",
-                          "parallelism": "independent replicas per GPU, no collective" if world > 1 else "single GPU"},
-               "e2e": e2e, "gpu_launches": launches, "roofline": roof, "cpu_baseline": cpu, "clocks": clocks}
-        print(json.dumps(out))
+    assert all(b.status() == L.OK for b in banks), "a bounded device wait expired during the benchmark"
+    out = {"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": steps,
+           "warmup": warmup, "ms_per_step": ms / steps, "ms_per_step_median": med, "ms_per_step_min": mn,
+           "cold_call_ms": cold_ms, "higher_is_better": True, "scaling": "weak",
+           "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
+           "config": config_of(name, cfg, world),
+           "observed": {"hit_fraction": hits / float(seqs), "hidden_dtype": "f32" if f32_in else "bf16",
+                        "distinct_batches": P},
+           "e2e": e2e, "gpu_launches": launches, "roofline": roof, "cpu_baseline": cpu, "clocks": clocks}
+    if sweep is not None:
+        out["tau_sweep"] = sweep
     for b in banks:
         b.close()
+    del banks, bufs, pool, miss_out, h_out
+    torch.cuda.empty_cache()
+    return out
+
+
+def brief(rec):
+    """A sub-record of the JSON line: the figures of a workload without the keys every line shares."""
+    drop = ("metric", "unit", "n_gpus", "higher_is_better", "scaling", "vs_baseline", "data")
+    return {k: v for k, v in rec.items() if k not in drop}
+
+
+def run_ours(args):
+    env = init_dist()
+    rank, local, world, dev, dist = env
+    name = HEADLINE if args.workload == "all" else args.workload
+    out = run_probe_workload(name, args, env, args.steps, args.warmup, args.e2e_steps, not args.no_cpu_baseline,
+                             tau_sweep=(0.80, 0.90, 0.95) if name == "bert_base" else ())
+    if args.workload == "all" and world == 1:
+        # sub-records: the two roofline targets at the bank-scan stress shape, then the smaller configurations
+        sub_steps, sub_warm = max(5, min(args.steps, 20)), max(3, min(args.warmup, 5))
+        scan = run_scan_stress(args, steps=10, warmup=3)
+        out["roofline_scan"] = dict(scan["roofline"], ms_per_step=scan["ms_per_step"], workload=scan["config"]["workload"],
+                                    hits=scan["config"]["hits"], expected_hits=scan["config"]["expected_hits"],
+                                    clocks=scan["clocks"])
+        gat = run_gather_stress(args, steps=3, warmup=3)
+        out["roofline_gather"] = dict(gat["roofline"], ms_per_step=gat["ms_per_step"], workload=gat["config"]["workload"],
+                                      hits=gat["config"]["hits"], expected_hits=gat["config"]["expected_hits"],
+                                      clocks=gat["clocks"])
+        out["sub_workloads"] = {}
+        for sub in SUB_WORKLOADS:
+            rec = run_probe_workload(sub, args, env, sub_steps, sub_warm, 0, False,
+                                     tau_sweep=(0.80, 0.90, 0.95) if sub == "bert_base" else ())
+            out["sub_workloads"][sub] = brief(rec)
+    if rank == 0:
+        print(json.dumps(out))
     if dist is not None:
         dist.destroy_process_group()
 
 
-def run_scan_stress(args):
-    """Bank-scan stress: d_model = fp_dim = 1024, precomputed bf16 fingerprints, top-1 + threshold 0.9."""
+def run_scan_stress(args, steps=None, warmup=None):
+    """Bank-scan stress: d_model = fp_dim = 1024, precomputed bf16 fingerprints, top-1 + threshold 0.9.
+    Returns the record."""
     from paper_2512_16843_b200 import binding as L
     from paper_2512_16843_b200 import synth
     L.lib()
     if not torch.cuda.is_available():
         raise SystemExit("bench.py needs a CUDA device (there is no CPU fallback)")
-    dev = torch.device("cuda", 0)
+    steps = args.steps if steps is None else steps
+    warmup = args.warmup if warmup is None else warmup
+    dev = torch.device("cuda", torch.cuda.current_device())
     N, B, k = args.bank, args.queries, 1024
     keys, q, src = synth.scan_stress(N, B, k, n_clusters=4096, spread=0.1, near_fraction=0.3, q_sigma=0.05,
                                      seed=synth.BASE_SEED + 4000, device=dev)
-    bank = L.Bank(capacity=N, seq_len=1, d_model=k, fp_dim=k, max_batch=B, store_act=0, tau=0.9)
+    bank = L.Bank(device=dev.index, capacity=N, seq_len=1, d_model=k, fp_dim=k, max_batch=B, store_act=0, tau=0.9)
     bufs = L.ProbeBuffers(B, k, dev)
-    for f in range(0, N, B):                             # fill through the library: tau 2 => every key inserts
+    # fill through the library (tau 2 => every key inserts); the commits choose their slots with the
+    # multi-block selection, timed here as well
+    bank.profile(True)
+    for f in range(0, N, B):
         c = min(B, N - f)
         bufs.fp[:c].copy_(keys[f:f + c])
         bank.probe_fp(bufs, c, tau=2.0)
         bank.commit(None, bufs)
     torch.cuda.synchronize()
+    fill = bank.profile_read()
+    bank.profile(False)
     assert bank.stats()["resident"] == N
     bufs.fp.copy_(q)
-    for _ in range(args.warmup):
+    for _ in range(warmup):
         bank.probe_fp(bufs, B)
     torch.cuda.synchronize()
-    sampler = ClockSampler(0)
+    sampler = ClockSampler(dev.index)
     sampler.start()
+    sampler.wait_ready()
+    sampler.mark()
     bank.profile(True)
-    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-    e0.record()
-    for _ in range(args.steps):
-        bank.probe_fp(bufs, B)
-    e1.record()
-    torch.cuda.synchronize()
+    ms, per_step = timed_steps(lambda: bank.probe_fp(bufs, B), steps, torch.cuda.synchronize)
     clocks = sampler.stop()
-    ms = e0.elapsed_time(e1)
     prof = bank.profile_read()
     scan_ms = prof["scan"][0] / prof["scan"][1]
     peaks, kind = measured_peaks()
@@ -465,25 +591,32 @@ def run_scan_stress(args):
     peak = peaks["bf16_tflops_sustained"] if capped else peaks["bf16_tflops"]
     H = int(bufs.counts[0])
     exp_hits = int((src >= 0).sum())
-    out = {"metric": METRIC, "value": B * args.steps / (ms * 1e-3), "unit": UNIT, "n_gpus": 1, "steps": args.steps,
-           "warmup": args.warmup, "ms_per_step": ms / args.steps, "higher_is_better": True, "scaling": "weak",
+    med, mn = median_min(per_step)
+    out = {"metric": METRIC, "value": B * steps / (ms * 1e-3), "unit": UNIT, "n_gpus": 1, "steps": steps,
+           "warmup": warmup, "ms_per_step": ms / steps, "ms_per_step_median": med, "ms_per_step_min": mn,
+           "higher_is_better": True, "scaling": "weak",
            "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
            "config": {"workload": f"bank-scan stress: {N} keys x {B} queries x fp_dim 1024 bf16, 4096 clusters "
                                   f"(spread 0.1), 30% near-duplicate queries, top-1 + tau 0.9, keys only",
                       "hits": H, "expected_hits": exp_hits, "l2": "key matrix %.0f MB per scan" % (N * k * 2 / 1e6)},
-           "gpu_launches": prof["scan"][1] + prof["rownorm"][1] + prof["decide"][1] + prof["touch"][1],
+           "gpu_launches": sum(v[1] for v in prof.values()),
            "roofline": {"kernel": "scan", "bound": "tensor", "achieved": ach, "peak": peak, "unit": "TFLOP/s",
                         "frac": ach / peak, "peak_kind": "of " + kind + (" sustained (power-capped run)" if capped else " burst"),
                         "frac_of_burst": ach / peaks["bf16_tflops"], "frac_of_sustained": ach / peaks["bf16_tflops_sustained"],
-                        "traffic": None, "ms_per_launch": scan_ms,
+                        "frac_of_nominal_2250": ach / 2250.0,
+                        "traffic": None, "ms_per_launch": scan_ms, "probe_ms_median": med, "probe_ms_min": mn,
                         "flops_per_launch": flops,
-                        "all_kernels": {n_: {"ms_per_launch": v[0] / v[1], "launches": v[1]} for n_, v in prof.items() if v[1]}},
+                        "all_kernels": {n_: {"ms_per_launch": v[0] / v[1], "launches": v[1]} for n_, v in prof.items() if v[1]},
+                        "fill_commit_kernels": {n_: {"ms_per_launch": v[0] / v[1], "launches": v[1]}
+                                                for n_, v in fill.items() if v[1] and n_ in ("select", "scatter", "decide")}},
            "clocks": clocks}
-    print(json.dumps(out))
     bank.close()
+    del keys, q, bufs
+    torch.cuda.empty_cache()
+    return out
 
 
-def run_gather_stress(args):
+def run_gather_stress(args, steps=None, warmup=None):
     """Second half of the bank-scan stress configuration: the gather of hit rows of 512 x 1024 bf16 activations
     (1 MiB each).  65,536 keys share an activation store of `--act-rows` rows (slot j uses row j mod act_rows:
     65,536 rows of 1 MiB would be 69 GB), and the 65,536 queries are probed 8,192 at a time."""
@@ -492,13 +625,15 @@ def run_gather_stress(args):
     L.lib()
     if not torch.cuda.is_available():
         raise SystemExit("bench.py needs a CUDA device (there is no CPU fallback)")
-    dev = torch.device("cuda", 0)
+    steps_req = args.steps if steps is None else steps
+    warmup = args.warmup if warmup is None else warmup
+    dev = torch.device("cuda", torch.cuda.current_device())
     N, k, n, act_rows = 65536, 1024, 512, args.act_rows
     Bq, chunk = 65536, 8192
     keys, q, src = synth.scan_stress(N, Bq, k, n_clusters=4096, spread=0.1, near_fraction=0.3, q_sigma=0.05,
                                      seed=synth.BASE_SEED + 4000, device=dev)
     # inverse norms of the keys from the library itself (the row-norm kernel of a keys-only bank)
-    tmp = L.Bank(capacity=N, seq_len=1, d_model=k, fp_dim=k, max_batch=N, store_act=0, tau=2.0)
+    tmp = L.Bank(device=dev.index, capacity=N, seq_len=1, d_model=k, fp_dim=k, max_batch=N, store_act=0, tau=2.0)
     tb = L.ProbeBuffers(N, k, dev)
     tb.fp.copy_(keys)
     tmp.probe_fp(tb, N)
@@ -506,7 +641,7 @@ def run_gather_stress(args):
     rb = tb.rq.clone()
     tmp.close()
     del tb
-    bank = L.Bank(capacity=N, seq_len=n, d_model=k, fp_dim=k, max_batch=chunk, act_rows=act_rows, tau=0.9)
+    bank = L.Bank(device=dev.index, capacity=N, seq_len=n, d_model=k, fp_dim=k, max_batch=chunk, act_rows=act_rows, tau=0.9)
     bank.import_(L.WHAT_FP, keys)
     bank.import_(L.WHAT_RB, rb)
     bank.import_(L.WHAT_VALID, torch.ones(N, dtype=torch.uint8))
@@ -528,22 +663,18 @@ def run_gather_stress(args):
             bank.probe_fp(bufs, chunk, h_out=h_out)
         return hits
 
-    for _ in range(max(1, args.warmup // 3)):
+    for _ in range(max(1, warmup // 3)):
         one_step()
     torch.cuda.synchronize()
-    steps = max(1, min(args.steps, 10))
-    sampler = ClockSampler(0)
+    steps = max(1, min(steps_req, 10))
+    sampler = ClockSampler(dev.index)
     sampler.start()
+    sampler.wait_ready()
+    sampler.mark()
     bank.profile(True)
     h0 = bank.stats()["hits"]
-    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-    e0.record()
-    for _ in range(steps):
-        one_step()
-    e1.record()
-    torch.cuda.synchronize()
+    ms, per_step = timed_steps(one_step, steps, torch.cuda.synchronize)
     clocks = sampler.stop()
-    ms = e0.elapsed_time(e1)
     prof = bank.profile_read()
     hits = (bank.stats()["hits"] - h0) / steps
     g_ms = prof["gather"][0] / prof["gather"][1]
@@ -551,8 +682,10 @@ def run_gather_stress(args):
     algo = hits / len(chunks) * row * 2                  # per launch: every hit row read once and written once
     peaks, kind = measured_peaks()
     ach = algo / (g_ms * 1e-3) / 1e9
+    med, mn = median_min(per_step)
     out = {"metric": METRIC, "value": Bq * steps / (ms * 1e-3), "unit": UNIT, "n_gpus": 1, "steps": steps,
-           "warmup": args.warmup, "ms_per_step": ms / steps, "higher_is_better": True, "scaling": "weak",
+           "warmup": warmup, "ms_per_step": ms / steps, "ms_per_step_median": med, "ms_per_step_min": mn,
+           "higher_is_better": True, "scaling": "weak",
            "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
            "config": {"workload": f"bank-scan stress, gather half: {N} keys x fp_dim 1024, activation store of {act_rows} rows "
                                   f"of 512 x 1024 bf16 (1 MiB, slot mod {act_rows}), {Bq} queries probed {chunk} at a time, "
@@ -561,12 +694,15 @@ def run_gather_stress(args):
                       "l2": "%.1f GB of hit rows per probe call" % (algo / 2e9)},
            "gpu_launches": sum(v[1] for v in prof.values()),
            "roofline": {"kernel": "gather", "bound": "hbm", "achieved": ach, "peak": peaks["hbm_gbs"], "unit": "GB/s",
-                        "frac": ach / peaks["hbm_gbs"], "peak_kind": "of " + kind, "traffic": None,
+                        "frac": ach / peaks["hbm_gbs"], "frac_of_nominal_8tbs": ach / NOMINAL_HBM_GBS,
+                        "peak_kind": "of " + kind, "traffic": None,
                         "ms_per_launch": g_ms, "algorithmic_bytes_per_launch": algo,
                         "all_kernels": {n_: {"ms_per_launch": v[0] / v[1], "launches": v[1]} for n_, v in prof.items() if v[1]}},
            "clocks": clocks}
-    print(json.dumps(out))
     bank.close()
+    del keys, q, bufs, h_out, chunks
+    torch.cuda.empty_cache()
+    return out
 
 
 def run_e2e(args):
@@ -702,8 +838,8 @@ def run_e2e(args):
         o.close()
 
 
-def ncu_traffic(kernel):
-    ent = NCU_TRAFFIC.get(kernel)
+def ncu_traffic(workload, kernel):
+    ent = NCU_TRAFFIC.get(workload, {}).get(kernel)
     if not ent:
         return None
     path = os.path.join(ROOT, "paper_2512_16843_b200", "csrc", ent["file"])
@@ -720,23 +856,59 @@ def blas_threads():
         return 1
 
 
-def cpu_baseline_from_gpu_state(banks, pool, proj, step, cfg, budget_s=15.0, max_layers=12, steps_per_layer=8):
+def host_cpu():
+    model = "unknown"
+    try:
+        for ln in open("/proc/cpuinfo"):
+            if ln.startswith("model name"):
+                model = ln.split(":", 1)[1].strip()
+                break
+    except OSError:
+        pass
+    return {"host_cpus": os.cpu_count(), "cpu_model": model, "blas_threads": blas_threads(),
+            "threads_note": "numpy: pooling, rounding and bookkeeping run on one thread; only the float64 "
+                            "matrix products use the BLAS pool"}
+
+
+def oracle_bank_from_gpu(O, L, gb, proj):
+    """An oracle bank with the configuration and the current contents of a GPU bank."""
+    d = gb.desc
+    bits = lambda t: t.detach().cpu().contiguous().view(torch.int16).numpy().view(np.uint16)
+    u32 = lambda t: t.detach().cpu().contiguous().numpy().view(np.uint32)
+    ob = O.Bank(capacity=d.capacity, seq_len=d.seq_len, d_model=d.d_model, fp_dim=d.fp_dim, act_rows=gb.act_rows,
+                tau=float(d.tau), cmp_ge=(d.cmp == L.GE), policy=int(d.policy), half_life_ticks=d.half_life_ticks or 8,
+                stale_floor_q8=d.stale_floor_q8 or 64, min_age_ticks=d.min_age_ticks or 4,
+                max_idle_ticks=d.max_idle_ticks or 32, proj=None if proj is None else bits(proj))
+    ob.fp = bits(gb.export(L.WHAT_FP))
+    ob.rb = gb.export(L.WHAT_RB).numpy().copy()
+    ob.valid = gb.export(L.WHAT_VALID).numpy().copy()
+    ob.last_use = u32(gb.export(L.WHAT_LAST_USE)).copy()
+    ob.insert_tick = u32(gb.export(L.WHAT_INSERT_TICK)).copy()
+    ob.hits = u32(gb.export(L.WHAT_HITS)).copy()
+    ob.m = u32(gb.export(L.WHAT_RATE)).copy()
+    ob.e_upd = u32(gb.export(L.WHAT_RATE_EPOCH)).copy()
+    ob.tick = int(gb.export(L.WHAT_TICK)[0])
+    ob.act = bits(gb.export(L.WHAT_ACT))
+    return ob
+
+
+def cpu_baseline_from_gpu_state(banks, pool, proj, step, cfg, budget_s=15.0, max_layers=6, steps_per_layer=4):
     """The oracle, as it stands, on the same batches and the banks' current contents."""
     from oracle import llmcache_oracle as O
     from paper_2512_16843_b200 import binding as L
     from paper_2512_16843_b200 import synth
-    from tests import parity_util as U
     Lyr, B, P = cfg["layers"], cfg["batch"], cfg["pool_batches"]
+    f32_in = cfg.get("hidden") == "f32"
     done, t_total = 0, 0.0
     for l in range(min(Lyr, max_layers)):
-        ob = U.oracle_bank_like(banks[l], proj, None)
-        U.pull_state(banks[l], ob, with_act=True)
+        ob = oracle_bank_from_gpu(O, L, banks[l], proj)
         mo = np.zeros((B, ob.seq_len * ob.d_model), dtype=np.uint16)
         h_out = np.zeros((B, ob.seq_len * ob.d_model), dtype=np.uint16)
         for s in range(steps_per_layer):                 # successive batches of the rotation, same bank
-            h = synth.bf16_bits(pool[(step + s + 2 * l) % P])
+            hb = pool[(step + s + 2 * l) % P]
+            h = hb.cpu().numpy() if f32_in else synth.bf16_bits(hb)
             t0 = time.perf_counter()
-            pr = O.probe(ob, h, "bf16", h_out=h_out)
+            pr = O.probe(ob, h, "f32" if f32_in else "bf16", h_out=h_out)
             O.commit(ob, pr, mo[:len(pr.miss_idx)], h_out)
             t_total += time.perf_counter() - t0
             done += 1
@@ -745,37 +917,60 @@ def cpu_baseline_from_gpu_state(banks, pool, proj, step, cfg, budget_s=15.0, max
         del ob
         if t_total > budget_s:
             break
-    return {"value": done * B / t_total, "unit": UNIT, "cores": blas_threads(), "kind": "oracle",
-            "sample": f"{done} layer-batches of {B} sequences (probe + commit) out of the {Lyr}-layer rotation, "
-                      f"{t_total:.1f} s of CPU time; numpy, float64"}
+    out = {"value": done * B / t_total, "unit": UNIT, "cores": blas_threads(), "kind": "oracle",
+           "sample": f"{done} layer-batches of {B} sequences (probe + commit) out of the {Lyr}-layer rotation, "
+                     f"{t_total:.1f} s of CPU time; numpy, float64"}
+    out.update(host_cpu())
+    return out
+
+
+REF_SLICE = 128                                          # sequences of one reference step
 
 
 def run_reference(args):
-    """Times the CPU oracle on the same workload shape; each step is one layer's batch (a bounded sample)."""
+    """Times the CPU oracle on the headline workload's shape.  Each step is the probe + commit of one layer's
+    bank for REF_SLICE sequences of a batch (a bounded sample of the 24-layer, 512-sequence step)."""
     rank = int(os.environ.get("RANK", "0"))
     if rank != 0:
         return
     from oracle import llmcache_oracle as O
     from paper_2512_16843_b200 import synth
-    d, n, B, N, k = (CFG[x] for x in ("d_model", "seq_len", "batch", "bank", "fp_dim"))
+    name = HEADLINE if args.workload == "all" else args.workload
+    if name not in WORKLOADS or WORKLOADS[name].get("kind") != "cluster":
+        name = HEADLINE
+    cfg = WORKLOADS[name]
+    d, n, B, N, k, C = (cfg[x] for x in ("d_model", "seq_len", "batch", "bank", "fp_dim", "centres"))
+    S = min(REF_SLICE, B)
     seed = synth.BASE_SEED + 2000
-    wl = synth.TokenWorkload(CFG["vocab"], n, d, seed, "cpu")
-    seeds_tok = wl.tokens(CFG["n_seeds"], seed + 5)
     proj = synth.projection(d, k, seed + 6, "cpu")
-    ob = O.Bank(capacity=N, seq_len=n, d_model=d, fp_dim=k, tau=CFG["tau"], proj=synth.bf16_bits(proj))
-    acts = np.zeros((B, n * d), dtype=np.uint16)
-    h_out = np.zeros((B, n * d), dtype=np.uint16)
-    warm_tok = [torch.cat([seeds_tok, wl.tokens(B - CFG["n_seeds"], seed + 7)])]
-    warm_tok += [wl.tokens(B, seed + 20 + i) for i in range(1, N // B)]
-    for tok in warm_tok:
-        pr = O.probe(ob, synth.bf16_bits(wl.hidden(tok)), "bf16")
+    ob = O.Bank(capacity=N, seq_len=n, d_model=d, fp_dim=k, tau=cfg["tau"], proj=synth.bf16_bits(proj),
+                policy=O.POLICY_LRU_STALENESS)
+    centres = synth.randn((C, n, d), seed + 1, "cpu", torch.bfloat16)
+    g = torch.Generator().manual_seed(seed + 2)
+    n_near = int(round(S * cfg["near_fraction"]))
+
+    def batch(i):                                        # generated outside the timed part
+        if i >= 0:                                       # the centres drift between measured batches
+            for c0 in range(0, C, 64):
+                centres[c0:c0 + 64] = (centres[c0:c0 + 64].float()
+                                       + synth.randn((min(64, C - c0), n, d), seed + 700000 + 10 * i + c0, "cpu",
+                                                     scale=cfg["drift"])).to(torch.bfloat16)
+        pick = torch.randint(0, C, (n_near,), generator=g)
+        near = (centres[pick].float() + synth.randn((n_near, n, d), seed + 1000 * (i + 1), "cpu", scale=cfg["noise"]))
+        junk = synth.randn((S - n_near, n, d), seed + 500000 + i, "cpu")
+        h = torch.cat([near, junk])[synth.shuffled(S, seed + 600000 + i, "cpu")].to(torch.bfloat16)
+        return synth.bf16_bits(h)
+
+    acts = np.zeros((S, n * d), dtype=np.uint16)
+    h_out = np.zeros((S, n * d), dtype=np.uint16)
+    for i in range(N // S):                              # fill the bank
+        pr = O.probe(ob, batch(-1 - i), "bf16")
         O.commit(ob, pr, acts[:len(pr.miss_idx)])
     total = args.warmup + args.steps
     hits = 0
     t_timed = 0.0
     for i in range(total):
-        hb = build_batches(wl, seeds_tok, 1, seed + 1000 + 10 * i, "cpu")[0]      # generated outside the timed part
-        h = synth.bf16_bits(hb)
+        h = batch(i)
         t0 = time.perf_counter()
         pr = O.probe(ob, h, "bf16", h_out=h_out)
         O.commit(ob, pr, acts[:len(pr.miss_idx)], h_out)
@@ -783,17 +978,15 @@ def run_reference(args):
         if i >= args.warmup:
             t_timed += dt
             hits += int(pr.hit.sum())
-    value = B * args.steps / t_timed
-    cores = blas_threads()
+    value = S * args.steps / t_timed
+    cpu = {"value": value, "unit": UNIT, "cores": blas_threads(), "kind": "oracle",
+           "sample": f"one layer's bank x {S} sequences of a batch per step (probe + commit); numpy, float64"}
+    cpu.update(host_cpu())
     out = {"impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus,
            "steps": args.steps, "warmup": args.warmup, "ms_per_step": 1e3 * t_timed / args.steps,
            "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
-           "config": {"workload": "BERT-base-shaped encoder: bank of 2048 entries (bf16 384x768), batch 256 x "
-                                  "seq_len 384, d_model 768, fp_dim 256 (projected), tau 0.90, 60% token-level edits "
-                                  "of 64 seeds", "step": "probe + commit of one layer's batch (bounded sample of the "
-                                  "12-layer step)", "hit_fraction": hits / float(B * args.steps)},
-           "cpu_baseline": {"value": value, "unit": UNIT, "cores": cores, "kind": "oracle",
-                            "sample": "one layer x the full batch of 256 sequences per step; numpy, float64"},
+           "config": config_of(name, cfg, 1), "observed": {"hit_fraction": hits / float(S * args.steps)},
+           "cpu_baseline": cpu,
            "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
            "gpu_launches": 0}
     print(json.dumps(out))
@@ -804,9 +997,11 @@ if __name__ == "__main__":
     if a.impl == "reference":
         run_reference(a)
     elif a.workload == "scan_stress":
-        run_scan_stress(a)
+        env = init_dist()
+        print(json.dumps(run_scan_stress(a)))
     elif a.workload == "gather_stress":
-        run_gather_stress(a)
+        env = init_dist()
+        print(json.dumps(run_gather_stress(a)))
     elif a.workload == "e2e_bert_base":
         run_e2e(a)
     else:

@@ -175,9 +175,9 @@ int llmcache_pool(llmcache_bank_t* bank, const void* h_in, uint32_t B, float* po
 int llmcache_fingerprint_pooled(llmcache_bank_t* bank, const float* pooled, uint32_t ld, uint32_t B,
                                 void* fp, float* rq, void* stream);
 
-/* Fingerprint for callers that must not allocate device memory.  (The paper has no counterpart:
- * this is a packaging variant of llmcache_fingerprint: the same arithmetic, run as two kernels whose
- * fp32 sums may be taken in another order, so results agree to rounding, not bit for bit.)
+/* Fingerprint for callers that must not allocate device memory.  (The paper has no counterpart: this
+ * is a packaging variant of llmcache_fingerprint.  It launches the same two kernels in the same shapes, so on
+ * one device its fp and rq are bit-identical to llmcache_fingerprint's.)
  *
  * Who needs it: code that runs after its host application has handed all device memory to its own
  * pool (an inference server that reserves the GPU at start-up, say), or inside a latency-critical
@@ -192,20 +192,26 @@ int llmcache_fingerprint_pooled(llmcache_bank_t* bank, const float* pooled, uint
  *   proj   device bf16 [d_model, fp_dim] or NULL (then fp_dim == d_model);  center  device f32 [d_model] or NULL
  *   fp     device bf16 [B, fp_dim] out;  rq  device f32 [B] out
  * Limits: same shape rules as a bank, and the partial sums must fit: (B + 3 * G) * d_model <=
- * LLMCACHE_FINGERPRINT_STATIC_MAX_FLOATS is always enough, where G <= min(4 * SM count, 640) is the number
- * of blocks of the pooling pass.  A larger call is refused with LLMCACHE_ERR_SHAPE before anything is
- * launched; llmcache_fingerprint_static_error() then holds the sizes.
+ * LLMCACHE_FINGERPRINT_STATIC_MAX_FLOATS is always enough, where G <= min(SM count, 640) is the number
+ * of blocks of the pooling pass (one per SM).  A larger call is refused with LLMCACHE_ERR_SHAPE before
+ * anything is launched; llmcache_fingerprint_static_error() then holds the sizes.
  * The first call on each device looks up the array's device address and sets a kernel attribute; make
- * that first call outside any stream capture.  All calls share the one array and it keeps whatever
- * the previous call left there (nothing in it needs to start at zero: each call overwrites what it
- * reads).  Two calls that may overlap on the GPU -- different streams, or different threads -- race
- * on it: serialise them. */
+ * that first call outside any stream capture.  The address is cached per device for the life of the
+ * process: after a cudaDeviceReset the cached address is stale and this entry point must not be used
+ * on that device again.  All calls share the one array and it keeps whatever the previous call left
+ * there (nothing in it needs to start at zero: each call overwrites what it reads).  Two calls that may
+ * overlap on the GPU -- different streams, or different threads -- race on it: serialise them.
+ * Every device-side wait of the two kernels is bounded; llmcache_fingerprint_static_status() tells
+ * whether one ever ran out (the outputs of that call are then not valid). */
 #define LLMCACHE_FINGERPRINT_STATIC_MAX_FLOATS (2u * 1024u * 1024u)
 int llmcache_fingerprint_static(const void* h_in, uint32_t hidden_dtype, uint32_t B, uint32_t seq_len,
                                 uint32_t d_model, uint32_t fp_dim, const void* proj, const float* center,
                                 void* fp, float* rq, void* stream);
 /* Text describing why the last llmcache_fingerprint_static call of this thread failed ("" if it did not). */
 const char* llmcache_fingerprint_static_error(void);
+/* Sticky device-side status of llmcache_fingerprint_static on the current device: LLMCACHE_OK, or
+ * LLMCACHE_ERR_TIMEOUT once a bounded wait of one of its kernels has expired.  Synchronises the device. */
+int llmcache_fingerprint_static_status(void);
 
 /* Lookup and reuse for one batch (Sec. III-C, Sec. IV-A case equation,
  * Algorithm 1 "if exists (f',h') with sim > tau then h_l <- h'").
@@ -218,7 +224,8 @@ const char* llmcache_fingerprint_static_error(void);
 int llmcache_probe(llmcache_bank_t* bank, const void* h_in, uint32_t B, float tau,
                    void* h_out, llmcache_probe_io* io, void* stream);
 
-/* Lookup by SimHash codes (Sec. III-A, IV-B: "SimHash ... compact and comparable vectors"): the code of a
+/* Lookup by SimHash codes (Sec. III-A and the dimensionality-reduction step of Sec. IV-B, which names SimHash
+ * as one way to shorten the fingerprint): the code of a
  * fingerprint is the sign bit of each projected component (the projection matrix is the random-hyperplane
  * matrix), k bits per key instead of 2k bytes.  The scan finds the occupied key nearest in Hamming distance
  * (ties: lowest slot); hit iff cos(pi * ham / k) > tau, i.e. ham < k * acos(tau) / pi; io->score receives
@@ -285,6 +292,17 @@ int llmcache_bank_profile_read(llmcache_bank_t* bank, uint32_t kernel_id, double
 /* Sticky device-side status (LLMCACHE_OK or LLMCACHE_ERR_TIMEOUT).  Synchronises the device. */
 int llmcache_bank_status(llmcache_bank_t* bank);
 
+/* Diagnostics for the failure path (the paper has no counterpart).  Every device-side wait of the library's
+ * kernels is bounded; when one runs out the kernel records LLMCACHE_ERR_TIMEOUT in the object's status word,
+ * lets its copies in flight land, releases its tensor memory and returns -- the CUDA context stays usable,
+ * the object's outputs and contents are no longer valid.  These calls let a test take that path without a
+ * fault: wait_limit_ns replaces the bound of every wait (0 => the built-in 2 s) and
+ * LLMCACHE_KNOB_PRODUCER_IDLE keeps the thread that feeds a kernel's shared-memory ring idle, so that the
+ * first wait of its consumers runs out.  They apply to the kernels launched for this object afterwards and
+ * stay set until changed.  Synchronises the device.  Not for production use. */
+#define LLMCACHE_KNOB_PRODUCER_IDLE 1u
+int llmcache_bank_debug_knobs(llmcache_bank_t* bank, uint64_t wait_limit_ns, uint32_t flags);
+
 /* ------------------------------------------------------------------------------------------------
  * Miss-path transformer layer f_l and the layer-wise caching loop.
  *
@@ -331,6 +349,8 @@ int llmcache_layer_forward(llmcache_layer_t* layer, const void* x, uint32_t n_se
                            void* out, void* stream);
 /* LLMCACHE_OK or LLMCACHE_ERR_TIMEOUT (a bounded device-side wait expired).  Synchronises the device. */
 int llmcache_layer_status(llmcache_layer_t* layer);
+/* As llmcache_bank_debug_knobs, for the layer's kernels. */
+int llmcache_layer_debug_knobs(llmcache_layer_t* layer, uint64_t wait_limit_ns, uint32_t flags);
 
 /* Algorithm 1 (LLMCache-Infer) for a batch of B sequences, without any host sync: for l = 1..n_layers,
  * probe banks[l] with the current hidden states (hits take the stored output), run layers[l] on the
@@ -349,8 +369,8 @@ int llmcache_infer_pooled(llmcache_bank_t** banks, llmcache_layer_t** layers, ui
                           uint32_t B, float tau, void* buf_a, void* buf_b, void* h_miss, void* miss_out,
                           llmcache_probe_io* io, float* pooled, void** h_final, void* stream);
 
-/* Divergence monitor (Sec. III-E: "tracking differences in successive outputs for a given fingerprint";
- * Sec. IV-D: "revalidates fingerprints").  Call after the commit of a probe, with that probe's h_in and io.
+/* Divergence monitor (Sec. III-E, divergence tracking: watch how much the output served for a fingerprint
+ * differs from a fresh computation; Sec. IV-D, the monitor that re-checks stored entries).  Call after the commit of a probe, with that probe's h_in and io.
  * For every stride-th hit (ascending batch order) the layer is recomputed on the sequence's input and
  * compared with the stored output it was served: rel = ||f_l(h) - h'|| / ||f_l(h)||.  Entries with
  * rel > bound are invalidated (not those re-inserted during the current tick).

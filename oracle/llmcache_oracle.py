@@ -396,7 +396,7 @@ def effective_rate(bank: Bank, j: int) -> int:
 
 
 def is_stale(bank: Bank, j: int) -> bool:
-    """Staleness class (Sec. IV-D "decayed match rates over time")."""
+    """Staleness class (Sec. IV-D: the staleness signal is a match rate that decays with time)."""
     return (bank.policy == POLICY_LRU_STALENESS
             and effective_rate(bank, j) < bank.stale_floor_q8
             and bank.tick - int(bank.insert_tick[j]) >= bank.min_age_ticks)
@@ -455,8 +455,8 @@ def commit(bank: Bank, pr: ProbeResult, miss_out: Optional[np.ndarray],
 
 
 def evict(bank: Bank, mode: int, slots=None) -> int:
-    """Refresh controller flush (Sec. III-E "temporal decay factors are used to
-    flush outdated fingerprints").  Returns the number of entries removed."""
+    """Refresh controller flush (Sec. III-E, time-based decay: entries that have gone unused or
+    unmatched for too long are dropped).  Returns the number of entries removed."""
     removed = 0
     for j in range(bank.capacity):
         if not bank.valid[j]:
@@ -478,7 +478,8 @@ def evict(bank: Bank, mode: int, slots=None) -> int:
 
 
 # --------------------------------------------------------------------------
-# SimHash fingerprints (Sec. III-A "MinHash or SimHash-based techniques"; Sec. IV-B "SimHash or PCA")
+# SimHash fingerprints (named in Sec. III-A among the hashing techniques and in Sec. IV-B as one of the two
+# ways to shorten the pooled vector)
 # --------------------------------------------------------------------------
 def simhash_bits(fp_bf16: np.ndarray) -> np.ndarray:
     """k-bit code of a fingerprint: bit c = sign bit of the projected component c (random-hyperplane

@@ -156,8 +156,8 @@ def infer(banks: List[O.Bank], layers: List[LayerWeights], h0_bits: np.ndarray, 
 
 def divergence_check(bank: O.Bank, w: LayerWeights, h_bits: np.ndarray, pr: O.ProbeResult, heads: int,
                      stride: int, bound: float, pre_ln=False, causal=False, tanh_gelu=False, round_bf16=False):
-    """Divergence monitor (Sec. III-E "tracking differences in successive outputs for a given fingerprint";
-    Sec. IV-D "revalidates fingerprints").  For every `stride`-th hit of the probe (in ascending batch
+    """Divergence monitor (Sec. III-E, divergence tracking of the outputs stored under a fingerprint;
+    Sec. IV-D, the monitor that re-checks stored entries).  For every `stride`-th hit of the probe (in ascending batch
     order) the layer is recomputed on that sequence's input and compared with the stored output it was
     served: rel = ||f_l(h) - h'||_2 / ||f_l(h)||_2.  An entry whose rel exceeds `bound` is invalidated,
     unless it was (re)inserted during the current tick.  Returns (list of (b, slot, rel), number invalidated)."""

@@ -35,8 +35,10 @@ EXPORTS = [
     "llmcache_layer_bytes", "llmcache_layer_create", "llmcache_layer_destroy", "llmcache_layer_forward",
     "llmcache_layer_status", "llmcache_infer", "llmcache_divergence_check", "llmcache_probe_simhash",
     "llmcache_pool", "llmcache_fingerprint_pooled", "llmcache_probe_pooled", "llmcache_bank_pool_out",
-    "llmcache_infer_pooled",
+    "llmcache_infer_pooled", "llmcache_fingerprint_static_status", "llmcache_bank_debug_knobs",
+    "llmcache_layer_debug_knobs",
 ]
+KNOB_PRODUCER_IDLE = 1
 FINGERPRINT_STATIC_MAX_FLOATS = 2 * 1024 * 1024
 KERNEL_NAMES = ["pool", "project", "rownorm", "scan", "decide", "touch", "gather", "select", "scatter", "evict",
                 "pool_finish"]
@@ -140,6 +142,9 @@ def lib():
         L.llmcache_fingerprint_static.argtypes = [vp, u32, u32, u32, u32, u32, vp, vp, vp, vp, vp]
         L.llmcache_fingerprint_static_error.restype = C.c_char_p
         L.llmcache_fingerprint_static_error.argtypes = []
+        L.llmcache_fingerprint_static_status.argtypes = []
+        L.llmcache_bank_debug_knobs.argtypes = [vp, C.c_uint64, u32]
+        L.llmcache_layer_debug_knobs.argtypes = [vp, C.c_uint64, u32]
         for name in EXPORTS:
             if name not in ("llmcache_abi_version", "llmcache_strerror", "llmcache_last_cuda_error",
                             "llmcache_fingerprint_static_error"):
@@ -293,6 +298,18 @@ def llmcache_bank_status(bank) -> int:
     return int(lib().llmcache_bank_status(bank))
 
 
+def llmcache_bank_debug_knobs(bank, wait_limit_ns: int, flags: int) -> None:
+    _check(lib().llmcache_bank_debug_knobs(bank, wait_limit_ns, flags), "llmcache_bank_debug_knobs")
+
+
+def llmcache_layer_debug_knobs(layer, wait_limit_ns: int, flags: int) -> None:
+    _check(lib().llmcache_layer_debug_knobs(layer, wait_limit_ns, flags), "llmcache_layer_debug_knobs")
+
+
+def llmcache_fingerprint_static_status() -> int:
+    return int(lib().llmcache_fingerprint_static_status())
+
+
 def llmcache_bank_profile(bank, enable: bool) -> None:
     _check(lib().llmcache_bank_profile(bank, 1 if enable else 0), "llmcache_bank_profile")
 
@@ -428,6 +445,9 @@ class Bank:
     def status(self) -> int:
         return llmcache_bank_status(self.handle)
 
+    def debug_knobs(self, wait_limit_ns: int = 0, flags: int = 0):
+        llmcache_bank_debug_knobs(self.handle, wait_limit_ns, flags)
+
     def profile(self, enable: bool):
         llmcache_bank_profile(self.handle, enable)
 
@@ -522,6 +542,9 @@ class Layer:
 
     def status(self) -> int:
         return llmcache_layer_status(self.handle)
+
+    def debug_knobs(self, wait_limit_ns: int = 0, flags: int = 0):
+        llmcache_layer_debug_knobs(self.handle, wait_limit_ns, flags)
 
     def close(self):
         if getattr(self, "handle", None):

@@ -84,7 +84,7 @@ Layout make_layout(const llmcache_bank_desc& d) {
   L.sort_key = take((size_t)L.sort_len * 8);
   L.sort_slot = take((size_t)L.sort_len * 4);
   L.stats = take(ST_COUNT * 8);
-  L.status = take(4);
+  L.status = take(16);                  // status word + three words of diagnostic knobs
   L.misc = take(64);
   L.blk_cnt = take(((size_t)d.max_batch + 1023) / 1024 * 8);
   L.sel_keys = take(N * 8);
@@ -585,6 +585,19 @@ int llmcache_bank_status(llmcache_bank_t* bk) {
     return LLMCACHE_ERR_CUDA;
   }
   return s ? LLMCACHE_ERR_TIMEOUT : LLMCACHE_OK;
+}
+
+int llmcache_bank_debug_knobs(llmcache_bank_t* bk, uint64_t wait_limit_ns, uint32_t flags) {
+  if (!bk) return LLMCACHE_ERR_ARG;
+  DeviceGuard guard(bk->desc.device);
+  if (!guard.ok) return LLMCACHE_ERR_CUDA;
+  uint32_t w[3] = {flags, (uint32_t)(wait_limit_ns & 0xFFFFFFFFull), (uint32_t)(wait_limit_ns >> 32)};
+  if (cudaDeviceSynchronize() != cudaSuccess ||
+      cudaMemcpy(bk->a.status + 1, w, sizeof(w), cudaMemcpyHostToDevice) != cudaSuccess) {
+    cudaGetLastError();
+    return LLMCACHE_ERR_CUDA;
+  }
+  return LLMCACHE_OK;
 }
 
 }  // extern "C"

@@ -1,5 +1,5 @@
-// Divergence monitor (Sec. III-E "tracking differences in successive outputs for a given fingerprint";
-// Sec. IV-D "revalidates fingerprints"): for every stride-th hit of the last probe the layer is run
+// Divergence monitor (Sec. III-E, divergence tracking of the outputs stored under a fingerprint;
+// Sec. IV-D, the monitor that re-checks stored entries): for every stride-th hit of the last probe the layer is run
 // again on that sequence's input and compared with the stored output it was served; entries whose
 // relative L2 difference exceeds a bound are invalidated.
 #include "llmcache_internal.cuh"

@@ -1,5 +1,5 @@
 // Replacement controller kernels (Sec. III-E, IV-D): the victim selection for inserts (routine in
-// select.cuh) and the explicit flushes ("temporal decay factors are used to flush outdated fingerprints").
+// select.cuh) and the explicit flushes (Sec. III-E: entries that have gone unused or unmatched for too long are dropped).
 #include "llmcache_internal.cuh"
 #include "select.cuh"
 

@@ -60,9 +60,9 @@ k_project(const __grid_constant__ CUtensorMap map_p, MeanSrc src, __nv_bfloat16*
   for (int i = 0; i < 2 * NT; ++i) vals[i] = 0.f;
   if (threadIdx.x >= PROJ_CONS) {
     asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
-    if (threadIdx.x == PROJ_CONS) {
+    if (threadIdx.x == PROJ_CONS && !producer_idle(status)) {
       uint32_t it = 0;
-      if (!proj_produce(m, S, &map_p, r0, nrows, blockIdx.x * 5u, it)) proj_drain(m, S, it, status);
+      if (!proj_produce(m, S, &map_p, r0, nrows, blockIdx.x * 5u, it, wait_limit(status))) proj_drain(m, S, it, status);
     }
     __syncwarp();
   } else {
@@ -324,8 +324,9 @@ namespace {
 
 // Partial sums of the pooling pass, [B, splits, d] floats.  8 MiB per GPU that loads the library.
 static __device__ __align__(256) float g_fp_static_scratch[LLMCACHE_FINGERPRINT_STATIC_MAX_FLOATS];
-// Set by the pooling kernel if one of its bounded waits ever expired (stays zero otherwise).
-static __device__ uint32_t g_fp_static_status;
+// Word 0 is set by the kernels if one of their bounded waits ever expired (stays zero otherwise); words 1-3
+// are the diagnostic knobs every status word carries, never set here.
+static __device__ __align__(16) uint32_t g_fp_static_status[4];
 
 constexpr int STATIC_MAX_DEVICES = 64;
 struct StaticDev { bool ready = false; float* scratch = nullptr; uint32_t* status = nullptr; int sm_count = 0; };
@@ -364,6 +365,23 @@ cudaError_t static_setup(int dev, StaticDev** out) {
 }  // namespace
 
 extern "C" const char* llmcache_fingerprint_static_error(void) { return g_static_err; }
+
+extern "C" int llmcache_fingerprint_static_status(void) {
+  int dev = -1;
+  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= STATIC_MAX_DEVICES) { cudaGetLastError(); return LLMCACHE_ERR_CUDA; }
+  uint32_t* sptr = nullptr;
+  {
+    std::lock_guard<std::mutex> lock(g_static_mu);
+    if (!g_static_dev[dev].ready) return LLMCACHE_OK;             // never used on this device
+    sptr = g_static_dev[dev].status;
+  }
+  uint32_t s = 0;
+  if (cudaDeviceSynchronize() != cudaSuccess || cudaMemcpy(&s, sptr, 4, cudaMemcpyDeviceToHost) != cudaSuccess) {
+    cudaGetLastError();
+    return LLMCACHE_ERR_CUDA;
+  }
+  return s ? LLMCACHE_ERR_TIMEOUT : LLMCACHE_OK;
+}
 
 extern "C" int llmcache_fingerprint_static(const void* h_in, uint32_t hidden_dtype, uint32_t B, uint32_t seq_len,
                                            uint32_t d_model, uint32_t fp_dim, const void* proj,

@@ -56,6 +56,7 @@ __device__ __forceinline__ void pool_phase(uint8_t* sm, const uint4* __restrict_
   volatile uint32_t* flags = head_flags(sm);
   auto full_bar = [&](uint32_t s) { return bar0 + 8 * s; };
   auto empty_bar = [&](uint32_t s) { return bar0 + 8 * (16 + s); };
+  const unsigned long long lim = wait_limit(status);
 
   if (threadIdx.x == 0) {
     for (uint32_t s = 0; s < stages; ++s) { mbar_init(full_bar(s), 1); mbar_init(empty_bar(s), cons_threads / 32); }
@@ -75,7 +76,7 @@ __device__ __forceinline__ void pool_phase(uint8_t* sm, const uint4* __restrict_
 
   if (threadIdx.x >= cons_threads) {
     // ---------------------------------------------------------------- producer (one thread)
-    if (threadIdx.x == cons_threads) {
+    if (threadIdx.x == cons_threads && !producer_idle(status)) {
       bool ok = true;
       while (r < r1 && ok) {
         unsigned long long seg_end = (unsigned long long)(b + 1) * n;
@@ -83,7 +84,7 @@ __device__ __forceinline__ void pool_phase(uint8_t* sm, const uint4* __restrict_
         while (r < seg_end) {
           const uint32_t rows = (uint32_t)min((unsigned long long)stage_rows, seg_end - r);
           const uint32_t s = it % stages, ph = (it / stages) & 1u;
-          if (!mbar_wait(empty_bar(s), ph ^ 1u, flags)) { ok = false; break; }
+          if (!mbar_wait(empty_bar(s), ph ^ 1u, flags, lim)) { ok = false; break; }
           mbar_expect_tx(full_bar(s), rows * row_bytes);
           bulk_load_1d(ring + s * stage_bytes, h + r * V, rows * row_bytes, full_bar(s));
           r += rows;
@@ -117,7 +118,7 @@ __device__ __forceinline__ void pool_phase(uint8_t* sm, const uint4* __restrict_
       while (r < seg_end) {
         const uint32_t rows = (uint32_t)min((unsigned long long)stage_rows, seg_end - r);
         const uint32_t s = it % stages, ph = (it / stages) & 1u;
-        if (!mbar_wait(full_bar(s), ph, flags)) { flags[0] = 1; atomicExch(status, 1u); }
+        if (!mbar_wait(full_bar(s), ph, flags, lim)) { flags[0] = 1; atomicExch(status, 1u); }
         if (active) {
           const uint32_t src = ring + s * stage_bytes + col * 16;
           for (uint32_t rr = rg; rr < rows; rr += R) {
@@ -260,7 +261,8 @@ __device__ __forceinline__ uint32_t proj_stage_at(uint32_t j, uint32_t nst, uint
 // Producer thread: the rows [r0, r0 + nrows) of P for one item, whole stages (rows past the item's end are
 // loaded too; the A operand is zero there).  `it` counts stages over all items of the block.
 __device__ __forceinline__ bool proj_produce(const ProjSmem& m, const ProjShape& S, const CUtensorMap* map,
-                                             uint32_t r0, uint32_t nrows, uint32_t rot, uint32_t& it) {
+                                             uint32_t r0, uint32_t nrows, uint32_t rot, uint32_t& it,
+                                             unsigned long long lim) {
   const uint32_t box_bytes = S.stage_rows * 128, stage_bytes = (S.k / 64) * box_bytes;
   for (uint32_t c0 = 0; c0 < nrows; c0 += S.a_rows) {
     const uint32_t crows = min(S.a_rows, nrows - c0);
@@ -268,7 +270,7 @@ __device__ __forceinline__ bool proj_produce(const ProjSmem& m, const ProjShape&
     for (uint32_t j = 0; j < nst; ++j, ++it) {
       const uint32_t ra = c0 + proj_stage_at(j, nst, rot) * S.stage_rows;
       const uint32_t s = it % S.stages, ph = (it / S.stages) & 1u;
-      if (!mbar_wait(m.empty_bar(s), ph ^ 1u, m.flags)) return false;
+      if (!mbar_wait(m.empty_bar(s), ph ^ 1u, m.flags, lim)) return false;
       mbar_expect_tx(m.full_bar(s), stage_bytes);
       for (uint32_t b = 0; b < S.k / 64; ++b)
         tma_load_2d(m.ring + s * stage_bytes + b * box_bytes, map, (int)(b * 64), (int)(r0 + ra), m.full_bar(s));
@@ -322,6 +324,7 @@ __device__ __forceinline__ void proj_consume(const ProjSmem& m, const ProjShape&
                                              uint32_t& it, uint32_t* __restrict__ status, float (&vals)[2 * NT]) {
   const uint32_t k = S.k, box_bytes = S.stage_rows * 128, stage_bytes = (k / 64) * box_bytes;
   const uint32_t warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const unsigned long long lim = wait_limit(status);
   const SeqBlocks* sq = reinterpret_cast<const SeqBlocks*>(m.seq_info);
   uint32_t more = 0;                                                 // most pooling blocks per sequence, less one
 #pragma unroll
@@ -403,7 +406,7 @@ __device__ __forceinline__ void proj_consume(const ProjSmem& m, const ProjShape&
       const uint32_t ra = proj_stage_at(j, nst, rot) * S.stage_rows;
       const uint32_t rows = min(S.stage_rows, crows - ra);
       const uint32_t s = it % S.stages, ph = (it / S.stages) & 1u;
-      if (!mbar_wait(m.full_bar(s), ph, m.flags)) { m.flags[0] = 1; atomicExch(status, 1u); }
+      if (!mbar_wait(m.full_bar(s), ph, m.flags, lim)) { m.flags[0] = 1; atomicExch(status, 1u); }
       if (col0 < k) {
         const uint32_t stage = m.ring + s * stage_bytes;
         for (uint32_t kk = 0; kk < rows; kk += PROJ_KSTEP) {

@@ -167,6 +167,17 @@ int llmcache_layer_status(llmcache_layer_t* L) {
   return s ? LLMCACHE_ERR_TIMEOUT : LLMCACHE_OK;
 }
 
+int llmcache_layer_debug_knobs(llmcache_layer_t* L, uint64_t wait_limit_ns, uint32_t flags) {
+  if (!L) return LLMCACHE_ERR_ARG;
+  uint32_t w[3] = {flags, (uint32_t)(wait_limit_ns & 0xFFFFFFFFull), (uint32_t)(wait_limit_ns >> 32)};
+  if (cudaDeviceSynchronize() != cudaSuccess ||
+      cudaMemcpy(L->status + 1, w, sizeof(w), cudaMemcpyHostToDevice) != cudaSuccess) {
+    cudaGetLastError();
+    return LLMCACHE_ERR_CUDA;
+  }
+  return LLMCACHE_OK;
+}
+
 int llmcache_infer(llmcache_bank_t** banks, llmcache_layer_t** layers, uint32_t n_layers, const void* h0, uint32_t B,
                    float tau, void* buf_a, void* buf_b, void* h_miss, void* miss_out, llmcache_probe_io* io,
                    void** h_final, void* stream) {

@@ -60,6 +60,7 @@ k_gemm_tc(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUt
   volatile uint32_t* abort_flag = misc + 1;
   volatile uint32_t* epi_go = misc + 2;
   const uint32_t warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const unsigned long long lim = wait_limit(status);
 
   // rows that hold data: all of them, or (sequences counted on the device) x (rows per sequence)
   uint32_t M = M_max;
@@ -89,13 +90,13 @@ k_gemm_tc(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUt
 
   uint32_t issued = 0;
   if (warp == 0) {
-    if (lane == 0) {                                   // ---- TMA producer
+    if (lane == 0 && !producer_idle(status)) {         // ---- TMA producer
       bool ok = true;
       for (uint32_t t = blockIdx.x; t < n_tiles && ok; t += gridDim.x) {
         const uint32_t mb = t / NB, nb = t % NB;       // consecutive blocks share the A tile in L2
         for (uint32_t kb = 0; kb < KB; ++kb) {
           const uint32_t s = issued % GSTAGES, ph = (issued / GSTAGES) & 1u;
-          if (!mbar_wait(empty_bar(s), ph ^ 1u, abort_flag)) { ok = false; break; }
+          if (!mbar_wait(empty_bar(s), ph ^ 1u, abort_flag, lim)) { ok = false; break; }
           mbar_expect_tx(full_bar(s), GA_BYTES + GB_BYTES);
           tma_load_2d(sA + s * GA_BYTES, &map_a, (int)(kb * GK), (int)(mb * GM), full_bar(s));
           tma_load_2d(sB + s * GB_BYTES, &map_w, (int)(kb * GK), (int)(nb * GN), full_bar(s));
@@ -110,12 +111,12 @@ k_gemm_tc(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUt
       uint32_t it = 0, tile = 0;
       for (uint32_t t = blockIdx.x; t < n_tiles && ok; t += gridDim.x, ++tile) {
         const uint32_t buf = tile & 1u, bph = (tile >> 1) & 1u;
-        if (!mbar_wait(tempty_bar(buf), bph ^ 1u, abort_flag)) { ok = false; break; }
+        if (!mbar_wait(tempty_bar(buf), bph ^ 1u, abort_flag, lim)) { ok = false; break; }
         tc_fence_after();
         const uint32_t d_tmem = tmem_base + buf * GN;
         for (uint32_t kb = 0; kb < KB; ++kb, ++it) {
           const uint32_t s = it % GSTAGES, ph = (it / GSTAGES) & 1u;
-          if (!mbar_wait(full_bar(s), ph, abort_flag)) { ok = false; break; }
+          if (!mbar_wait(full_bar(s), ph, abort_flag, lim)) { ok = false; break; }
           tc_fence_after();
           const uint64_t da = smem_desc_sw128(sA + s * GA_BYTES), db = smem_desc_sw128(sB + s * GB_BYTES);
 #pragma unroll
@@ -143,7 +144,7 @@ k_gemm_tc(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUt
       if (et == 0) epi_go[buf] = *abort_flag;
       asm volatile("bar.sync 1, 128;" ::: "memory");
       if (epi_go[buf]) break;
-      if (!mbar_wait(tfull_bar(buf), bph, abort_flag)) { *abort_flag = 1; atomicExch(status, 1u); }
+      if (!mbar_wait(tfull_bar(buf), bph, abort_flag, lim)) { *abort_flag = 1; atomicExch(status, 1u); }
       tc_fence_after();
       const uint32_t taddr = tmem_base + buf * GN + ((quarter * 32u) << 16);
       const uint32_t row = mb * GM + row_in_tile;

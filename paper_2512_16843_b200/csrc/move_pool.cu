@@ -110,10 +110,12 @@ k_move_pool(const MoveArgs a) {
 
   uint32_t i = (uint32_t)(r / n);                                     // sequence of the list
   uint32_t it = 0;
+  const unsigned long long lim = wait_limit(a.status);
 
   if (threadIdx.x == cons_threads) {
     // ------------------------------------------------------------------ producer (one thread)
     bool ok = true;
+    if (producer_idle(a.status)) r = r1;
     while (r < r1 && ok) {
       const unsigned long long seg0 = (unsigned long long)i * n;
       unsigned long long seg_end = seg0 + n;
@@ -122,7 +124,7 @@ k_move_pool(const MoveArgs a) {
       while (r < seg_end) {
         const uint32_t rows = (uint32_t)min((unsigned long long)stage_rows, seg_end - r);
         const uint32_t s = it % stages, ph = (it / stages) & 1u;
-        if (!mbar_wait(empty_bar(s), ph ^ 1u, flags)) { ok = false; break; }
+        if (!mbar_wait(empty_bar(s), ph ^ 1u, flags, lim)) { ok = false; break; }
         mbar_expect_tx(full_bar(s), rows * row_bytes);
         bulk_load_1d(ring + s * stage_bytes, src + (size_t)(r - seg0) * row_bytes, rows * row_bytes, full_bar(s));
         r += rows;
@@ -153,7 +155,7 @@ k_move_pool(const MoveArgs a) {
       while (r < seg_end) {
         const uint32_t rows = (uint32_t)min((unsigned long long)stage_rows, seg_end - r);
         const uint32_t s = it % stages, ph = (it / stages) & 1u;
-        if (!mbar_wait(full_bar(s), ph, flags)) { ok = false; break; }
+        if (!mbar_wait(full_bar(s), ph, flags, lim)) { ok = false; break; }
         const size_t off = (size_t)(r - seg0) * row_bytes;
         if (p.d0) bulk_store_1d(p.d0 + off, ring + s * stage_bytes, rows * row_bytes);
         if (p.d1) bulk_store_1d(p.d1 + off, ring + s * stage_bytes, rows * row_bytes);
@@ -200,7 +202,7 @@ k_move_pool(const MoveArgs a) {
       while (r < seg_end) {
         const uint32_t rows = (uint32_t)min((unsigned long long)stage_rows, seg_end - r);
         const uint32_t s = it % stages, ph = (it / stages) & 1u;
-        if (!mbar_wait(full_bar(s), ph, flags)) { flags[0] = 1; atomicExch(a.status, 1u); }
+        if (!mbar_wait(full_bar(s), ph, flags, lim)) { flags[0] = 1; atomicExch(a.status, 1u); }
         if (active) {
           const uint32_t src = ring + s * stage_bytes + col * 16;
           for (uint32_t rr = rg; rr < rows; rr += R) {

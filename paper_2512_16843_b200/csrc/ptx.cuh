@@ -8,6 +8,18 @@ namespace llmc {
 
 constexpr unsigned long long WAIT_LIMIT_NS = 2000000000ull;   // bound of every device-side wait
 
+// A status word is the first of four 32-bit words.  The other three are diagnostic knobs (zero in normal
+// use; see llmcache_bank_debug_knobs): word 1 bit 0 keeps the kernel's producer thread idle, so that a
+// consumer's wait runs out; words 2-3 (one 64-bit value) replace the wait limit, in nanoseconds.
+constexpr uint32_t KNOB_PRODUCER_IDLE = 1u;
+__device__ __forceinline__ unsigned long long wait_limit(const uint32_t* status) {
+  const unsigned long long v = *reinterpret_cast<const volatile unsigned long long*>(status + 2);
+  return v ? v : WAIT_LIMIT_NS;
+}
+__device__ __forceinline__ bool producer_idle(const uint32_t* status) {
+  return (*reinterpret_cast<const volatile uint32_t*>(status + 1) & KNOB_PRODUCER_IDLE) != 0u;
+}
+
 __device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
 
 __device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {

@@ -5,16 +5,19 @@
 // The scan is the dense contraction  S[b, j] = sum_c q[b, c] * f[j, c]  over bf16
 // fingerprints, both stored with the fingerprint dimension contiguous.  It runs
 // on the 5th-generation tensor cores:
-//   - one warp streams 128 x 64 query tiles and 256 x 64 key tiles into shared
+//   - one warp streams 128 x 64 query tiles and BN x 64 key tiles into shared
 //     memory with TMA (128-byte swizzle), four stages deep;
-//   - one thread issues tcgen05.mma (M = 128 queries, N = 256 slots, K = 16 per
-//     instruction) into one of two 256-column fp32 accumulators in tensor memory;
+//   - one thread issues tcgen05.mma (M = 128 queries, N = BN slots, K = 16 per
+//     instruction) into one of two BN-column fp32 accumulators in tensor memory;
 //   - four warps drain the other accumulator with tcgen05.ld: each thread owns
 //     one query row, scales by the slot's inverse norm, masks free slots to -inf
 //     and keeps a running (best score, lowest slot) in registers.
 // A block walks a run of key tiles for one query tile and publishes its result
 // with one 64-bit atomicMax per query (score in orderable form above, inverted
 // slot below, so that equal scores resolve to the lowest slot).
+// BN is 256 where the scan is a throughput problem; a bank of a few thousand keys
+// is cut into tiles of 128 or 64 keys instead, so that its few tiles spread over
+// more SMs and an epilogue thread walks fewer columns.
 //
 // Every wait on an mbarrier is bounded: on expiry the block records
 // LLMCACHE_ERR_TIMEOUT in the bank's status word, drains what it has in flight,
@@ -26,16 +29,16 @@
 namespace llmc {
 
 constexpr int BM = 128;            // queries per tile (MMA M)
-constexpr int BN = 256;            // slots per tile   (MMA N)
 constexpr int BK = 64;             // fingerprint elements per stage (128 bytes: one swizzle span)
 constexpr int STAGES = 4;
 constexpr int UMMA_K = 16;
 constexpr int SCAN_THREADS = 192;  // warp 0: TMA, warp 1: MMA + TMEM owner, warps 2..5: epilogue
 constexpr uint32_t A_BYTES = BM * BK * 2;   // 16 KB
-constexpr uint32_t B_BYTES = BN * BK * 2;   // 32 KB
-constexpr uint32_t TMEM_COLS = 512;         // two accumulators of 256 columns
 
+template <int BN>                  // slots per tile (MMA N): 64, 128 or 256
 struct ScanSmem {
+  static constexpr uint32_t B_BYTES = BN * BK * 2;              // 8 / 16 / 32 KB
+  static constexpr uint32_t TMEM_COLS = 2 * BN;                 // two accumulators of BN columns (a power of two >= 32)
   // offsets from the 1024-byte aligned base of dynamic shared memory
   static constexpr uint32_t A = 0;
   static constexpr uint32_t B = A + STAGES * A_BYTES;
@@ -43,13 +46,13 @@ struct ScanSmem {
   static constexpr uint32_t BAR = SB + 2 * BN * 8;              // full[4] empty[4] tfull[2] tempty[2]
   static constexpr uint32_t MISC = BAR + 16 * 8;                // tmem base, abort flag, epilogue go flags
   static constexpr uint32_t TOTAL = MISC + 64;
+  static constexpr uint32_t BYTES = TOTAL + 1024;               // slack for manual alignment
+  // kind::f16 instruction descriptor: fp32 accumulator, bf16 A and B, both K-major, M = 128, N = BN.
+  static constexpr uint32_t IDESC = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(BN >> 3) << 17) | ((uint32_t)(BM >> 4) << 24);
 };
-constexpr uint32_t SCAN_SMEM_BYTES = ScanSmem::TOTAL + 1024;    // slack for manual alignment
-
-// kind::f16 instruction descriptor: fp32 accumulator, bf16 A and B, both K-major, M = 128, N = 256.
-constexpr uint32_t IDESC = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(BN >> 3) << 17) | ((uint32_t)(BM >> 4) << 24);
 
 // ---------------------------------------------------------------------------
+template <int BN>
 __global__ void __launch_bounds__(SCAN_THREADS, 1)
 k_scan_tc(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CUtensorMap map_bank,
           const float* __restrict__ rb, const uint8_t* __restrict__ valid,
@@ -59,19 +62,22 @@ k_scan_tc(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CUt
   extern __shared__ uint8_t smem_raw[];
   const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;
   uint8_t* gbase = smem_raw + (base - smem_u32(smem_raw));
-  const uint32_t sA = base + ScanSmem::A, sB = base + ScanSmem::B;
-  float2* sb = reinterpret_cast<float2*>(gbase + ScanSmem::SB);
-  const uint32_t bar0 = base + ScanSmem::BAR;
+  using SM = ScanSmem<BN>;
+  constexpr uint32_t B_BYTES = SM::B_BYTES, TMEM_COLS = SM::TMEM_COLS, IDESC = SM::IDESC;
+  const uint32_t sA = base + SM::A, sB = base + SM::B;
+  float2* sb = reinterpret_cast<float2*>(gbase + SM::SB);
+  const uint32_t bar0 = base + SM::BAR;
   auto full_bar = [&](uint32_t s) { return bar0 + 8 * s; };
   auto empty_bar = [&](uint32_t s) { return bar0 + 8 * (STAGES + s); };
   auto tfull_bar = [&](uint32_t b) { return bar0 + 8 * (2 * STAGES + b); };
   auto tempty_bar = [&](uint32_t b) { return bar0 + 8 * (2 * STAGES + 2 + b); };
-  volatile uint32_t* misc = reinterpret_cast<volatile uint32_t*>(gbase + ScanSmem::MISC);
+  volatile uint32_t* misc = reinterpret_cast<volatile uint32_t*>(gbase + SM::MISC);
   volatile uint32_t* tmem_slot = misc + 0;
   volatile uint32_t* abort_flag = misc + 1;
   volatile uint32_t* epi_go = misc + 2;          // [2]
 
   const uint32_t warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const unsigned long long lim = wait_limit(status);
 
   if (threadIdx.x == 0) {
     for (uint32_t s = 0; s < STAGES; ++s) { mbar_init(full_bar(s), 1); mbar_init(empty_bar(s), 1); }
@@ -93,7 +99,7 @@ k_scan_tc(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CUt
   uint32_t issued = 0;                            // producer: stages armed so far
   if (warp == 0) {
     // ------------------------------------------------------------ TMA producer
-    if (lane == 0) {
+    if (lane == 0 && !producer_idle(status)) {
       bool ok = true;
       for (uint32_t u = blockIdx.x; u < n_units && ok; u += gridDim.x) {
         const uint32_t mb = u % MB, ch = u / MB;
@@ -101,7 +107,7 @@ k_scan_tc(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CUt
         for (uint32_t nb = nb0; nb < nb1 && ok; ++nb) {
           for (uint32_t kb = 0; kb < KB; ++kb) {
             const uint32_t s = issued % STAGES, ph = (issued / STAGES) & 1u;
-            if (!mbar_wait(empty_bar(s), ph ^ 1u, abort_flag)) { ok = false; break; }
+            if (!mbar_wait(empty_bar(s), ph ^ 1u, abort_flag, lim)) { ok = false; break; }
             mbar_expect_tx(full_bar(s), A_BYTES + B_BYTES);
             tma_load_2d(sA + s * A_BYTES, &map_q, (int)(kb * BK), (int)(mb * BM), full_bar(s));
             tma_load_2d(sB + s * B_BYTES, &map_bank, (int)(kb * BK), (int)(nb * BN), full_bar(s));
@@ -121,12 +127,12 @@ k_scan_tc(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CUt
         const uint32_t nb0 = ch * chunk_len, nb1 = min(NB, nb0 + chunk_len);
         for (uint32_t nb = nb0; nb < nb1 && ok; ++nb, ++tile) {
           const uint32_t buf = tile & 1u, bph = (tile >> 1) & 1u;
-          if (!mbar_wait(tempty_bar(buf), bph ^ 1u, abort_flag)) { ok = false; break; }
+          if (!mbar_wait(tempty_bar(buf), bph ^ 1u, abort_flag, lim)) { ok = false; break; }
           tc_fence_after();
           const uint32_t d_tmem = tmem_base + buf * BN;
           for (uint32_t kb = 0; kb < KB; ++kb, ++it) {
             const uint32_t s = it % STAGES, ph = (it / STAGES) & 1u;
-            if (!mbar_wait(full_bar(s), ph, abort_flag)) { ok = false; break; }
+            if (!mbar_wait(full_bar(s), ph, abort_flag, lim)) { ok = false; break; }
             tc_fence_after();
             const uint64_t da = smem_desc_sw128(sA + s * A_BYTES), db = smem_desc_sw128(sB + s * B_BYTES);
 #pragma unroll
@@ -163,7 +169,7 @@ k_scan_tc(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CUt
         if (et == 0) epi_go[buf] = *abort_flag;
         asm volatile("bar.sync 1, 128;" ::: "memory");
         if (epi_go[buf]) { stop = true; break; }  // uniform over the 128 threads
-        if (!mbar_wait(tfull_bar(buf), bph, abort_flag)) { *abort_flag = 1; atomicExch(status, 1u); }
+        if (!mbar_wait(tfull_bar(buf), bph, abort_flag, lim)) { *abort_flag = 1; atomicExch(status, 1u); }
         tc_fence_after();
         const uint32_t taddr = tmem_base + buf * BN + ((quarter * 32u) << 16);
 #pragma unroll 1
@@ -209,12 +215,14 @@ k_scan_tc(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CUt
 // ---------------------------------------------------------------------------
 cudaError_t setup_scan_kernels() {
   cudaError_t e = tensor_map_setup();
-  if (e != cudaSuccess) return e;
-  return cudaFuncSetAttribute(k_scan_tc, cudaFuncAttributeMaxDynamicSharedMemorySize, SCAN_SMEM_BYTES);
+  if (e == cudaSuccess) e = cudaFuncSetAttribute(k_scan_tc<256>, cudaFuncAttributeMaxDynamicSharedMemorySize, ScanSmem<256>::BYTES);
+  if (e == cudaSuccess) e = cudaFuncSetAttribute(k_scan_tc<128>, cudaFuncAttributeMaxDynamicSharedMemorySize, ScanSmem<128>::BYTES);
+  if (e == cudaSuccess) e = cudaFuncSetAttribute(k_scan_tc<64>, cudaFuncAttributeMaxDynamicSharedMemorySize, ScanSmem<64>::BYTES);
+  return e;
 }
 
-cudaError_t launch_scan(llmcache_bank* bk, const __nv_bfloat16* q, uint32_t B, cudaStream_t st) {
-  if (B == 0) return cudaSuccess;
+template <int BN>
+static cudaError_t launch_scan_bn(llmcache_bank* bk, const __nv_bfloat16* q, uint32_t B, cudaStream_t st) {
   const uint32_t N = bk->desc.capacity, k = bk->desc.fp_dim;
   alignas(64) CUtensorMap map_q, map_bank;
   if (!make_tensor_map_bf16(&map_q, q, B, k, BM) || !make_tensor_map_bf16(&map_bank, bk->a.fp, N, k, BN))
@@ -230,9 +238,18 @@ cudaError_t launch_scan(llmcache_bank* bk, const __nv_bfloat16* q, uint32_t B, c
   const uint32_t n_units = MB * chunks;
   const uint32_t grid = n_units < (uint32_t)bk->sm_count ? n_units : (uint32_t)bk->sm_count;
   ProfScope prof(bk, LLMCACHE_K_SCAN, st);
-  return launch_k(k_scan_tc, dim3(grid), dim3(SCAN_THREADS), SCAN_SMEM_BYTES, st, map_q, map_bank,
+  return launch_k(k_scan_tc<BN>, dim3(grid), dim3(SCAN_THREADS), ScanSmem<BN>::BYTES, st, map_q, map_bank,
                   (const float*)bk->a.rb, (const uint8_t*)bk->a.valid, bk->a.best, bk->a.status, B, N, KB, MB, NB,
                   chunk_len, n_units);
+}
+
+cudaError_t launch_scan(llmcache_bank* bk, const __nv_bfloat16* q, uint32_t B, cudaStream_t st) {
+  if (B == 0) return cudaSuccess;
+  // the widest key tile that still gives every SM a tile; small banks take narrower tiles
+  const unsigned long long MB = (B + BM - 1) / BM, N = bk->desc.capacity, sms = (unsigned long long)bk->sm_count;
+  if (MB * ((N + 255) / 256) >= sms) return launch_scan_bn<256>(bk, q, B, st);
+  if (MB * ((N + 127) / 128) >= sms) return launch_scan_bn<128>(bk, q, B, st);
+  return launch_scan_bn<64>(bk, q, B, st);
 }
 
 }  // namespace llmc

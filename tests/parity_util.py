@@ -146,7 +146,7 @@ def assert_position_means(pooled_gpu: np.ndarray, h_bits: np.ndarray, n: int, d:
 
 def lockstep_step(gb: L.Bank, ob: O.Bank, bufs: L.ProbeBuffers, h_dev: torch.Tensor, dtype: str,
                   miss_out_dev: torch.Tensor, tau=None, with_act=True, fp_only=False, do_commit=True,
-                  pooled_dev: torch.Tensor = None):
+                  pooled_dev: torch.Tensor = None, before_commit=None):
     """One probe (+ commit) on both sides from the same state.  Returns dict of counters.
     pooled_dev: the GPU side probes from these position means instead of pooling h_dev itself (the
     oracle always starts from the hidden states: the result is defined to be the same)."""
@@ -198,6 +198,10 @@ def lockstep_step(gb: L.Bank, ob: O.Bank, bufs: L.ProbeBuffers, h_dev: torch.Ten
     if not do_commit:
         return res
     M = len(gp.miss_idx)
+    if before_commit is not None:
+        # (stale-class slots, decayed entries) of the oracle's state as the commit will find it
+        stale_set, res["decayed"] = before_commit(ob)
+        was_valid = ob.valid.copy()
     h_out2 = h_out.clone()
     gb.commit(miss_out_dev, bufs, h_out=h_out2)
     torch.cuda.synchronize()
@@ -207,6 +211,8 @@ def lockstep_step(gb: L.Bank, ob: O.Bank, bufs: L.ProbeBuffers, h_dev: torch.Ten
     new_or = O.commit(ob, gp, mo, ho)
     new_gpu = bufs.new_slot[:M].cpu().numpy()
     assert np.array_equal(new_gpu, new_or), f"new_slot {new_gpu} vs {new_or}"
+    if before_commit is not None:
+        res["stale_victims"] = sum(1 for v in new_or.tolist() if v >= 0 and was_valid[v] and v in stale_set)
     if with_act:
         assert np.array_equal(bits(h_out2), ho), "scattered outputs"
     assert_state_equal(gb, ob, with_act=with_act, where="after commit")

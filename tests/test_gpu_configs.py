@@ -80,12 +80,12 @@ def test_config3_gpt2_small_shaped_layer():
     gb.close()
 
 
-@pytest.mark.parametrize("N", [65536, 262144])
+@pytest.mark.parametrize("N", [65536, 262144, 1048576])
 def test_config4_bank_scan_stress_sampled(N):
     """fp_dim 1024, 65,536 queries against N keys from 4,096 clusters, 30% near-duplicates, top-1 + tau 0.9.
     The oracle scores a seeded sample of the queries against the whole bank."""
     B, k = 65536, 1024
-    n_sample = 512 if N <= 65536 else 256
+    n_sample = 512 if N <= 65536 else 256 if N <= 262144 else 128
     keys, q, src = synth.scan_stress(N, B, k, n_clusters=4096, spread=0.1, near_fraction=0.3, q_sigma=0.05,
                                      seed=SEED + 4000, device=DEV)
     gb = L.Bank(capacity=N, seq_len=1, d_model=k, fp_dim=k, max_batch=B, store_act=0, tau=0.9)
@@ -156,39 +156,66 @@ def test_config4_gather_of_one_mebibyte_rows():
     gb.close()
 
 
-def test_config5_bert_large_shaped_churn_lockstep():
+@pytest.mark.parametrize("layer", [1, 12, 24])
+def test_config5_bert_large_shaped_churn_lockstep(layer):
     """d_model 1024, seq_len 512, batch 512, bank of 1024 with insert on miss and LRU + staleness eviction under
-    drifting cluster centres (shift 0.02 per batch), junk that never repeats and topic turnover; lock-step."""
+    drifting cluster centres (shift 0.02 per batch), junk that never repeats and topic turnover; lock-step.
+    Three separately seeded banks (standing for layers 1, 12 and 24 of the encoder), each for 24 batches = three
+    half-lives of the decayed match rate with the default policy constants; every batch is compared in full
+    (decisions, gathered rows, which slot each miss takes, every array of the bank).  With the default constants
+    the ~110 evictions per batch recycle every low-rate entry within about seven batches, before its rate has
+    halved three times, so rates are seen decayed but no entry lives long enough to turn stale; the third bank
+    therefore halves the rate every batch, which makes junk stale after four batches, and must take victims
+    from the stale class."""
     N, n, d, B, k = 1024, 512, 1024, 512, 256
     n_centres = 256
-    proj = synth.projection(d, k, SEED + 5006, DEV)
+    S = SEED + 97 * layer
+    proj = synth.projection(d, k, S + 5006, DEV)
     gb = L.Bank(capacity=N, seq_len=n, d_model=d, fp_dim=k, max_batch=B, hidden_dtype=L.BF16, proj=proj, tau=0.9,
-                policy=L.LRU_STALENESS)
+                policy=L.LRU_STALENESS, half_life_ticks=1 if layer == 24 else 0)
     ob = U.oracle_bank_like(gb, proj, None)
     bufs = L.ProbeBuffers(B, k, DEV)
-    centres = synth.randn((n_centres, n, d), SEED + 5000, DEV, torch.bfloat16)
-    g = torch.Generator().manual_seed(SEED + 5001)
+    centres = synth.randn((n_centres, n, d), S + 5000, DEV, torch.bfloat16)
+    g = torch.Generator().manual_seed(S + 5001)
     tot = dict(H=0, inserted=0, near_thr=0, near_tie=0)
-    steps = 6
+    steps = 24
+    stale_victims = 0
+    decayed_seen = 0
     for step in range(steps):
-        centres = (centres.float() + synth.randn(centres.shape, SEED + 5100 + step, DEV, scale=0.02)).to(torch.bfloat16)
+        centres = (centres.float() + synth.randn(centres.shape, S + 5100 + step, DEV, scale=0.02)).to(torch.bfloat16)
         for c in torch.randint(0, n_centres, (2,), generator=g).tolist():      # topic turnover
-            centres[c] = synth.randn((n, d), SEED + 5200 + 10 * step + c, DEV, torch.bfloat16)
+            centres[c] = synth.randn((n, d), S + 5200 + 10 * step + c, DEV, torch.bfloat16)
         n_near = int(B * 0.75)
         pick = torch.randint(0, n_centres, (n_near,), generator=g).to(DEV)
         h = torch.empty((B, n, d), dtype=torch.bfloat16, device=DEV)
         for i0 in range(0, n_near, 64):
             sl = slice(i0, min(n_near, i0 + 64))
-            h[sl] = (centres[pick[sl]].float() + synth.randn((sl.stop - sl.start, n, d), SEED + 5300 + 100 * step + i0,
+            h[sl] = (centres[pick[sl]].float() + synth.randn((sl.stop - sl.start, n, d), S + 5300 + 100 * step + i0,
                                                              DEV, scale=0.05)).to(torch.bfloat16)
-        h[n_near:] = synth.randn((B - n_near, n, d), SEED + 5400 + step, DEV, torch.bfloat16)
-        h = h[synth.shuffled(B, SEED + 5500 + step, DEV)].contiguous()
-        r = U.lockstep_step(gb, ob, bufs, h, "bf16", synth.activations(B, n, d, SEED + 5600 + step, DEV))
+        h[n_near:] = synth.randn((B - n_near, n, d), S + 5400 + step, DEV, torch.bfloat16)
+        h = h[synth.shuffled(B, S + 5500 + step, DEV)].contiguous()
+        r = U.lockstep_step(gb, ob, bufs, h, "bf16", synth.activations(B, n, d, S + 5600 + step, DEV),
+                            before_commit=lambda bank: stale_and_decayed(bank))
+        stale_victims += r["stale_victims"]
+        decayed_seen = max(decayed_seen, r["decayed"])
         for key in tot:
             tot[key] += r[key]
         del h
     st = gb.stats()
-    print("config5: %d steps, hits %d, inserted %d, evictions %d, near-threshold %d, near-tie %d"
-          % (steps, tot["H"], tot["inserted"], st["evictions"], tot["near_thr"], tot["near_tie"]))
+    print("config5 bank %d: %d steps, hits %d, inserted %d, evictions %d, stale-class victims %d, decayed entries (max) %d, "
+          "near-threshold %d, near-tie %d" % (layer, steps, tot["H"], tot["inserted"], st["evictions"], stale_victims,
+                                              decayed_seen, tot["near_thr"], tot["near_tie"]))
     assert st["evictions"] > 0 and tot["H"] > 0 and st["resident"] == N
+    if layer == 24:
+        assert stale_victims > 0, "no victim was ever taken from the stale class"
+    assert decayed_seen > 0, "no stored entry's match rate was ever seen decayed"
     gb.close()
+
+
+def stale_and_decayed(ob):
+    """From the oracle bank's state between a probe and its commit: the slots in the stale class, and how many
+    occupied entries carry a match rate that has decayed since it was last written."""
+    occ = np.flatnonzero(ob.valid)
+    stale = {int(j) for j in occ if O.is_stale(ob, int(j))}
+    decayed = sum(1 for j in occ if O.effective_rate(ob, int(j)) < int(ob.m[j]))
+    return stale, decayed

@@ -127,7 +127,8 @@ def test_probe_fp_path_and_act_rows_aliasing():
     gb.close()
 
 
-@pytest.mark.parametrize("N,k,B", [(20000, 1024, 1000), (3000, 64, 130), (70000, 128, 40), (513, 512, 257)])
+@pytest.mark.parametrize("N,k,B", [(20000, 1024, 1000), (3000, 64, 130), (70000, 128, 40), (513, 512, 257),
+                                   (8192, 256, 512), (9000, 192, 300)])
 def test_scan_many_tiles_and_runs(N, k, B):
     """Key counts and batch sizes that span many tensor-core tiles, several runs per block and ragged tails."""
     bank_fp, q, src = synth.scan_stress(N, B, k, n_clusters=64, seed=41 + k, device=DEV)

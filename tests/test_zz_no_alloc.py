@@ -1,19 +1,22 @@
-"""The allocation-free fingerprint entry point against the ordinary one.
+"""The allocation-free fingerprint entry point against the ordinary one and against the oracle.
 
 Some users of this library cannot let it allocate device memory: their host
 application has already given the whole GPU to its own memory pool, or they
 sit in a loop where the device-wide stall of cudaMalloc is unaffordable.  For
 them llmcache_fingerprint_static keeps its scratch in a fixed array inside the
 library.  This file checks, through the C ABI, that it returns what
-llmcache_fingerprint returns -- on two calls in a row, because the second call
-finds the array as the first one left it -- and that it refuses a batch that
-would not fit.  It is named to be collected last, so that a run stopping at the
+llmcache_fingerprint returns (bit for bit: both launch the same two kernels in
+the same shapes) and what the CPU oracle computes (within the fingerprint
+tolerance) -- on two calls in a row, because the second call finds the array
+as the first one left it --, that the second call leaves the amount of free
+device memory unchanged, and that it refuses a batch that would not fit.  It is named to be collected last, so that a run stopping at the
 first failure has already run every other test.
 """
 import numpy as np
 import pytest
 import torch
 
+from oracle import llmcache_oracle as O
 from paper_2512_16843_b200 import binding as L
 from paper_2512_16843_b200 import synth
 from tests import parity_util as U
@@ -22,19 +25,29 @@ pytestmark = pytest.mark.gpu
 DEV = "cuda"
 
 
-def _both(bank, h, dtype_code, n, d, k, proj, center):
+def _both(bank, h, dtype, dtype_code, n, d, k, proj, center, check_memory=False):
     B = h.shape[0]
     fp_a = torch.zeros((B, k), dtype=torch.bfloat16, device=DEV)
     rq_a = torch.zeros(B, dtype=torch.float32, device=DEV)
     fp_b = torch.full((B, k), 7.0, dtype=torch.bfloat16, device=DEV)
     rq_b = torch.full((B,), 7.0, dtype=torch.float32, device=DEV)
     L.llmcache_fingerprint(bank.handle, h, B, fp_a, rq_a)
+    torch.cuda.synchronize()
+    free_before = torch.cuda.mem_get_info()[0]
     L.llmcache_fingerprint_static(h, dtype_code, B, n, d, k, proj, center, fp_b, rq_b)
     torch.cuda.synchronize()
-    # same tolerance as the parity tests use for fingerprints (1e-3 relative over the vector, one bf16
-    # rounding step per element): the two entry points add the same fp32 terms, but not in the same order
-    # (the bank's runs as one persistent kernel, this one as two kernels that split the projection's rows)
-    flipped = U.compare_fingerprints(U.bits(fp_b), rq_b.cpu().numpy(), U.bits(fp_a), rq_a.cpu().numpy())
+    if check_memory:                       # the property the entry point exists for: it allocates nothing
+        assert torch.cuda.mem_get_info()[0] == free_before
+    assert L.llmcache_fingerprint_static_status() == L.OK
+    # the two entry points launch the same kernels with the same launch shapes: identical bits
+    assert torch.equal(fp_b.view(torch.int16), fp_a.view(torch.int16))
+    assert torch.equal(rq_b.view(torch.int32), rq_a.view(torch.int32))
+    # and against the oracle, with the tolerance the parity tests use for fingerprints (1e-3 relative over
+    # the vector, one bf16 rounding step per element)
+    host = h.cpu()
+    fp_o, rq_o = O.fingerprint(U.bits(host) if dtype == "bf16" else host.numpy(), dtype,
+                               None if proj is None else U.bits(proj), None if center is None else center.cpu().numpy())
+    flipped = U.compare_fingerprints(U.bits(fp_b), rq_b.cpu().numpy(), fp_o, rq_o)
     assert flipped < 0.01
 
 
@@ -50,8 +63,8 @@ def test_static_fingerprint_matches_the_bank_one_twice_in_a_row(dtype, n, d, k, 
     h1 = synth.randn((64, n, d), 21, DEV, tdt)
     h2 = synth.randn((37, n, d), 22, DEV, tdt)
     h2[5] = 0
-    _both(bank, h1, code, n, d, k, proj, center)
-    _both(bank, h2, code, n, d, k, proj, center)
+    _both(bank, h1, dtype, code, n, d, k, proj, center)
+    _both(bank, h2, dtype, code, n, d, k, proj, center, check_memory=True)
     bank.close()
 
 
