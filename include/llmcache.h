@@ -53,7 +53,9 @@ typedef enum {
   LLMCACHE_ERR_CUDA = -4,         /* a CUDA runtime/driver call failed (incl. no device) */
   LLMCACHE_ERR_STATE = -5,        /* calls out of order (commit without matching probe, ...) */
   LLMCACHE_ERR_TIMEOUT = -6,      /* a bounded device-side wait expired (sticky, see bank_status) */
-  LLMCACHE_ERR_UNSUPPORTED = -7   /* valid request this build does not serve */
+  LLMCACHE_ERR_UNSUPPORTED = -7,  /* valid request this build does not serve */
+  LLMCACHE_ERR_BOUNDS = -8        /* debug build only: a computed slot, row or batch index was out of range
+                                     (sticky, see bank_status); the access was skipped */
 } llmcache_status;
 
 enum { LLMCACHE_F32 = 0, LLMCACHE_BF16 = 1 };                 /* dtype of probe inputs h_in */
@@ -289,7 +291,8 @@ int llmcache_bank_stats(llmcache_bank_t* bank, llmcache_stats* host_out);
 int llmcache_bank_profile(llmcache_bank_t* bank, int enable);
 int llmcache_bank_profile_read(llmcache_bank_t* bank, uint32_t kernel_id, double* total_ms, uint64_t* launches);
 
-/* Sticky device-side status (LLMCACHE_OK or LLMCACHE_ERR_TIMEOUT).  Synchronises the device. */
+/* Sticky device-side status (LLMCACHE_OK, LLMCACHE_ERR_TIMEOUT, or LLMCACHE_ERR_BOUNDS in a debug build).
+ * Synchronises the device. */
 int llmcache_bank_status(llmcache_bank_t* bank);
 
 /* Diagnostics for the failure path (the paper has no counterpart).  Every device-side wait of the library's
@@ -302,6 +305,11 @@ int llmcache_bank_status(llmcache_bank_t* bank);
  * stay set until changed.  Synchronises the device.  Not for production use. */
 #define LLMCACHE_KNOB_PRODUCER_IDLE 1u
 int llmcache_bank_debug_knobs(llmcache_bank_t* bank, uint64_t wait_limit_ns, uint32_t flags);
+/* 1 if the library was built with -DLLMCACHE_DEBUG_BOUNDS, else 0.  That build range-checks every slot, row
+ * and batch index the row movers, the decision and the victim selection compute before using it; the first
+ * violation is recorded in the bank's status word (llmcache_bank_status -> LLMCACHE_ERR_BOUNDS) and the access
+ * is skipped.  (It stands in for a memory checker on systems where none can be run.) */
+int llmcache_debug_bounds_build(void);
 
 /* ------------------------------------------------------------------------------------------------
  * Miss-path transformer layer f_l and the layer-wise caching loop.

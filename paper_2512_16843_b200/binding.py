@@ -15,10 +15,11 @@ from typing import Optional
 import torch
 
 _HERE = os.path.dirname(os.path.abspath(__file__))
-LIB_PATH = os.path.join(_HERE, "libllmcache.so")
+# LLMCACHE_LIB selects another build of the same library (the range-checking debug build)
+LIB_PATH = os.environ.get("LLMCACHE_LIB") or os.path.join(_HERE, "libllmcache.so")
 
 OK = 0
-ERR_ARG, ERR_SHAPE, ERR_NOMEM, ERR_CUDA, ERR_STATE, ERR_TIMEOUT, ERR_UNSUPPORTED = -1, -2, -3, -4, -5, -6, -7
+ERR_ARG, ERR_SHAPE, ERR_NOMEM, ERR_CUDA, ERR_STATE, ERR_TIMEOUT, ERR_UNSUPPORTED, ERR_BOUNDS = -1, -2, -3, -4, -5, -6, -7, -8
 F32, BF16 = 0, 1
 GT, GE = 0, 1
 LRU, LRU_STALENESS = 0, 1
@@ -36,7 +37,7 @@ EXPORTS = [
     "llmcache_layer_status", "llmcache_infer", "llmcache_divergence_check", "llmcache_probe_simhash",
     "llmcache_pool", "llmcache_fingerprint_pooled", "llmcache_probe_pooled", "llmcache_bank_pool_out",
     "llmcache_infer_pooled", "llmcache_fingerprint_static_status", "llmcache_bank_debug_knobs",
-    "llmcache_layer_debug_knobs",
+    "llmcache_layer_debug_knobs", "llmcache_debug_bounds_build",
 ]
 KNOB_PRODUCER_IDLE = 1
 FINGERPRINT_STATIC_MAX_FLOATS = 2 * 1024 * 1024
@@ -143,6 +144,7 @@ def lib():
         L.llmcache_fingerprint_static_error.restype = C.c_char_p
         L.llmcache_fingerprint_static_error.argtypes = []
         L.llmcache_fingerprint_static_status.argtypes = []
+        L.llmcache_debug_bounds_build.argtypes = []
         L.llmcache_bank_debug_knobs.argtypes = [vp, C.c_uint64, u32]
         L.llmcache_layer_debug_knobs.argtypes = [vp, C.c_uint64, u32]
         for name in EXPORTS:
@@ -304,6 +306,10 @@ def llmcache_bank_debug_knobs(bank, wait_limit_ns: int, flags: int) -> None:
 
 def llmcache_layer_debug_knobs(layer, wait_limit_ns: int, flags: int) -> None:
     _check(lib().llmcache_layer_debug_knobs(layer, wait_limit_ns, flags), "llmcache_layer_debug_knobs")
+
+
+def llmcache_debug_bounds_build() -> bool:
+    return bool(lib().llmcache_debug_bounds_build())
 
 
 def llmcache_fingerprint_static_status() -> int:

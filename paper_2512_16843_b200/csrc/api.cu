@@ -151,6 +151,7 @@ const char* llmcache_strerror(int s) {
     case LLMCACHE_ERR_STATE: return "calls out of order";
     case LLMCACHE_ERR_TIMEOUT: return "bounded device wait expired";
     case LLMCACHE_ERR_UNSUPPORTED: return "not supported";
+    case LLMCACHE_ERR_BOUNDS: return "index out of range (debug build)";
     default: return "unknown status";
   }
 }
@@ -584,7 +585,16 @@ int llmcache_bank_status(llmcache_bank_t* bk) {
     cudaGetLastError();
     return LLMCACHE_ERR_CUDA;
   }
+  if (s & STATUS_BOUNDS) return LLMCACHE_ERR_BOUNDS;
   return s ? LLMCACHE_ERR_TIMEOUT : LLMCACHE_OK;
+}
+
+int llmcache_debug_bounds_build(void) {
+#ifdef LLMCACHE_DEBUG_BOUNDS
+  return 1;
+#else
+  return 0;
+#endif
 }
 
 int llmcache_bank_debug_knobs(llmcache_bank_t* bk, uint64_t wait_limit_ns, uint32_t flags) {

@@ -38,7 +38,7 @@ k_decide_compact(unsigned long long* __restrict__ best, const float* __restrict_
                  unsigned long long* __restrict__ stats,
                  uint32_t* __restrict__ last_use, uint32_t* __restrict__ hits_total, uint32_t* __restrict__ rate,
                  uint32_t* __restrict__ rate_epoch, uint32_t tick, uint32_t epoch,
-                 uint32_t sim_k, int32_t ham_max) {
+                 uint32_t sim_k, int32_t ham_max, uint32_t* __restrict__ status, uint32_t N) {
   griddep_sync();
   __shared__ uint32_t warp_tot[32];
   uint32_t hbase = 0, mbase = 0, ndegen = 0;
@@ -69,6 +69,7 @@ k_decide_compact(unsigned long long* __restrict__ best, const float* __restrict_
           sc = orderable_float((uint32_t)(pk >> 32)) * r;
           is_hit = cmp_ge ? (sc >= tau) : (sc > tau);
         }
+        if (!bounds_ok((uint32_t)sl < N, status, SITE_DECIDE)) is_hit = false;
       }
       if (!is_hit) sl = -1;
       hit[b] = is_hit ? 1 : 0;
@@ -135,7 +136,8 @@ k_decide_compact(unsigned long long* __restrict__ best, const float* __restrict_
 __global__ void __launch_bounds__(DEC_THREADS)
 k_decide_flags(unsigned long long* __restrict__ best, const float* __restrict__ rq, uint32_t B, float tau, int cmp_ge,
                uint8_t* __restrict__ hit, int32_t* __restrict__ slot, float* __restrict__ score,
-               uint32_t* __restrict__ hitcnt, uint32_t* __restrict__ blk_cnt, uint32_t sim_k, int32_t ham_max) {
+               uint32_t* __restrict__ hitcnt, uint32_t* __restrict__ blk_cnt, uint32_t sim_k, int32_t ham_max,
+               uint32_t* __restrict__ status, uint32_t N) {
   griddep_sync();
   __shared__ uint32_t warp_tot[32];
   __shared__ uint32_t sdeg;
@@ -163,6 +165,7 @@ k_decide_flags(unsigned long long* __restrict__ best, const float* __restrict__ 
         sc = orderable_float((uint32_t)(pk >> 32)) * r;
         is_hit = cmp_ge ? (sc >= tau) : (sc > tau);
       }
+      if (!bounds_ok((uint32_t)sl < N, status, SITE_DECIDE)) is_hit = false;
     }
     if (!is_hit) sl = -1;
     hit[b] = is_hit ? 1 : 0;
@@ -254,11 +257,11 @@ cudaError_t launch_decide(llmcache_bank* bk, uint32_t B, float tau, const float*
     return launch_k(k_decide_compact, dim3(1), dim3(DEC_THREADS), 0, st, bk->a.best, rq, B, tau,
                     (int)(bk->desc.cmp == LLMCACHE_GE), io->hit, io->slot, io->score, io->hit_idx, io->miss_idx,
                     io->counts, bk->a.hitcnt, bk->a.stats, bk->a.last_use, bk->a.hits, bk->a.rate, bk->a.rate_epoch,
-                    tick, epoch, sim_k, ham_max);
+                    tick, epoch, sim_k, ham_max, bk->a.status, bk->desc.capacity);
   const uint32_t nblk = (B + DEC_THREADS - 1) / DEC_THREADS;
   cudaError_t e = launch_k(k_decide_flags, dim3(nblk), dim3(DEC_THREADS), 0, st, bk->a.best, rq, B, tau,
                            (int)(bk->desc.cmp == LLMCACHE_GE), io->hit, io->slot, io->score, bk->a.hitcnt,
-                           bk->a.blk_cnt, sim_k, ham_max);
+                           bk->a.blk_cnt, sim_k, ham_max, bk->a.status, bk->desc.capacity);
   if (e != cudaSuccess) return e;
   bk->n_launches += 1;
   return launch_k(k_compact_touch, dim3(nblk), dim3(DEC_THREADS), 0, st, (const uint8_t*)io->hit,

@@ -65,6 +65,7 @@ cudaError_t launch_select_victims(llmcache_bank* bk, const llmcache_probe_io* io
   sel.g_val = bk->a.sort_slot;
   sel.sort_cap = bk->sort_len;
   sel.tally = bk->a.misc;
+  sel.status = bk->a.status;
   ProfScope prof(bk, LLMCACHE_K_SELECT, st);
   k_select_victims<<<1, SEL_THREADS, 0, st>>>(sel);
   return cudaGetLastError();

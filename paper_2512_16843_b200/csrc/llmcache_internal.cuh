@@ -169,6 +169,22 @@ inline cudaError_t launch_k(void (*kernel)(KArgs...), dim3 grid, dim3 block, siz
 }
 
 // ---- small device helpers ---------------------------------------------------
+// Range checks of computed indices (slots, batch indices, rows).  In the ordinary build they cost nothing
+// (the function is `true`).  A library built with -DLLMCACHE_DEBUG_BOUNDS evaluates them: the first violation
+// is recorded in the status word as STATUS_BOUNDS | site and the access is skipped, so that a wrong index
+// shows up as LLMCACHE_ERR_BOUNDS instead of a memory fault.
+constexpr uint32_t STATUS_TIMEOUT = 1u;
+constexpr uint32_t STATUS_BOUNDS = 0x100u;
+enum { SITE_GATHER_HIT = 1, SITE_GATHER_MISS, SITE_SCATTER, SITE_DECIDE, SITE_SELECT, SITE_MOVE };
+#ifdef LLMCACHE_DEBUG_BOUNDS
+__device__ __forceinline__ bool bounds_ok(bool ok, uint32_t* status, uint32_t site) {
+  if (!ok) atomicCAS(status, 0u, STATUS_BOUNDS | site);
+  return ok;
+}
+#else
+__device__ __forceinline__ bool bounds_ok(bool, uint32_t*, uint32_t) { return true; }
+#endif
+
 // First statement of every kernel: wait for the previous grid of the stream, then let the next one
 // be scheduled.
 __device__ __forceinline__ void griddep_sync() {

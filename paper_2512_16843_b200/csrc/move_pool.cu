@@ -41,6 +41,7 @@ struct MoveArgs {
   float* partial;            // [gridDim.x * Jmax, d]
   uint32_t* status;
   uint32_t act_rows, n, d, V, R, Jmax, stage_rows, stages, cons_threads;
+  uint32_t B, N;             // batch size and bank capacity (range checks of a debug build)
   // scatter only: the new entries' keys and metadata (Algorithm 1 "C_l[f_X] <- h_l"), written by the block
   // that moves the first row of a sequence; block 0 also reports the slots and adds up the counters
   const uint4* q_fp; const float* rq; uint32_t kv;                  // query fingerprints, 16-byte vectors per row
@@ -55,6 +56,13 @@ struct SeqPtrs { const char* src; char* d0; char* d1; };
 __device__ __forceinline__ SeqPtrs seq_ptrs(const MoveArgs& a, uint32_t i, size_t seq_bytes) {
   SeqPtrs p;
   const int32_t b = a.idx[i];
+  if (!bounds_ok(i < a.B && (uint32_t)b < a.B && (!a.slot || (uint32_t)a.slot[b] < a.N) &&
+                 (!a.new_slot || a.new_slot[i] == -1 || (uint32_t)a.new_slot[i] < a.N), a.status, SITE_MOVE)) {
+    p.src = a.src;                       // a readable row; nothing is written
+    p.d0 = nullptr;
+    p.d1 = nullptr;
+    return p;
+  }
   const size_t src_row = a.slot ? (size_t)((uint32_t)a.slot[b] % a.act_rows) : (size_t)i;
   p.src = a.src + src_row * seq_bytes;
   p.d0 = a.dst_out ? a.dst_out + (size_t)b * seq_bytes : nullptr;
@@ -300,6 +308,8 @@ cudaError_t launch_move_pool(llmcache_bank* bk, int which, const void* miss_out,
   a.count = (const uint32_t*)io->counts + which;
   a.partial = bk->a.move_partial + (size_t)which * move_partial_floats(D.max_batch, D.d_model);
   a.status = bk->a.status;
+  a.B = B;
+  a.N = bk->desc.capacity;
   a.act_rows = D.act_rows;
   a.n = D.seq_len; a.d = D.d_model; a.V = P.V; a.R = P.R; a.Jmax = P.Jmax;
   a.stage_rows = P.stage_rows; a.stages = P.stages; a.cons_threads = P.cons_threads;

@@ -54,7 +54,8 @@ __global__ void __launch_bounds__(COPY_THREADS, 6)
 k_gather(const char* __restrict__ act, uint32_t act_rows, char* __restrict__ h_out, size_t row_bytes,
          const char* __restrict__ h_in, char* __restrict__ h_miss, size_t in_row_bytes,
          const int32_t* __restrict__ slot, const int32_t* __restrict__ hit_idx,
-         const int32_t* __restrict__ miss_idx, const uint32_t* __restrict__ counts) {
+         const int32_t* __restrict__ miss_idx, const uint32_t* __restrict__ counts,
+         uint32_t* __restrict__ status, uint32_t B, uint32_t N) {
   griddep_sync();
   const uint32_t H = counts[0], M = counts[1];
   const uint32_t upr = (uint32_t)((row_bytes + COPY_UNIT - 1) / COPY_UNIT);
@@ -69,19 +70,23 @@ k_gather(const char* __restrict__ act, uint32_t act_rows, char* __restrict__ h_o
       const unsigned long long left = (u1 < n_hit ? u1 : n_hit) - u;
       const uint32_t w1 = (uint32_t)min((unsigned long long)upr, w0 + left);
       const int32_t b = hit_idx[i];
-      const uint32_t row = (uint32_t)slot[b] % act_rows;
-      const size_t off = (size_t)w0 * COPY_UNIT;
-      const uint32_t bytes = (uint32_t)(min(row_bytes, (size_t)w1 * COPY_UNIT) - off);
-      copy_bytes(act + (size_t)row * row_bytes + off, h_out + (size_t)b * row_bytes + off, nullptr, bytes);
+      if (bounds_ok(i < B && (uint32_t)b < B && (uint32_t)slot[b] < N, status, SITE_GATHER_HIT)) {
+        const uint32_t row = (uint32_t)slot[b] % act_rows;
+        const size_t off = (size_t)w0 * COPY_UNIT;
+        const uint32_t bytes = (uint32_t)(min(row_bytes, (size_t)w1 * COPY_UNIT) - off);
+        copy_bytes(act + (size_t)row * row_bytes + off, h_out + (size_t)b * row_bytes + off, nullptr, bytes);
+      }
       u += w1 - w0;
     } else {
       const unsigned long long jt = u - n_hit;
       const uint32_t m = (uint32_t)(jt / upr_in), w0 = (uint32_t)(jt - (unsigned long long)m * upr_in);
       const uint32_t w1 = (uint32_t)min((unsigned long long)upr_in, w0 + (u1 - u));
       const int32_t b = miss_idx[m];
-      const size_t off = (size_t)w0 * COPY_UNIT;
-      const uint32_t bytes = (uint32_t)(min(in_row_bytes, (size_t)w1 * COPY_UNIT) - off);
-      copy_bytes(h_in + (size_t)b * in_row_bytes + off, h_miss + (size_t)m * in_row_bytes + off, nullptr, bytes);
+      if (bounds_ok(m < B && (uint32_t)b < B, status, SITE_GATHER_MISS)) {
+        const size_t off = (size_t)w0 * COPY_UNIT;
+        const uint32_t bytes = (uint32_t)(min(in_row_bytes, (size_t)w1 * COPY_UNIT) - off);
+        copy_bytes(h_in + (size_t)b * in_row_bytes + off, h_miss + (size_t)m * in_row_bytes + off, nullptr, bytes);
+      }
       u += w1 - w0;
     }
   }
@@ -98,7 +103,7 @@ k_scatter_insert(const char* __restrict__ miss_out, char* __restrict__ h_out, ch
                  uint32_t* __restrict__ last_use, uint32_t* __restrict__ insert_tick, uint32_t* __restrict__ hits,
                  uint32_t* __restrict__ rate, uint32_t* __restrict__ rate_epoch, uint32_t tick, uint32_t epoch,
                  int32_t* __restrict__ new_slot_out, const uint32_t* __restrict__ tally,
-                 unsigned long long* __restrict__ stats) {
+                 unsigned long long* __restrict__ stats, uint32_t* __restrict__ status, uint32_t B, uint32_t N) {
   griddep_sync();
   const uint32_t M = counts[1];
   if (blockIdx.x == 0) {
@@ -120,6 +125,10 @@ k_scatter_insert(const char* __restrict__ miss_out, char* __restrict__ h_out, ch
     const uint32_t w1 = (uint32_t)min((unsigned long long)upr, w0 + (u1 - u));
     const int32_t b = miss_idx[m];
     const int32_t v = new_slot[m];
+    if (!bounds_ok(m < B && (uint32_t)b < B && (v == -1 || (uint32_t)v < N), status, SITE_SCATTER)) {
+      u += w1 - w0;
+      continue;
+    }
     const size_t off = (size_t)w0 * COPY_UNIT;
     const uint32_t bytes = (uint32_t)(min(row_bytes, (size_t)w1 * COPY_UNIT) - off);
     char* d0 = h_out ? h_out + (size_t)b * row_bytes + off : nullptr;
@@ -174,7 +183,7 @@ cudaError_t launch_gather(llmcache_bank* bk, const void* h_in, void* h_out,
                   (const char*)(want_hit ? bk->a.act : nullptr), D.act_rows, (char*)(want_hit ? h_out : nullptr), row_bytes,
                   (const char*)(want_miss ? h_in : nullptr), (char*)(want_miss ? io->h_miss : nullptr), in_row_bytes,
                   (const int32_t*)io->slot, (const int32_t*)io->hit_idx, (const int32_t*)io->miss_idx,
-                  (const uint32_t*)io->counts);
+                  (const uint32_t*)io->counts, bk->a.status, B, D.capacity);
 }
 
 cudaError_t launch_scatter_insert(llmcache_bank* bk, const void* miss_out, const llmcache_probe_io* io,
@@ -189,7 +198,7 @@ cudaError_t launch_scatter_insert(llmcache_bank* bk, const void* miss_out, const
                   (const int32_t*)bk->a.new_slot, (const uint32_t*)io->counts, (const uint4*)io->fp,
                   (const float*)io->rq, D.fp_dim, (uint4*)bk->a.fp, bk->a.rb, bk->a.valid, bk->a.last_use,
                   bk->a.insert_tick, bk->a.hits, bk->a.rate, bk->a.rate_epoch, (uint32_t)bk->tick, epoch,
-                  new_slot_out, (const uint32_t*)bk->a.misc, bk->a.stats);
+                  new_slot_out, (const uint32_t*)bk->a.misc, bk->a.stats, bk->a.status, B, D.capacity);
 }
 
 }  // namespace llmc

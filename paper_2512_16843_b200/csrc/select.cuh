@@ -169,6 +169,7 @@ struct SelectArgs {
   uint32_t* g_val;
   uint32_t sort_cap;
   uint32_t* tally;
+  uint32_t* status;
 };
 
 __device__ __forceinline__ void select_victims_block(const SelectArgs& A) {
@@ -341,7 +342,8 @@ __device__ __forceinline__ void select_victims_block(const SelectArgs& A) {
     }
     if (in_smem) bitonic_sort(skey, sval, pow2);
     else         bitonic_sort_large(skey, sval, pow2, s_key, s_val, SEL_SMEM);
-    for (uint32_t i = threadIdx.x; i < take; i += SEL_THREADS) victims[i] = (int32_t)sval[i];
+    for (uint32_t i = threadIdx.x; i < take; i += SEL_THREADS)
+      victims[i] = bounds_ok(sval[i] < N, A.status, SITE_SELECT) ? (int32_t)sval[i] : -1;
   }
   __syncthreads();
 

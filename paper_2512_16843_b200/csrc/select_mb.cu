@@ -42,6 +42,7 @@ struct SelMbArgs {
   unsigned long long* sort_key;
   uint32_t* sort_slot;
   uint32_t* tally;
+  uint32_t* status;
 };
 
 __device__ __forceinline__ unsigned long long ld_u64(const uint32_t* state, int word) {
@@ -271,7 +272,14 @@ __global__ void __launch_bounds__(MB_THREADS) k_selmb_assign(SelMbArgs A) {
   const bool ok = m < M && A.rq[A.miss_idx[m]] > 0.f;
   uint32_t tot;
   const uint32_t r = before + mb_rank(ok, warp_tot, tot);
-  if (m < M) A.new_slot[m] = (ok && r < take) ? (int32_t)A.sort_slot[r] : -1;
+  if (m < M) {
+    int32_t v = -1;
+    if (ok && r < take) {
+      const uint32_t sv = A.sort_slot[r];
+      if (bounds_ok(sv < A.N, A.status, SITE_SELECT)) v = (int32_t)sv;
+    }
+    A.new_slot[m] = v;
+  }
   if (blockIdx.x == 0 && threadIdx.x == 0) {
     A.tally[0] = take;
     A.tally[1] = A.state[SS_NOCC];
@@ -302,6 +310,7 @@ cudaError_t launch_select_victims_mb(llmcache_bank* bk, const llmcache_probe_io*
   A.sort_key = bk->a.sort_key;
   A.sort_slot = bk->a.sort_slot;
   A.tally = bk->a.misc;
+  A.status = bk->a.status;
   const uint32_t N = A.N;
   const uint32_t nblk_n = (N + MB_THREADS - 1) / MB_THREADS, nblk_b = (B + MB_THREADS - 1) / MB_THREADS;
   ProfScope prof(bk, LLMCACHE_K_SELECT, st);
