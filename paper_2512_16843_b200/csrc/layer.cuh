@@ -17,5 +17,12 @@ cudaError_t launch_layernorm(const __nv_bfloat16* x, const float* g, const float
                              cudaStream_t st);
 cudaError_t launch_attention(const __nv_bfloat16* qkv, __nv_bfloat16* out, uint32_t n, uint32_t d, uint32_t heads,
                              uint32_t seq_max, const uint32_t* m_seq_dev, int causal, cudaStream_t st);
+// Attention on the tcgen05 tensor cores; vt: scratch for the per-head transposes of V,
+// seq_max * heads * 64 rows of attention_vt_pitch(n) elements.
+cudaError_t setup_attention_kernel();
+uint32_t attention_vt_pitch(uint32_t n);
+cudaError_t launch_attention_tc(const __nv_bfloat16* qkv, __nv_bfloat16* vt, __nv_bfloat16* out, uint32_t* status,
+                                uint32_t n, uint32_t d, uint32_t heads, uint32_t seq_max, const uint32_t* m_seq_dev,
+                                int causal, cudaStream_t st);
 
 }  // namespace llmc

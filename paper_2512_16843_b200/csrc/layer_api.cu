@@ -11,7 +11,7 @@ struct llmcache_layer {
   int sm_count = 0;
   char* ws = nullptr;            // workspace
   bool owns_ws = false;
-  __nv_bfloat16 *qkv = nullptr, *a = nullptr, *t = nullptr, *y = nullptr, *f = nullptr;
+  __nv_bfloat16 *qkv = nullptr, *a = nullptr, *t = nullptr, *y = nullptr, *f = nullptr, *vt = nullptr;
   uint32_t* status = nullptr;    // device word: a bounded wait expired
 };
 
@@ -35,7 +35,8 @@ int check_layer_desc(const llmcache_layer_desc* d) {
 
 size_t layer_ws_bytes(const llmcache_layer_desc& d) {
   const size_t T = (size_t)d.max_seqs * d.seq_len;
-  return up256(T * 3 * d.d_model * 2) + 3 * up256(T * d.d_model * 2) + up256(T * d.ffn * 2) + WS_ALIGN;
+  const size_t vt = (size_t)d.max_seqs * d.d_model * attention_vt_pitch(d.seq_len) * 2;      // per-head transposes of V
+  return up256(T * 3 * d.d_model * 2) + 3 * up256(T * d.d_model * 2) + up256(T * d.ffn * 2) + up256(vt) + WS_ALIGN;
 }
 }  // namespace
 
@@ -83,10 +84,12 @@ int llmcache_layer_create(const llmcache_layer_desc* desc, llmcache_layer_t** la
     L->a = (__nv_bfloat16*)p; p += up256(T * d * 2);
     L->t = (__nv_bfloat16*)p; p += up256(T * d * 2);
     L->y = (__nv_bfloat16*)p; p += up256(T * d * 2);
-    L->f = (__nv_bfloat16*)p;
+    L->f = (__nv_bfloat16*)p; p += up256(T * desc->ffn * 2);
+    L->vt = (__nv_bfloat16*)p;
     e = cudaMemset(L->status, 0, WS_ALIGN);
   }
   if (e == cudaSuccess) e = setup_gemm_kernel();
+  if (e == cudaSuccess) e = setup_attention_kernel();
   if (e == cudaSuccess) e = cudaDeviceSynchronize();
   cudaSetDevice(prev);
   if (e != cudaSuccess) {
@@ -137,7 +140,7 @@ int llmcache_layer_forward(llmcache_layer_t* L, const void* x, uint32_t n_seqs, 
   };
   if (!D.pre_ln) {
     e = gemm(X, D.w_qkv, D.b_qkv, nullptr, L->qkv, 3 * d, d, LAYER_ACT_NONE);
-    if (e == cudaSuccess) e = launch_attention(L->qkv, L->a, n, d, D.heads, n_seqs, n_seqs_dev, D.causal, st);
+    if (e == cudaSuccess) e = launch_attention_tc(L->qkv, L->vt, L->a, L->status, n, d, D.heads, n_seqs, n_seqs_dev, D.causal, st);
     if (e == cudaSuccess) e = gemm(L->a, D.w_o, D.b_o, X, L->t, d, d, LAYER_ACT_NONE);
     if (e == cudaSuccess) e = ln(L->t, D.ln1_g, D.ln1_b, L->y);
     if (e == cudaSuccess) e = gemm(L->y, D.w_1, D.b_1, nullptr, L->f, D.ffn, d, act);
@@ -146,7 +149,7 @@ int llmcache_layer_forward(llmcache_layer_t* L, const void* x, uint32_t n_seqs, 
   } else {
     e = ln(X, D.ln1_g, D.ln1_b, L->y);
     if (e == cudaSuccess) e = gemm(L->y, D.w_qkv, D.b_qkv, nullptr, L->qkv, 3 * d, d, LAYER_ACT_NONE);
-    if (e == cudaSuccess) e = launch_attention(L->qkv, L->a, n, d, D.heads, n_seqs, n_seqs_dev, D.causal, st);
+    if (e == cudaSuccess) e = launch_attention_tc(L->qkv, L->vt, L->a, L->status, n, d, D.heads, n_seqs, n_seqs_dev, D.causal, st);
     if (e == cudaSuccess) e = gemm(L->a, D.w_o, D.b_o, X, L->t, d, d, LAYER_ACT_NONE);
     if (e == cudaSuccess) e = ln(L->t, D.ln2_g, D.ln2_b, L->y);
     if (e == cudaSuccess) e = gemm(L->y, D.w_1, D.b_1, nullptr, L->f, D.ffn, d, act);

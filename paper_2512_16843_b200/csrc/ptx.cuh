@@ -118,5 +118,9 @@ __device__ __forceinline__ uint64_t smem_desc_sw128(uint32_t saddr) {
 cudaError_t tensor_map_setup();
 // bf16 [rows, k] row-major matrix, boxes of box_rows x 64 elements, 128-byte swizzle, zero fill outside.
 bool make_tensor_map_bf16(CUtensorMap* map, const void* ptr, uint64_t rows, uint64_t k, uint32_t box_rows);
+// the same for rows that are `pitch` elements apart (pitch >= k, a multiple of 8); columns k..pitch-1 are not part
+// of the matrix (a box that reaches them is filled with zeros there)
+bool make_tensor_map_bf16_pitch(CUtensorMap* map, const void* ptr, uint64_t rows, uint64_t k, uint64_t pitch,
+                                uint32_t box_rows);
 
 }  // namespace llmc

@@ -21,9 +21,14 @@ cudaError_t tensor_map_setup() {
 }
 
 bool make_tensor_map_bf16(CUtensorMap* map, const void* ptr, uint64_t rows, uint64_t k, uint32_t box_rows) {
+  return make_tensor_map_bf16_pitch(map, ptr, rows, k, k, box_rows);
+}
+
+bool make_tensor_map_bf16_pitch(CUtensorMap* map, const void* ptr, uint64_t rows, uint64_t k, uint64_t pitch,
+                                uint32_t box_rows) {
   if (!g_encode) return false;
   const cuuint64_t dims[2] = {k, rows};
-  const cuuint64_t strides[1] = {k * 2};
+  const cuuint64_t strides[1] = {pitch * 2};
   const cuuint32_t box[2] = {64u, box_rows};
   const cuuint32_t estr[2] = {1, 1};
   return g_encode(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(ptr), dims, strides, box, estr,
