@@ -132,14 +132,16 @@ int llmcache_layer_forward(llmcache_layer_t* L, const void* x, uint32_t n_seqs, 
   const int sm = L->sm_count;
   cudaError_t e;
   auto gemm = [&](const __nv_bfloat16* a, const void* w, const float* bias, const __nv_bfloat16* res,
-                  __nv_bfloat16* o, uint32_t N, uint32_t K, uint32_t a_) {
-    return launch_gemm(a, (const __nv_bfloat16*)w, bias, res, o, L->status, T, N, K, n_seqs_dev, n, a_, sm, st);
+                  __nv_bfloat16* o, uint32_t N, uint32_t K, uint32_t a_, VtOut vt = VtOut{nullptr, 0, 0, 0}) {
+    return launch_gemm(a, (const __nv_bfloat16*)w, bias, res, o, L->status, T, N, K, n_seqs_dev, n, a_, sm, st, vt);
   };
+  // the V third of the q|k|v product is written transposed per head (what the attention kernel reads)
+  const VtOut vt_out{L->vt, 2 * d, attention_vt_pitch(n), D.heads};
   auto ln = [&](const __nv_bfloat16* in, const float* g, const float* b, __nv_bfloat16* o) {
     return launch_layernorm(in, g, b, o, T, d, n_seqs_dev, n, D.eps, sm, st);
   };
   if (!D.pre_ln) {
-    e = gemm(X, D.w_qkv, D.b_qkv, nullptr, L->qkv, 3 * d, d, LAYER_ACT_NONE);
+    e = gemm(X, D.w_qkv, D.b_qkv, nullptr, L->qkv, 3 * d, d, LAYER_ACT_NONE, vt_out);
     if (e == cudaSuccess) e = launch_attention_tc(L->qkv, L->vt, L->a, L->status, n, d, D.heads, n_seqs, n_seqs_dev, D.causal, st);
     if (e == cudaSuccess) e = gemm(L->a, D.w_o, D.b_o, X, L->t, d, d, LAYER_ACT_NONE);
     if (e == cudaSuccess) e = ln(L->t, D.ln1_g, D.ln1_b, L->y);
@@ -148,7 +150,7 @@ int llmcache_layer_forward(llmcache_layer_t* L, const void* x, uint32_t n_seqs, 
     if (e == cudaSuccess) e = ln(L->t, D.ln2_g, D.ln2_b, O);
   } else {
     e = ln(X, D.ln1_g, D.ln1_b, L->y);
-    if (e == cudaSuccess) e = gemm(L->y, D.w_qkv, D.b_qkv, nullptr, L->qkv, 3 * d, d, LAYER_ACT_NONE);
+    if (e == cudaSuccess) e = gemm(L->y, D.w_qkv, D.b_qkv, nullptr, L->qkv, 3 * d, d, LAYER_ACT_NONE, vt_out);
     if (e == cudaSuccess) e = launch_attention_tc(L->qkv, L->vt, L->a, L->status, n, d, D.heads, n_seqs, n_seqs_dev, D.causal, st);
     if (e == cudaSuccess) e = gemm(L->a, D.w_o, D.b_o, X, L->t, d, d, LAYER_ACT_NONE);
     if (e == cudaSuccess) e = ln(L->t, D.ln2_g, D.ln2_b, L->y);

@@ -8,8 +8,8 @@
 //   P  = softmax step four warps, one thread per query row: two passes over the row in tensor memory (maximum, then
 //                     exponentials and their sum), P written as bf16 into shared memory in the swizzled K-major
 //                     layout the next product reads
-//   PV = P V          tcgen05.mma 128 x 64 x 128 into a second accumulator; V is read through its per-head
-//                     transpose V^T [64, n] (written by k_transpose_v), so that both operands are K-major
+//   PV = P V          tcgen05.mma 128 x 64 x 128; V is read through its per-head transpose V^T [64, n] (written
+//                     by the epilogue of the q|k|v product), so that both operands are K-major
 //   O  = O * exp(m_old - m_new) + PV   in registers (running maximum m and sum l per row: on-line softmax)
 // causal: position i attends to j <= i; key tiles beyond the diagonal are skipped.
 // Warp 0 produces (TMA), warp 1 issues the MMAs and owns the tensor memory, warps 2..5 do the softmax and the
@@ -23,17 +23,19 @@ namespace llmc {
 
 namespace {
 constexpr int AT_Q = 128, AT_K = 128, AT_DH = 64;
-constexpr int AT_THREADS = 192;
+constexpr int AT_THREADS = 320;                          // warp 0: TMA, warp 1: MMA, warps 2..9: softmax (2 threads per query row)
+constexpr int AT_SOFT = 256;
 constexpr int AT_SLOTS = 3;                              // ring of 16 KB operand tiles: K_j, V_j, K_j+1, ...
 constexpr uint32_t AT_TILE = 16384;                      // bytes of a 128 x 64 (or 2 x 64 x 64) bf16 tile
-constexpr uint32_t AT_TMEM_COLS = 256;                   // S: columns 0..127, PV: columns 128..191
+constexpr uint32_t AT_TMEM_COLS = 256;                   // two accumulators of 128 columns
 struct AttSmem {
   static constexpr uint32_t Q = 0;
   static constexpr uint32_t RING = Q + AT_TILE;
   static constexpr uint32_t P = RING + AT_SLOTS * AT_TILE;            // two 128 x 64 sub-tiles
-  static constexpr uint32_t BAR = P + 2 * AT_TILE;                    // q_full, full[3], empty[3], s_full, s_empty, p_full, pv_full, pv_empty
+  static constexpr uint32_t BAR = P + 2 * AT_TILE;                    // q_full, full[3], empty[3], s_full[2], p_full, pv_full, pv_read[2]
   static constexpr uint32_t MISC = BAR + 16 * 8;
-  static constexpr uint32_t TOTAL = MISC + 64;
+  static constexpr uint32_t XCH = MISC + 64;                          // float [2 tile parities + 1][2 halves][128 rows]: row maxima; row sums
+  static constexpr uint32_t TOTAL = XCH + 3 * 2 * 128 * 4;
 };
 constexpr uint32_t ATT_SMEM_BYTES = AttSmem::TOTAL + 1024;            // slack for manual alignment
 // kind::f16 instruction descriptors: fp32 accumulator, bf16 A and B, both K-major, M = 128
@@ -49,36 +51,35 @@ __device__ __forceinline__ uint32_t pack2(float a, float b) {
   const __nv_bfloat162 v = __floats2bfloat162_rn(a, b);
   return *reinterpret_cast<const uint32_t*>(&v);
 }
+// packed pairs of fp32 (one instruction for two lanes of arithmetic)
+__device__ __forceinline__ unsigned long long f2_pack(float lo, float hi) {
+  return ((unsigned long long)__float_as_uint(hi) << 32) | (unsigned long long)__float_as_uint(lo);
+}
+__device__ __forceinline__ float f2_lo(unsigned long long v) { return __uint_as_float((uint32_t)v); }
+__device__ __forceinline__ float f2_hi(unsigned long long v) { return __uint_as_float((uint32_t)(v >> 32)); }
+__device__ __forceinline__ unsigned long long f2_fma(unsigned long long a, unsigned long long b, unsigned long long c) {
+  unsigned long long d;
+  asm("fma.rn.f32x2 %0, %1, %2, %3;" : "=l"(d) : "l"(a), "l"(b), "l"(c));
+  return d;
+}
+__device__ __forceinline__ unsigned long long f2_add(unsigned long long a, unsigned long long b) {
+  unsigned long long d;
+  asm("add.rn.f32x2 %0, %1, %2;" : "=l"(d) : "l"(a), "l"(b));
+  return d;
+}
+// named barrier of the two softmax warps that share TMEM lane quarter q (barrier 0 is __syncthreads)
+__device__ __forceinline__ void pair_sync(uint32_t q) {
+  switch (q) {
+    case 0: asm volatile("bar.sync 1, 64;" ::: "memory"); break;
+    case 1: asm volatile("bar.sync 2, 64;" ::: "memory"); break;
+    case 2: asm volatile("bar.sync 3, 64;" ::: "memory"); break;
+    default: asm volatile("bar.sync 4, 64;" ::: "memory"); break;
+  }
+}
 __device__ __forceinline__ void sts16(uint32_t addr, uint32_t a, uint32_t b, uint32_t c, uint32_t d) {
   asm volatile("st.shared.v4.u32 [%0], {%1,%2,%3,%4};" ::"r"(addr), "r"(a), "r"(b), "r"(c), "r"(d) : "memory");
 }
 }  // namespace
-
-// V^T per (sequence, head): vt[((seq * heads + h) * 64 + c) * pitch + pos] = v[seq, pos, h * 64 + c].
-// One block per (sequence * heads + h, tile of 64 positions).
-__global__ void __launch_bounds__(256)
-k_transpose_v(const __nv_bfloat16* __restrict__ qkv, __nv_bfloat16* __restrict__ vt, uint32_t n, uint32_t d,
-              uint32_t heads, uint32_t pitch, uint32_t seq_max, const uint32_t* __restrict__ m_seq_dev) {
-  griddep_sync();
-  __shared__ __nv_bfloat16 tile[64][AT_DH + 2];
-  uint32_t n_seq = seq_max;
-  if (m_seq_dev) n_seq = min(seq_max, *m_seq_dev);
-  const uint32_t sh = blockIdx.x, seq = sh / heads, h = sh % heads;
-  if (seq >= n_seq) return;
-  const uint32_t p0 = blockIdx.y * 64;
-  for (uint32_t idx = threadIdx.x; idx < 64 * 32; idx += 256) {        // 64 positions x 32 pairs of head dims
-    const uint32_t r = idx >> 5, c2 = idx & 31u;
-    uint32_t w = 0;
-    if (p0 + r < n)
-      w = *reinterpret_cast<const uint32_t*>(qkv + ((size_t)seq * n + p0 + r) * 3 * d + 2 * d + h * AT_DH + c2 * 2);
-    *reinterpret_cast<uint32_t*>(&tile[r][c2 * 2]) = w;
-  }
-  __syncthreads();
-  for (uint32_t idx = threadIdx.x; idx < 64 * 64; idx += 256) {
-    const uint32_t c = idx >> 6, r = idx & 63u;
-    if (p0 + r < n) vt[((size_t)sh * AT_DH + c) * pitch + p0 + r] = tile[r][c];
-  }
-}
 
 __global__ void __launch_bounds__(AT_THREADS, 2)
 k_attention_tc(const __grid_constant__ CUtensorMap map_qkv, const __grid_constant__ CUtensorMap map_vt,
@@ -103,8 +104,9 @@ k_attention_tc(const __grid_constant__ CUtensorMap map_qkv, const __grid_constan
   const uint32_t q_full = bar0;
   auto full_bar = [&](uint32_t s) { return bar0 + 8 * (1 + s); };
   auto empty_bar = [&](uint32_t s) { return bar0 + 8 * (1 + AT_SLOTS + s); };
-  const uint32_t s_full = bar0 + 8 * 7, s_empty = bar0 + 8 * 8, p_full = bar0 + 8 * 9, pv_full = bar0 + 8 * 10,
-                 pv_empty = bar0 + 8 * 11;
+  // s_full[2]: S of a tile is complete in accumulator 0 / 1; p_full: P of a tile is in shared memory (and its S
+  // has been read); pv_full: PV of a tile is complete; pv_read[2]: the PV in accumulator 0 / 1 has been read
+  const uint32_t s_full = bar0 + 8 * 7, p_full = bar0 + 8 * 9, pv_full = bar0 + 8 * 10, pv_read = bar0 + 8 * 11;
   volatile uint32_t* misc = reinterpret_cast<volatile uint32_t*>(gbase + AttSmem::MISC);
   volatile uint32_t* tmem_slot = misc + 0;
   volatile uint32_t* abort_flag = misc + 1;
@@ -117,7 +119,8 @@ k_attention_tc(const __grid_constant__ CUtensorMap map_qkv, const __grid_constan
   if (threadIdx.x == 0) {
     mbar_init(q_full, 1);
     for (uint32_t s = 0; s < AT_SLOTS; ++s) { mbar_init(full_bar(s), 1); mbar_init(empty_bar(s), 1); }
-    mbar_init(s_full, 1); mbar_init(s_empty, 128); mbar_init(p_full, 128); mbar_init(pv_full, 1); mbar_init(pv_empty, 128);
+    mbar_init(s_full, 1); mbar_init(s_full + 8, 1); mbar_init(p_full, AT_SOFT); mbar_init(pv_full, 1);
+    mbar_init(pv_read, AT_SOFT); mbar_init(pv_read + 8, AT_SOFT);
     misc[1] = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
@@ -131,7 +134,6 @@ k_attention_tc(const __grid_constant__ CUtensorMap map_qkv, const __grid_constan
   __syncthreads();
   tc_fence_after();
   const uint32_t tmem_base = *tmem_slot;
-  const uint32_t tmem_s = tmem_base, tmem_pv = tmem_base + AT_K;
 
   uint32_t issued = 0;                                   // producer: ring tiles armed so far
   bool q_armed = false;
@@ -144,7 +146,7 @@ k_attention_tc(const __grid_constant__ CUtensorMap map_qkv, const __grid_constan
       q_armed = true;
       for (uint32_t i = 0; i < 2 * nkv && ok; ++i) {
         const uint32_t s = i % AT_SLOTS, ph = (i / AT_SLOTS) & 1u, j = i >> 1;
-        if (!mbar_wait(empty_bar(s), ph ^ 1u, abort_flag, lim)) { ok = false; break; }
+        if (!mbar_wait(empty_bar(s), ph ^ 1u, abort_flag, lim, 64)) { ok = false; break; }
         mbar_expect_tx(full_bar(s), AT_TILE);
         const uint32_t dst = sRing + s * AT_TILE;
         if ((i & 1u) == 0) {
@@ -160,34 +162,43 @@ k_attention_tc(const __grid_constant__ CUtensorMap map_qkv, const __grid_constan
     }
   } else if (warp == 1) {
     // ------------------------------------------------------------ MMA issuer
+    // Tile j uses accumulator j % 2: first for S_j (128 columns), then, once the softmax has read it, for
+    // PV_j (its first 64 columns).  S_(j+1) is issued while the softmax works on tile j, so the softmax never
+    // waits for a product that could have run earlier.  Operand tiles are consumed in the order
+    // K_0, K_1, V_0, K_2, V_1, ...; item i of the load order K_0, V_0, K_1, V_1, ... sits in ring slot i % 3.
     if (lane == 0) {
-      bool ok = mbar_wait(q_full, 0u, abort_flag, lim);
+      bool ok = mbar_wait(q_full, 0u, abort_flag, lim, 64);
       tc_fence_after();
       const uint64_t dq = smem_desc_sw128(sQ);
-      for (uint32_t j = 0; j < nkv && ok; ++j) {
-        const uint32_t jp = j & 1u;
-        // S = Q K_j^T
+      auto issue_s = [&](uint32_t j) -> bool {          // S_j = Q K_j^T into accumulator j % 2
         const uint32_t ik = 2 * j, sk = ik % AT_SLOTS, phk = (ik / AT_SLOTS) & 1u;
-        if (!mbar_wait(full_bar(sk), phk, abort_flag, lim)) { ok = false; break; }
-        if (!mbar_wait(s_empty, jp ^ 1u, abort_flag, lim)) { ok = false; break; }      // softmax is done with S_(j-1)
+        if (!mbar_wait(full_bar(sk), phk, abort_flag, lim, 64)) return false;
+        // the accumulator held PV_(j-2): the softmax must have read it
+        if (j >= 2 && !mbar_wait(pv_read + 8 * (j & 1u), ((j >> 1) - 1u) & 1u, abort_flag, lim, 64)) return false;
         tc_fence_after();
         const uint64_t dk = smem_desc_sw128(sRing + sk * AT_TILE);
+        const uint32_t acc = tmem_base + (j & 1u) * AT_K;
 #pragma unroll
         for (uint32_t kk = 0; kk < AT_DH / 16; ++kk)
-          tc_mma_bf16(tmem_s, dq + kk * 2, dk + kk * 2, IDESC_S, kk != 0u);
+          tc_mma_bf16(acc, dq + kk * 2, dk + kk * 2, IDESC_S, kk != 0u);
         tc_commit(empty_bar(sk));
-        tc_commit(s_full);
-        // PV = P_j V_j
+        tc_commit(s_full + 8 * (j & 1u));                // the (j / 2)-th completion of this barrier
+        return true;
+      };
+      if (ok && nkv) ok = issue_s(0);
+      for (uint32_t j = 0; j < nkv && ok; ++j) {
+        if (j + 1 < nkv && !issue_s(j + 1)) { ok = false; break; }
+        // PV_j = P_j V_j into the first 64 columns of accumulator j % 2 (S_j has been read: p_full says so)
         const uint32_t iv = 2 * j + 1, sv = iv % AT_SLOTS, phv = (iv / AT_SLOTS) & 1u;
-        if (!mbar_wait(full_bar(sv), phv, abort_flag, lim)) { ok = false; break; }
-        if (!mbar_wait(p_full, jp, abort_flag, lim)) { ok = false; break; }
-        if (!mbar_wait(pv_empty, jp ^ 1u, abort_flag, lim)) { ok = false; break; }     // PV_(j-1) has been read
+        if (!mbar_wait(full_bar(sv), phv, abort_flag, lim, 64)) { ok = false; break; }
+        if (!mbar_wait(p_full, j & 1u, abort_flag, lim, 64)) { ok = false; break; }
         tc_fence_after();
+        const uint32_t acc = tmem_base + (j & 1u) * AT_K;
 #pragma unroll
         for (uint32_t kk = 0; kk < AT_K / 16; ++kk) {
           const uint64_t dp = smem_desc_sw128(sP + (kk >> 2) * AT_TILE) + (kk & 3u) * 2;
           const uint64_t dv = smem_desc_sw128(sRing + sv * AT_TILE + (kk >> 2) * (AT_TILE / 2)) + (kk & 3u) * 2;
-          tc_mma_bf16(tmem_pv, dp, dv, IDESC_PV, kk != 0u);
+          tc_mma_bf16(acc, dp, dv, IDESC_PV, kk != 0u);
         }
         tc_commit(empty_bar(sv));
         tc_commit(pv_full);
@@ -195,86 +206,123 @@ k_attention_tc(const __grid_constant__ CUtensorMap map_qkv, const __grid_constan
       if (!ok) { *abort_flag = 1; atomicExch(status, 1u); }
     }
   } else {
-    // ------------------------------------------------------------ softmax + output (128 threads, one query row each)
+    // ------------------------------------------------------------ softmax + output
+    // 256 threads, two per query row: warps w and w + 4 read the same 32 lanes of tensor memory; the first takes
+    // key columns 0..63 of a tile and output columns 0..31, the second key columns 64..127 and output columns
+    // 32..63.  The two exchange their row maxima through shared memory once per tile; the row sums are kept
+    // apart until the end (both threads scale by the same factors).
     const uint32_t quarter = warp & 3u;                  // TMEM lanes this warp may read
+    const uint32_t hf = (warp - 2u) >> 2;                // which half of the columns
     const uint32_t r = quarter * 32 + lane;              // row of the tile
     const uint32_t qrow = q0 + r;
     const uint32_t lane_addr = (quarter * 32u) << 16;
     const float sc = 0.125f * 1.4426950408889634f;       // 1 / sqrt(64), in base-2 exponent units
-    float o[AT_DH];
+    float* xch = reinterpret_cast<float*>(gbase + AttSmem::XCH);
+    unsigned long long o2[16];                           // 32 output columns as packed pairs
 #pragma unroll
-    for (int c = 0; c < AT_DH; ++c) o[c] = 0.f;
-    float m_run = -INFINITY, l_run = 0.f;
+    for (int c = 0; c < 16; ++c) o2[c] = 0ull;
+    float m_run = -INFINITY, l_run = 0.f, corr_prev = 1.f;
     bool ok = true;
-    for (uint32_t j = 0; j < nkv; ++j) {
-      const uint32_t jp = j & 1u, k0 = j * AT_K;
-      if (!mbar_wait(s_full, jp, abort_flag, lim)) { *abort_flag = 1; atomicExch(status, 1u); ok = false; break; }
+    // O = O * corr + PV of tile j (its product sits in the first 64 columns of accumulator j % 2)
+    auto accumulate = [&](uint32_t j, float corr) -> bool {
+      if (!mbar_wait(pv_full, j & 1u, abort_flag, lim, 32)) return false;
       tc_fence_after();
-      // pass 1: row maximum
-      float m_new = m_run;
-#pragma unroll 1
-      for (uint32_t c = 0; c < AT_K; c += 32) {
-        uint32_t v[32];
-        tc_ld_32x32(tmem_s + lane_addr + c, v);
-        tc_wait_ld();
+      uint32_t v[32];
+      tc_ld_32x32(tmem_base + (j & 1u) * AT_K + lane_addr + hf * 32, v);
+      tc_wait_ld();
+      const unsigned long long c2 = f2_pack(corr, corr);
 #pragma unroll
-        for (uint32_t i = 0; i < 32; ++i) {
-          const uint32_t key = k0 + c + i;
-          const bool live = key < n && (!causal || key <= qrow);
-          m_new = fmaxf(m_new, live ? __uint_as_float(v[i]) * sc : -INFINITY);
+      for (uint32_t i = 0; i < 16; ++i)
+        o2[i] = f2_fma(o2[i], c2, f2_pack(__uint_as_float(v[2 * i]), __uint_as_float(v[2 * i + 1])));
+      tc_fence_before();
+      mbar_arrive(pv_read + 8 * (j & 1u));
+      return true;
+    };
+    for (uint32_t j = 0; j < nkv; ++j) {
+      const uint32_t k0 = j * AT_K + hf * 64;            // first key of this thread's columns
+      const uint32_t acc = tmem_base + (j & 1u) * AT_K + lane_addr + hf * 64;
+      // masking is needed only in the tile that holds the end of the sequence and, if causal, on the diagonal
+      const bool masked = (j * AT_K + AT_K > n) || (causal && j * AT_K + AT_K > q0 + 1);
+      if (!mbar_wait(s_full + 8 * (j & 1u), (j >> 1) & 1u, abort_flag, lim, 32)) { ok = false; break; }
+      tc_fence_after();
+      // pass 1: maximum of the raw products over this thread's 64 columns (the scale is positive)
+      float mx = -INFINITY;
+      {
+        uint32_t v0[32], v1[32];
+        tc_ld_32x32(acc, v0);
+        tc_ld_32x32(acc + 32, v1);
+        tc_wait_ld();
+        if (masked) {
+#pragma unroll
+          for (uint32_t i = 0; i < 32; ++i) {
+            const uint32_t ka = k0 + i, kb = ka + 32;
+            if (ka < n && (!causal || ka <= qrow)) mx = fmaxf(mx, __uint_as_float(v0[i]));
+            if (kb < n && (!causal || kb <= qrow)) mx = fmaxf(mx, __uint_as_float(v1[i]));
+          }
+        } else {
+#pragma unroll
+          for (uint32_t i = 0; i < 32; ++i) mx = fmaxf(mx, fmaxf(__uint_as_float(v0[i]), __uint_as_float(v1[i])));
         }
       }
-      const float corr = (m_new == -INFINITY) ? 1.f : ex2f(m_run - m_new);
+      float* xm = xch + (j & 1u) * 256;
+      xm[hf * 128 + r] = mx;
+      pair_sync(quarter);                                // the two warps that share these rows
+      const float m_new = fmaxf(m_run, fmaxf(mx, xm[(hf ^ 1u) * 128 + r]) * sc);
+      // the product of the previous tile, while the tensor cores are free to start the next S
+      if (j > 0 && !accumulate(j - 1, corr_prev)) { ok = false; break; }
+      const bool dead = m_new == -INFINITY;              // no key of any tile so far is visible to this row
+      const float corr = dead ? 1.f : ex2f(m_run - m_new);
+      const unsigned long long sc2 = f2_pack(sc, sc), nm2 = f2_pack(dead ? 0.f : -m_new, dead ? 0.f : -m_new);
       // pass 2: exponentials, their sum, P as bf16 into shared memory (16-byte chunk c of row r at chunk c ^ (r % 8))
-      float psum = 0.f;
+      unsigned long long ps2 = 0ull;
+      const uint32_t sub = sP + hf * AT_TILE + r * 128u;
 #pragma unroll 1
-      for (uint32_t c = 0; c < AT_K; c += 32) {
+      for (uint32_t c = 0; c < 64; c += 32) {
         uint32_t v[32];
-        tc_ld_32x32(tmem_s + lane_addr + c, v);
+        tc_ld_32x32(acc + c, v);
         tc_wait_ld();
-        float p[32];
-#pragma unroll
-        for (uint32_t i = 0; i < 32; ++i) {
-          const uint32_t key = k0 + c + i;
-          const bool live = key < n && (!causal || key <= qrow) && m_new != -INFINITY;
-          p[i] = live ? ex2f(__uint_as_float(v[i]) * sc - m_new) : 0.f;
-          psum += p[i];
-        }
-        const uint32_t sub = sP + (c >> 6) * AT_TILE + r * 128u;
 #pragma unroll
         for (uint32_t q4 = 0; q4 < 4; ++q4) {
-          const uint32_t chunk = ((c & 63u) >> 3) + q4;
-          sts16(sub + ((chunk ^ (r & 7u)) << 4), pack2(p[q4 * 8], p[q4 * 8 + 1]), pack2(p[q4 * 8 + 2], p[q4 * 8 + 3]),
-                pack2(p[q4 * 8 + 4], p[q4 * 8 + 5]), pack2(p[q4 * 8 + 6], p[q4 * 8 + 7]));
+          uint32_t pk[4];
+#pragma unroll
+          for (uint32_t e = 0; e < 4; ++e) {
+            const uint32_t i = q4 * 8 + 2 * e;
+            const unsigned long long t2 = f2_fma(f2_pack(__uint_as_float(v[i]), __uint_as_float(v[i + 1])), sc2, nm2);
+            float pa = ex2f(f2_lo(t2)), pb = ex2f(f2_hi(t2));
+            if (masked) {
+              const uint32_t key = k0 + c + i;
+              if (dead || !(key < n && (!causal || key <= qrow))) pa = 0.f;
+              if (dead || !(key + 1 < n && (!causal || key + 1 <= qrow))) pb = 0.f;
+            }
+            ps2 = f2_add(ps2, f2_pack(pa, pb));
+            pk[e] = pack2(pa, pb);
+          }
+          const uint32_t chunk = (c >> 3) + q4;
+          sts16(sub + ((chunk ^ (r & 7u)) << 4), pk[0], pk[1], pk[2], pk[3]);
         }
       }
-      tc_fence_before();
-      mbar_arrive(s_empty);                                           // S_j has been read
-      asm volatile("fence.proxy.async.shared::cta;" ::: "memory");    // P visible to the tensor cores
+      tc_fence_before();                                              // S_j has been read ...
+      asm volatile("fence.proxy.async.shared::cta;" ::: "memory");    // ... and P_j is visible to the tensor cores
       mbar_arrive(p_full);
-      l_run = l_run * corr + psum;
+      l_run = l_run * corr + (f2_lo(ps2) + f2_hi(ps2));
       m_run = m_new;
-      // O = O * corr + P_j V_j
-      if (!mbar_wait(pv_full, jp, abort_flag, lim)) { *abort_flag = 1; atomicExch(status, 1u); ok = false; break; }
-      tc_fence_after();
-#pragma unroll
-      for (uint32_t c = 0; c < AT_DH; c += 32) {
-        uint32_t v[32];
-        tc_ld_32x32(tmem_pv + lane_addr + c, v);
-        tc_wait_ld();
-#pragma unroll
-        for (uint32_t i = 0; i < 32; ++i) o[c + i] = fmaf(o[c + i], corr, __uint_as_float(v[i]));
-      }
-      tc_fence_before();
-      mbar_arrive(pv_empty);
+      corr_prev = corr;
     }
+    if (ok && nkv) ok = accumulate(nkv - 1, corr_prev);
+    if (!ok) { *abort_flag = 1; atomicExch(status, 1u); }
+    // the row's sum is the sum of the two threads' sums
+    xch[512 + hf * 128 + r] = l_run;
+    pair_sync(quarter);
+    const float l_tot = l_run + xch[512 + (hf ^ 1u) * 128 + r];
     if (ok && qrow < n) {
-      const float inv = 1.0f / l_run;
-      uint4* op = reinterpret_cast<uint4*>(out + ((size_t)tok0 + qrow) * d + h * AT_DH);
+      const float inv = 1.0f / l_tot;
+      uint4* op = reinterpret_cast<uint4*>(out + ((size_t)tok0 + qrow) * d + h * AT_DH + hf * 32);
 #pragma unroll
-      for (int q4 = 0; q4 < 8; ++q4)
-        op[q4] = make_uint4(pack2(o[q4 * 8] * inv, o[q4 * 8 + 1] * inv), pack2(o[q4 * 8 + 2] * inv, o[q4 * 8 + 3] * inv),
-                            pack2(o[q4 * 8 + 4] * inv, o[q4 * 8 + 5] * inv), pack2(o[q4 * 8 + 6] * inv, o[q4 * 8 + 7] * inv));
+      for (int q4 = 0; q4 < 4; ++q4)
+        op[q4] = make_uint4(pack2(f2_lo(o2[q4 * 4]) * inv, f2_hi(o2[q4 * 4]) * inv),
+                            pack2(f2_lo(o2[q4 * 4 + 1]) * inv, f2_hi(o2[q4 * 4 + 1]) * inv),
+                            pack2(f2_lo(o2[q4 * 4 + 2]) * inv, f2_hi(o2[q4 * 4 + 2]) * inv),
+                            pack2(f2_lo(o2[q4 * 4 + 3]) * inv, f2_hi(o2[q4 * 4 + 3]) * inv));
     }
   }
 
@@ -307,7 +355,7 @@ cudaError_t setup_attention_kernel() {
 // Positions between the rows of V^T: a multiple of 8 (16 bytes), so that every row can start a TMA box.
 uint32_t attention_vt_pitch(uint32_t n) { return (n + 7u) / 8u * 8u; }
 
-cudaError_t launch_attention_tc(const __nv_bfloat16* qkv, __nv_bfloat16* vt, __nv_bfloat16* out, uint32_t* status,
+cudaError_t launch_attention_tc(const __nv_bfloat16* qkv, const __nv_bfloat16* vt, __nv_bfloat16* out, uint32_t* status,
                                 uint32_t n, uint32_t d, uint32_t heads, uint32_t seq_max, const uint32_t* m_seq_dev,
                                 int causal, cudaStream_t st) {
   if (seq_max == 0) return cudaSuccess;
@@ -316,9 +364,6 @@ cudaError_t launch_attention_tc(const __nv_bfloat16* qkv, __nv_bfloat16* vt, __n
   if (!make_tensor_map_bf16(&map_qkv, qkv, (uint64_t)seq_max * n, 3ull * d, AT_Q) ||
       !make_tensor_map_bf16_pitch(&map_vt, vt, (uint64_t)seq_max * heads * AT_DH, n, pitch, AT_DH))
     return cudaErrorInvalidValue;
-  cudaError_t e = launch_k(k_transpose_v, dim3(seq_max * heads, (n + 63) / 64), dim3(256), 0, st, qkv, vt, n, d, heads,
-                           pitch, seq_max, m_seq_dev);
-  if (e != cudaSuccess) return e;
   const uint32_t qtiles = (n + AT_Q - 1) / AT_Q;
   return launch_k(k_attention_tc, dim3(seq_max * heads * qtiles), dim3(AT_THREADS), ATT_SMEM_BYTES, st, map_qkv, map_vt,
                   out, status, n, d, heads, seq_max, m_seq_dev, causal);

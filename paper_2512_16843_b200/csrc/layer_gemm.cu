@@ -43,7 +43,7 @@ k_gemm_tc(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUt
           const float* __restrict__ bias, const __nv_bfloat16* __restrict__ residual,
           __nv_bfloat16* __restrict__ out, uint32_t* __restrict__ status,
           uint32_t M_max, uint32_t N, uint32_t KB, const uint32_t* __restrict__ m_seq_dev, uint32_t rows_per_seq,
-          uint32_t act) {
+          uint32_t act, VtOut vt) {
   griddep_sync();
   extern __shared__ uint8_t smem_raw[];
   const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;
@@ -166,6 +166,16 @@ k_gemm_tc(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUt
 #pragma unroll
             for (int i = 0; i < 32; ++i) f[i] = gelu_tanh_f(f[i]);
           }
+          if (vt.ptr && col0 >= vt.col0) {
+            // the V third of a q|k|v product goes out transposed per head, for the attention kernel:
+            // vt[((seq * heads + h) * 64 + c) * pitch + pos]; the lanes of a warp are consecutive positions
+            const uint32_t seq = row / rows_per_seq, pos = row - seq * rows_per_seq;
+            const uint32_t hc = col0 - vt.col0;                       // h * 64 + c of the first column
+            __nv_bfloat16* dst = vt.ptr + ((size_t)seq * vt.heads * 64 + hc) * vt.pitch + pos;
+#pragma unroll
+            for (int i = 0; i < 32; ++i) dst[(size_t)i * vt.pitch] = __float2bfloat16_rn(f[i]);
+            continue;
+          }
           const size_t off = (size_t)row * N + col0;
           if (residual) {
             const uint4* r4 = reinterpret_cast<const uint4*>(residual + off);
@@ -219,7 +229,7 @@ cudaError_t setup_gemm_kernel() {
 cudaError_t launch_gemm(const __nv_bfloat16* a, const __nv_bfloat16* w, const float* bias,
                         const __nv_bfloat16* residual, __nv_bfloat16* out, uint32_t* status, uint32_t M_max,
                         uint32_t N, uint32_t K, const uint32_t* m_seq_dev, uint32_t rows_per_seq, uint32_t act,
-                        int sm_count, cudaStream_t st) {
+                        int sm_count, cudaStream_t st, VtOut vt) {
   if (M_max == 0) return cudaSuccess;
   alignas(64) CUtensorMap map_a, map_w;
   if (!make_tensor_map_bf16(&map_a, a, M_max, K, GM) || !make_tensor_map_bf16(&map_w, w, N, K, GN))
@@ -227,7 +237,7 @@ cudaError_t launch_gemm(const __nv_bfloat16* a, const __nv_bfloat16* w, const fl
   const uint32_t tiles = ((M_max + GM - 1) / GM) * ((N + GN - 1) / GN);
   const uint32_t grid = tiles < (uint32_t)sm_count ? tiles : (uint32_t)sm_count;
   return launch_k(k_gemm_tc, dim3(grid), dim3(GEMM_THREADS), GEMM_SMEM_BYTES, st, map_a, map_w, bias, residual, out,
-                  status, M_max, N, K / GK, m_seq_dev, rows_per_seq, act);
+                  status, M_max, N, K / GK, m_seq_dev, rows_per_seq, act, vt);
 }
 
 }  // namespace llmc

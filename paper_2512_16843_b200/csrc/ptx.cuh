@@ -37,8 +37,10 @@ __device__ __forceinline__ unsigned long long global_ns() {
   return t;
 }
 // Bounded wait for the phase with the given parity.  Returns false on expiry or abort.
+// backoff_ns > 0: sleep that long between polls (for waiters that share an SM with warps that have work to
+// issue: a bare polling loop takes issue slots from them).
 __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile uint32_t* abort_flag,
-                                          unsigned long long limit_ns = WAIT_LIMIT_NS) {
+                                          unsigned long long limit_ns = WAIT_LIMIT_NS, uint32_t backoff_ns = 0) {
   if (*abort_flag) return false;
   unsigned long long t0 = 0;
   for (uint32_t spin = 0;; ++spin) {
@@ -49,6 +51,7 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatil
         "selp.u32 %0, 1, 0, p;\n\t}"
         : "=r"(done) : "r"(bar), "r"(parity) : "memory");
     if (done) return true;
+    if (backoff_ns) __nanosleep(backoff_ns);
     if ((spin & 255u) == 255u) {
       if (*abort_flag) return false;
       const unsigned long long now = global_ns();
