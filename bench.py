@@ -822,7 +822,10 @@ def run_e2e(args):
     torch_ms = e0.elapsed_time(e1) / 5 * Lyr
     out = {"metric": "end-to-end batch latency, layer-wise caching loop (Algorithm 1) vs no caching", "unit": "ms",
            "value": res["llmcache"], "nocache_ms": res["nocache"], "speedup": res["nocache"] / res["llmcache"],
+           "pool_bytes_read_per_batch": Lyr * B * n * d * 2,   # every layer's probe reads its whole input to pool it
            "fingerprint_on_write": {"ms": res["llmcache_fused"], "speedup": res["nocache"] / res["llmcache_fused"],
+                                    "pool_bytes_read_per_batch": B * n * d * 2,   # only layer 1 does; the row movers sum the rest
+
                                     "hit_fraction_mean": res["llmcache_fused_hits"],
                                     "bank_kernels_ms_per_batch": res["llmcache_fused_bank_kernels_ms_per_batch"]},
            "bank_kernels_ms_per_batch": res["llmcache_bank_kernels_ms_per_batch"],

@@ -365,7 +365,9 @@ int llmcache_layer_debug_knobs(llmcache_layer_t* layer, uint64_t wait_limit_ns, 
  * compacted misses, commit (write back + insert).  banks == NULL runs every layer in full (no caching).
  * h0: device bf16 [B,n,d].  buf_a, buf_b: device [B,n,d] bf16 ping-pong outputs; h_miss, miss_out: device
  * [B,n,d] scratch (unused without banks); io: probe buffers for B.  *h_final receives the pointer (buf_a or
- * buf_b) that holds h_L once the stream has run. */
+ * buf_b) that holds h_L once the stream has run.  When every bank was created with fused_pool = 1 the loop
+ * takes the fingerprint-on-write path by itself (see llmcache_infer_pooled; the position means travel in
+ * buffers the banks own): only layer 1 reads its input to pool it. */
 int llmcache_infer(llmcache_bank_t** banks, llmcache_layer_t** layers, uint32_t n_layers, const void* h0, uint32_t B,
                    float tau, void* buf_a, void* buf_b, void* h_miss, void* miss_out, llmcache_probe_io* io,
                    void** h_final, void* stream);

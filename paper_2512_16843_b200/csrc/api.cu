@@ -17,7 +17,7 @@ inline uint32_t pow2_ceil(uint32_t x) { uint32_t p = 1; while (p < x) p <<= 1; r
 
 struct Layout {
   size_t fp, rb, valid, last_use, insert_tick, hits, rate, rate_epoch, act, proj, center;
-  size_t pool_partial, move_partial, best, hitcnt, victims, new_slot, bits, qbits, sort_key, sort_slot, stats, status, misc, blk_cnt, sel_keys, sel_state, sel_blk, sel_mcnt, total;
+  size_t pool_partial, move_partial, pooled_own, best, hitcnt, victims, new_slot, bits, qbits, sort_key, sort_slot, stats, status, misc, blk_cnt, sel_keys, sel_state, sel_blk, sel_mcnt, total;
   uint32_t sort_len;
 };
 
@@ -73,6 +73,7 @@ Layout make_layout(const llmcache_bank_desc& d) {
   // scratch: one vector of partial sums per (pool block, sequence it touches)
   L.pool_partial = take(((size_t)d.max_batch + 3 * POOL_MAX_GRID) * dm * 4);
   L.move_partial = take(d.fused_pool ? 2 * move_partial_floats(d.max_batch, d.d_model) * 4 : 0);
+  L.pooled_own = take(d.fused_pool ? (size_t)d.max_batch * dm * 4 : 0);
   L.best = take((size_t)d.max_batch * 8);
   L.hitcnt = take(N * 4);
   const uint32_t vmax = d.max_batch < d.capacity ? d.max_batch : d.capacity;
@@ -218,6 +219,7 @@ int llmcache_bank_create(const llmcache_bank_desc* desc, llmcache_bank_t** bank_
   a.center = desc->center ? (float*)(base + L.center) : nullptr;
   a.pool_partial = (float*)(base + L.pool_partial);
   a.move_partial = desc->fused_pool ? (float*)(base + L.move_partial) : nullptr;
+  a.pooled_own = desc->fused_pool ? (float*)(base + L.pooled_own) : nullptr;
   a.best = (unsigned long long*)(base + L.best);
   a.hitcnt = (uint32_t*)(base + L.hitcnt);
   a.victims = (int32_t*)(base + L.victims);

@@ -183,11 +183,51 @@ int llmcache_layer_debug_knobs(llmcache_layer_t* L, uint64_t wait_limit_ns, uint
   return LLMCACHE_OK;
 }
 
+// Algorithm 1 with fingerprint-on-write: only layer 1 pools its input; every later probe takes the position means
+// that the previous layer's row movers produced.  pooled == nullptr: each bank's own buffer carries them.
+static int infer_fused(llmcache_bank_t** banks, llmcache_layer_t** layers, uint32_t n_layers, const void* h0,
+                       uint32_t B, float tau, void* buf_a, void* buf_b, void* h_miss, void* miss_out,
+                       llmcache_probe_io* io, float* pooled, void** h_final, void* stream) {
+  const void* cur = h0;
+  void* bufs[2] = {buf_a, buf_b};
+  const float* prev_means = nullptr;
+  int rc = LLMCACHE_OK;
+  for (uint32_t l = 0; l < n_layers && rc == LLMCACHE_OK; ++l) {
+    void* next = bufs[l & 1u];
+    const uint32_t ld = banks[l]->desc.d_model;
+    float* means_out = pooled ? pooled : banks[l]->a.pooled_own;
+    io->h_miss = h_miss;
+    // the rows this layer writes are summed on the way: means_out then holds the next layer's position means.
+    // (With one shared buffer the probe has consumed its previous contents before the commit overwrites them.)
+    rc = llmcache_bank_pool_out(banks[l], l + 1 < n_layers ? means_out : nullptr, ld);
+    if (rc != LLMCACHE_OK) break;
+    if (l == 0) rc = llmcache_probe(banks[l], cur, B, tau, next, io, stream);
+    else        rc = llmcache_probe_pooled(banks[l], prev_means, ld, cur, B, tau, next, io, stream);
+    if (rc == LLMCACHE_OK) rc = llmcache_layer_forward(layers[l], h_miss, B, io->counts + 1, miss_out, stream);
+    if (rc == LLMCACHE_OK) rc = llmcache_commit(banks[l], miss_out, io, next, nullptr, stream);
+    if (rc == LLMCACHE_OK) rc = llmcache_bank_pool_out(banks[l], nullptr, 0);
+    prev_means = means_out;
+    cur = next;
+  }
+  if (rc != LLMCACHE_OK) return rc;
+  *h_final = const_cast<void*>(cur);
+  return LLMCACHE_OK;
+}
+
 int llmcache_infer(llmcache_bank_t** banks, llmcache_layer_t** layers, uint32_t n_layers, const void* h0, uint32_t B,
                    float tau, void* buf_a, void* buf_b, void* h_miss, void* miss_out, llmcache_probe_io* io,
                    void** h_final, void* stream) {
   if (!layers || !h0 || !buf_a || !buf_b || !h_final || n_layers == 0) return LLMCACHE_ERR_ARG;
   if (banks && (!io || !h_miss || !miss_out)) return LLMCACHE_ERR_ARG;
+  if (banks) {
+    // banks created with fused_pool (all of them, same width) take the fingerprint-on-write path by themselves
+    bool fused = true;
+    for (uint32_t l = 0; l < n_layers; ++l)
+      fused = fused && banks[l] && banks[l]->a.pooled_own && banks[l]->desc.d_model == banks[0]->desc.d_model &&
+              B <= banks[l]->desc.max_batch;
+    if (fused) return infer_fused(banks, layers, n_layers, h0, B, tau, buf_a, buf_b, h_miss, miss_out, io, nullptr,
+                                  h_final, stream);
+  }
   const void* cur = h0;
   void* bufs[2] = {buf_a, buf_b};
   for (uint32_t l = 0; l < n_layers; ++l) {
@@ -214,27 +254,7 @@ int llmcache_infer_pooled(llmcache_bank_t** banks, llmcache_layer_t** layers, ui
                           llmcache_probe_io* io, float* pooled, void** h_final, void* stream) {
   if (!banks || !layers || !h0 || !buf_a || !buf_b || !h_final || n_layers == 0) return LLMCACHE_ERR_ARG;
   if (!io || !h_miss || !miss_out || !pooled) return LLMCACHE_ERR_ARG;
-  const void* cur = h0;
-  void* bufs[2] = {buf_a, buf_b};
-  int rc = LLMCACHE_OK;
-  for (uint32_t l = 0; l < n_layers && rc == LLMCACHE_OK; ++l) {
-    void* next = bufs[l & 1u];
-    const uint32_t ld = banks[l]->desc.d_model;
-    io->h_miss = h_miss;
-    // the rows this layer writes are summed on the way: `pooled` then holds the next layer's position means.
-    // (The probe has consumed the previous contents of `pooled` before the commit overwrites them.)
-    rc = llmcache_bank_pool_out(banks[l], l + 1 < n_layers ? pooled : nullptr, ld);
-    if (rc != LLMCACHE_OK) break;
-    if (l == 0) rc = llmcache_probe(banks[l], cur, B, tau, next, io, stream);
-    else        rc = llmcache_probe_pooled(banks[l], pooled, ld, cur, B, tau, next, io, stream);
-    if (rc == LLMCACHE_OK) rc = llmcache_layer_forward(layers[l], h_miss, B, io->counts + 1, miss_out, stream);
-    if (rc == LLMCACHE_OK) rc = llmcache_commit(banks[l], miss_out, io, next, nullptr, stream);
-    if (rc == LLMCACHE_OK) rc = llmcache_bank_pool_out(banks[l], nullptr, 0);
-    cur = next;
-  }
-  if (rc != LLMCACHE_OK) return rc;
-  *h_final = const_cast<void*>(cur);
-  return LLMCACHE_OK;
+  return infer_fused(banks, layers, n_layers, h0, B, tau, buf_a, buf_b, h_miss, miss_out, io, pooled, h_final, stream);
 }
 
 }  // extern "C"

@@ -39,6 +39,8 @@ struct BankArrays {
   // scratch
   float*    pool_partial;   // [(max_batch + 3 * POOL_MAX_GRID), d] partial sums of the pooling pass
   float*    move_partial;   // 2 x the same: partial sums of the rows moved for hits / for misses (or nullptr)
+  float*    pooled_own;     // [max_batch, d] position means of the rows this bank's passes wrote (fused_pool banks;
+                            // used by llmcache_infer to hand them to the next layer's probe), or nullptr
   unsigned long long* best; // [max_batch] packed (orderable score << 32 | ~slot); 0 = none
   uint32_t* hitcnt;         // [N] matches per slot within the current probe (zero between calls)
   int32_t*  victims;        // [min(max_batch,N)]

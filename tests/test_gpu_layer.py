@@ -138,7 +138,9 @@ def test_infer_algorithm1_matches_oracle_and_chain_property(pre_ln):
 
 def test_infer_with_fingerprint_on_write_equals_plain_loop():
     """Same batches through llmcache_infer and llmcache_infer_pooled (own banks each): same hits per layer,
-    same output bits.  (The two differ only in where the position means of h_1..h_{L-1} are taken.)"""
+    same output bits.  (The two differ only in where the position means of h_1..h_{L-1} are taken.)  A third
+    set of banks, created with fused_pool, goes through llmcache_infer, which must take the pooled path by
+    itself: same bits again, and the same number of kernel launches as the explicit pooled loop."""
     n, d, heads, ffn, B, Lyr, N, k = 40, 128, 2, 256, 14, 4, 64, 64
     ws = [synth.layer_weights(d, ffn, 400 + 20 * l, DEV) for l in range(Lyr)]
     for w in ws:
@@ -148,7 +150,7 @@ def test_infer_with_fingerprint_on_write_equals_plain_loop():
     layers = [L.Layer(w, heads=heads, seq_len=n, max_seqs=B) for w in ws]
     mkb = lambda fused: [L.Bank(capacity=N, seq_len=n, d_model=d, fp_dim=k, max_batch=B, proj=proj, tau=0.9,
                                 fused_pool=fused) for _ in range(Lyr)]
-    banks_a, banks_b = mkb(0), mkb(1)
+    banks_a, banks_b, banks_c = mkb(0), mkb(1), mkb(1)
     bufs = L.ProbeBuffers(B, k, DEV)
     mk = lambda: torch.zeros((B, n, d), dtype=torch.bfloat16, device=DEV)
     buf_a, buf_b, h_miss, miss_out = mk(), mk(), mk(), mk()
@@ -156,7 +158,9 @@ def test_infer_with_fingerprint_on_write_equals_plain_loop():
     hl = [l.handle for l in layers]
 
     def run(h0, fused):
-        if fused:
+        if fused == 2:
+            ptr = L.llmcache_infer([b.handle for b in banks_c], hl, h0, B, None, buf_a, buf_b, h_miss, miss_out, bufs.io)
+        elif fused:
             ptr = L.llmcache_infer_pooled([b.handle for b in banks_b], hl, h0, B, None, buf_a, buf_b, h_miss, miss_out,
                                           bufs.io, pooled)
         else:
@@ -173,7 +177,8 @@ def test_infer_with_fingerprint_on_write_equals_plain_loop():
     prev_a, prev_b = [0] * Lyr, [0] * Lyr
     total = 0
     for i, hb in enumerate(batches):
-        oa, ob = run(hb, False), run(hb, True)
+        oa, ob, oc = run(hb, False), run(hb, True), run(hb, 2)
+        assert torch.equal(oc.view(torch.int16), ob.view(torch.int16)), f"batch {i} (banks with fused_pool through llmcache_infer)"
         ha = [b.stats()["hits"] for b in banks_a]
         hb_ = [b.stats()["hits"] for b in banks_b]
         assert [x - y for x, y in zip(ha, prev_a)] == [x - y for x, y in zip(hb_, prev_b)], f"batch {i}"
@@ -184,8 +189,10 @@ def test_infer_with_fingerprint_on_write_equals_plain_loop():
     launches_a = sum(b.stats()["kernel_launches"] for b in banks_a)
     launches_b = sum(b.stats()["kernel_launches"] for b in banks_b)
     assert launches_b != launches_a                      # the pooled loop really took the other path
-    assert all(l.status() == L.OK for l in layers) and all(b.status() == L.OK for b in banks_a + banks_b)
-    for o in layers + banks_a + banks_b:
+    assert sum(b.stats()["kernel_launches"] for b in banks_c) == launches_b
+    assert [b.stats()["hits"] for b in banks_c] == [b.stats()["hits"] for b in banks_b]
+    assert all(l.status() == L.OK for l in layers) and all(b.status() == L.OK for b in banks_a + banks_b + banks_c)
+    for o in layers + banks_a + banks_b + banks_c:
         o.close()
 
 
