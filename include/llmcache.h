@@ -221,7 +221,8 @@ int llmcache_fingerprint_static_status(void);
  * against every occupied slot, best slot (ties: lowest), hit iff best > tau
  * (>= under LLMCACHE_GE).  h_out[b] (device bf16 [B,n,d]) receives the stored
  * layer output of each hit, byte for byte; rows of misses are left untouched.
- * tau: NaN => the bank's default.  B == 0 is valid and does nothing but tick.
+ * tau: NaN => the bank's default.  B == 0 is valid and does nothing but tick.  A bank serves 2^32 - 1 probe
+ * calls (the recency stamps are 32-bit ticks); the next one returns LLMCACHE_ERR_STATE.
  * All sequences see the bank as it was when the call began. */
 int llmcache_probe(llmcache_bank_t* bank, const void* h_in, uint32_t B, float tau,
                    void* h_out, llmcache_probe_io* io, void* stream);

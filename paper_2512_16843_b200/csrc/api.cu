@@ -353,6 +353,7 @@ static int probe_common(llmcache_bank_t* bk, const void* h_in, bool compute_fp, 
     return LLMCACHE_ERR_ARG;
   }
   if (std::isnan(tau)) tau = bk->desc.tau;
+  if (bk->tick >= 0xFFFFFFFFull) return LLMCACHE_ERR_STATE;       // the device keeps ticks in 32 bits
   DeviceGuard guard(bk->desc.device);
   if (!guard.ok) return LLMCACHE_ERR_CUDA;
   cudaStream_t st = (cudaStream_t)stream;
@@ -533,13 +534,13 @@ int llmcache_bank_stats(llmcache_bank_t* bk, llmcache_stats* out) {
     cudaGetLastError();
     return LLMCACHE_ERR_CUDA;
   }
-  const size_t N = bk->desc.capacity;
-  uint8_t* v = (uint8_t*)std::malloc(N);
-  if (!v) return LLMCACHE_ERR_NOMEM;
-  if (cudaMemcpy(v, bk->a.valid, N, cudaMemcpyDeviceToHost) != cudaSuccess) { std::free(v); cudaGetLastError(); return LLMCACHE_ERR_CUDA; }
-  uint64_t res = 0;
-  for (size_t i = 0; i < N; ++i) res += v[i] ? 1 : 0;
-  std::free(v);
+  // occupied slots, counted on the device (misc[4] is free between calls: the device is idle here)
+  uint32_t res = 0;
+  if (launch_count_valid(bk, bk->a.misc + 4, nullptr) != cudaSuccess || cudaDeviceSynchronize() != cudaSuccess ||
+      cudaMemcpy(&res, bk->a.misc + 4, sizeof(res), cudaMemcpyDeviceToHost) != cudaSuccess) {
+    cudaGetLastError();
+    return LLMCACHE_ERR_CUDA;
+  }
   out->probes = bk->n_probes;
   out->sequences = h[ST_SEQ];
   out->hits = h[ST_HIT];

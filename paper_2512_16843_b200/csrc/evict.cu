@@ -40,6 +40,21 @@ __global__ void k_evict(uint8_t* __restrict__ valid, const uint32_t* __restrict_
   }
 }
 
+// Number of occupied slots (for llmcache_bank_stats): one thread per slot, one atomic per warp.
+__global__ void k_count_valid(const uint8_t* __restrict__ valid, uint32_t N, uint32_t* __restrict__ count) {
+  const uint32_t i = blockIdx.x * blockDim.x + threadIdx.x;
+  const uint32_t bal = __ballot_sync(0xFFFFFFFFu, i < N && valid[i] != 0);
+  if ((threadIdx.x & 31) == 0 && bal) atomicAdd(count, (uint32_t)__popc(bal));
+}
+
+cudaError_t launch_count_valid(llmcache_bank* bk, uint32_t* count_dev, cudaStream_t st) {
+  cudaError_t e = cudaMemsetAsync(count_dev, 0, sizeof(uint32_t), st);
+  if (e != cudaSuccess) return e;
+  const uint32_t N = bk->desc.capacity;
+  k_count_valid<<<(N + 255) / 256, 256, 0, st>>>(bk->a.valid, N, count_dev);
+  return cudaGetLastError();
+}
+
 constexpr uint32_t SEL_ONE_BLOCK_MAX = 4096;
 
 // One block.  Runs on the bank's side stream, next to the gather of the same probe.

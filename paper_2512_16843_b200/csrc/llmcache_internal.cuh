@@ -145,6 +145,7 @@ cudaError_t launch_gather(llmcache_bank* bk, const void* h_in, void* h_out,
                           const llmcache_probe_io* io, uint32_t B, cudaStream_t st);
 cudaError_t launch_select_victims(llmcache_bank* bk, const llmcache_probe_io* io, uint32_t B, cudaStream_t st);
 cudaError_t setup_select_kernels();
+cudaError_t launch_count_valid(llmcache_bank* bk, uint32_t* count_dev, cudaStream_t st);
 cudaError_t launch_select_victims_mb(llmcache_bank* bk, const llmcache_probe_io* io, uint32_t B, cudaStream_t st);
 cudaError_t launch_scatter_insert(llmcache_bank* bk, const void* miss_out, const llmcache_probe_io* io,
                                   void* h_out, int32_t* new_slot_out, uint32_t B, cudaStream_t st);
