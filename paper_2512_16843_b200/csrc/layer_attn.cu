@@ -5,15 +5,16 @@
 // overlaps the other's matrix products.  Per tile of 128 keys:
 //   S  = Q K^T        tcgen05.mma 128 x 128 x 64 into tensor memory (Q and K tiles come straight out of the
 //                     [tokens, 3d] q|k|v matrix by TMA, 128-byte swizzle)
-//   P  = softmax step four warps, one thread per query row: two passes over the row in tensor memory (maximum, then
-//                     exponentials and their sum), P written as bf16 into shared memory in the swizzled K-major
-//                     layout the next product reads
+//   P  = softmax step eight warps, two threads per query row: two passes over the row in tensor memory (maximum,
+//                     then exponentials and their sum), P written as bf16 into shared memory in the swizzled
+//                     K-major layout the next product reads
 //   PV = P V          tcgen05.mma 128 x 64 x 128; V is read through its per-head transpose V^T [64, n] (written
 //                     by the epilogue of the q|k|v product), so that both operands are K-major
 //   O  = O * exp(m_old - m_new) + PV   in registers (running maximum m and sum l per row: on-line softmax)
 // causal: position i attends to j <= i; key tiles beyond the diagonal are skipped.
-// Warp 0 produces (TMA), warp 1 issues the MMAs and owns the tensor memory, warps 2..5 do the softmax and the
-// output.  Every wait is bounded (status word, as in scan.cu).
+// Warp 0 produces (TMA), warp 1 issues the MMAs and owns the tensor memory, warps 2..9 do the softmax and the
+// output.  Two accumulators of 128 columns alternate between key tiles, so that the S of the next tile is computed
+// while the softmax works on the current one.  Every wait is bounded (status word, as in scan.cu).
 #include <cuda.h>
 #include "llmcache_internal.cuh"
 #include "ptx.cuh"
