@@ -176,6 +176,9 @@ def parse():
     ap.add_argument("--batch", type=int, default=0, help="e2e_bert_base: sequences per batch (default 256)")
     ap.add_argument("--seq-len", type=int, default=0, help="e2e_bert_base: sequence length (default 384)")
     ap.add_argument("--layers", type=int, default=0, help="number of per-layer banks (default: the workload's; fewer only for profiler captures)")
+    ap.add_argument("--input-stable", type=int, default=1,
+                    help="1: tell the banks that the probe inputs are resident buffers that no kernel of the run writes "
+                         "(the pooling pass may then start before the preceding kernel has finished); 0: do not")
     ap.add_argument("--pool-batches", type=int, default=0, help="distinct input batches in rotation (default: the workload's)")
     return ap.parse_args()
 
@@ -341,6 +344,8 @@ def run_probe_workload(name, args, env, steps, warmup, e2e_steps, with_cpu, tau_
     banks = [L.Bank(device=local, capacity=N, seq_len=n, d_model=d, fp_dim=k, max_batch=B,
                     hidden_dtype=L.F32 if f32_in else L.BF16, proj=proj, tau=cfg["tau"], policy=L.LRU_STALENESS)
              for _ in range(Lyr)]
+    for b in banks:
+        b.input_stable(bool(args.input_stable))
     bufs = [L.ProbeBuffers(B, k, dev) for _ in range(Lyr)]
     P = cfg["pool_batches"]
     warm, pool = make_inputs(cfg, seed, dev)
@@ -498,6 +503,7 @@ def run_probe_workload(name, args, env, steps, warmup, e2e_steps, with_cpu, tau_
            "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
            "config": config_of(name, cfg, world),
            "observed": {"hit_fraction": hits / float(seqs), "hidden_dtype": "f32" if f32_in else "bf16",
+                        "input_stable": bool(args.input_stable),
                         "distinct_batches": P},
            "e2e": e2e, "gpu_launches": launches, "roofline": roof, "cpu_baseline": cpu, "clocks": clocks}
     if sweep is not None:

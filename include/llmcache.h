@@ -237,6 +237,14 @@ int llmcache_probe(llmcache_bank_t* bank, const void* h_in, uint32_t B, float ta
 int llmcache_probe_simhash(llmcache_bank_t* bank, const void* h_in, uint32_t B, float tau,
                            void* h_out, llmcache_probe_io* io, void* stream);
 
+/* A promise about the inputs of llmcache_probe / llmcache_fingerprint on this bank: with stable != 0 the caller
+ * states that h_in is never written by the kernel that precedes the call in its stream (it was produced earlier,
+ * or on another stream that has been waited for).  The pooling pass then starts reading h_in while that
+ * preceding kernel is still finishing, instead of after it.  Results are unchanged.  Do not set it when h_in is
+ * the output of the previous layer's kernels enqueued just before (the layer-wise loop of Algorithm 1 as
+ * llmcache_infer runs it): the pooling pass would read rows that are still being written.  Default: 0. */
+int llmcache_bank_input_stable(llmcache_bank_t* bank, int stable);
+
 /* Same with precomputed fingerprints (Algorithm 1 computes f_X once and reuses
  * it at every layer): io->fp holds bf16 [B,k] on entry; io->rq is written.
  * h_in may be NULL (then io->h_miss is not produced). */

@@ -37,7 +37,7 @@ EXPORTS = [
     "llmcache_layer_status", "llmcache_infer", "llmcache_divergence_check", "llmcache_probe_simhash",
     "llmcache_pool", "llmcache_fingerprint_pooled", "llmcache_probe_pooled", "llmcache_bank_pool_out",
     "llmcache_infer_pooled", "llmcache_fingerprint_static_status", "llmcache_bank_debug_knobs",
-    "llmcache_layer_debug_knobs", "llmcache_debug_bounds_build",
+    "llmcache_layer_debug_knobs", "llmcache_debug_bounds_build", "llmcache_bank_input_stable",
 ]
 KNOB_PRODUCER_IDLE = 1
 FINGERPRINT_STATIC_MAX_FLOATS = 2 * 1024 * 1024
@@ -145,6 +145,7 @@ def lib():
         L.llmcache_fingerprint_static_error.argtypes = []
         L.llmcache_fingerprint_static_status.argtypes = []
         L.llmcache_debug_bounds_build.argtypes = []
+        L.llmcache_bank_input_stable.argtypes = [vp, C.c_int]
         L.llmcache_bank_debug_knobs.argtypes = [vp, C.c_uint64, u32]
         L.llmcache_layer_debug_knobs.argtypes = [vp, C.c_uint64, u32]
         for name in EXPORTS:
@@ -453,6 +454,10 @@ class Bank:
 
     def debug_knobs(self, wait_limit_ns: int = 0, flags: int = 0):
         llmcache_bank_debug_knobs(self.handle, wait_limit_ns, flags)
+
+    def input_stable(self, stable: bool = True):
+        """Promise that probe inputs are never written by the kernel preceding the probe in its stream."""
+        _check(lib().llmcache_bank_input_stable(self.handle, 1 if stable else 0), "llmcache_bank_input_stable")
 
     def profile(self, enable: bool):
         llmcache_bank_profile(self.handle, enable)

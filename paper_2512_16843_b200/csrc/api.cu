@@ -600,6 +600,12 @@ int llmcache_debug_bounds_build(void) {
 #endif
 }
 
+int llmcache_bank_input_stable(llmcache_bank_t* bk, int stable) {
+  if (!bk) return LLMCACHE_ERR_ARG;
+  bk->input_stable = stable != 0;
+  return LLMCACHE_OK;
+}
+
 int llmcache_bank_debug_knobs(llmcache_bank_t* bk, uint64_t wait_limit_ns, uint32_t flags) {
   if (!bk) return LLMCACHE_ERR_ARG;
   DeviceGuard guard(bk->desc.device);

@@ -15,7 +15,7 @@ namespace llmc {
 template <bool BF16>
 __global__ void __launch_bounds__(1024, 1)
 k_pool(const uint4* __restrict__ h, float* __restrict__ partial, uint32_t* __restrict__ status, PoolShape S) {
-  griddep_sync();
+  if (!S.early) griddep_sync();
   extern __shared__ __align__(128) uint8_t sm_raw[];
   pool_phase<BF16>(sm_raw, h, partial, status, S);
 }
@@ -223,14 +223,14 @@ PoolPlan pool_plan(uint32_t B, uint32_t n, uint32_t d, bool bf16, int sm_count) 
   return P;
 }
 
-static PoolShape pool_shape(const PoolPlan& P, uint32_t B, uint32_t n, uint32_t d) {
-  return PoolShape{B, n, d, P.V, P.R, P.L, P.Jmax, P.stage_rows, P.stages, P.cons_threads};
+static PoolShape pool_shape(const PoolPlan& P, uint32_t B, uint32_t n, uint32_t d, bool early) {
+  return PoolShape{B, n, d, P.V, P.R, P.L, P.Jmax, P.stage_rows, P.stages, P.cons_threads, early ? 1u : 0u};
 }
 
 static cudaError_t launch_pool(const PoolPlan& P, bool bf16, const void* h_in, float* partial, uint32_t* status,
-                               uint32_t B, uint32_t n, uint32_t d, cudaStream_t st) {
+                               uint32_t B, uint32_t n, uint32_t d, cudaStream_t st, bool early = false) {
   return launch_k(bf16 ? k_pool<true> : k_pool<false>, dim3(P.grid), dim3(P.threads), P.smem, st,
-                  (const uint4*)h_in, partial, status, pool_shape(P, B, n, d));
+                  (const uint4*)h_in, partial, status, pool_shape(P, B, n, d, early));
 }
 
 // Second kernel of the fingerprint: from the pooling pass's partial sums (pooled == nullptr) or from given
@@ -272,7 +272,7 @@ cudaError_t launch_fingerprint(llmcache_bank* bk, const void* h_in, uint32_t B,
   cudaError_t e;
   {
     ProfScope prof(bk, LLMCACHE_K_POOL, st);
-    e = launch_pool(P, bf16, h_in, bk->a.pool_partial, bk->a.status, B, D.seq_len, D.d_model, st);
+    e = launch_pool(P, bf16, h_in, bk->a.pool_partial, bk->a.status, B, D.seq_len, D.d_model, st, bk->input_stable);
   }
   if (e != cudaSuccess) return e;
   ProfScope prof(bk, LLMCACHE_K_PROJECT, st);

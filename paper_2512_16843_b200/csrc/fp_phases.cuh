@@ -40,7 +40,9 @@ __device__ __forceinline__ volatile uint32_t* head_flags(uint8_t* sm) {
 // in a fixed order (deterministic).  A stage never crosses a sequence boundary.
 // Threads [0, cons_threads) consume, thread cons_threads produces.  Called by all threads of the block.
 // ---------------------------------------------------------------------------
-struct PoolShape { uint32_t B, n, d, V, R, L, Jmax, stage_rows, stages, cons_threads; };
+// early: the input is not written by the grid that precedes this one in the stream (the caller says so), so the
+// producer may start streaming it before that grid has finished; the consumers still wait before they write.
+struct PoolShape { uint32_t B, n, d, V, R, L, Jmax, stage_rows, stages, cons_threads, early; };
 
 template <bool BF16>
 __device__ __forceinline__ void pool_phase(uint8_t* sm, const uint4* __restrict__ h, float* __restrict__ partial,
@@ -76,6 +78,7 @@ __device__ __forceinline__ void pool_phase(uint8_t* sm, const uint4* __restrict_
 
   if (threadIdx.x >= cons_threads) {
     // ---------------------------------------------------------------- producer (one thread)
+    if (S.early) asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
     if (threadIdx.x == cons_threads && !producer_idle(status)) {
       bool ok = true;
       while (r < r1 && ok) {
@@ -106,6 +109,7 @@ __device__ __forceinline__ void pool_phase(uint8_t* sm, const uint4* __restrict_
     }
   } else {
     // ---------------------------------------------------------------- consumers
+    if (S.early) griddep_sync();                       // nothing is written to global memory before this
     const bool active = threadIdx.x < V * R;
     const uint32_t col = threadIdx.x % V, rg = threadIdx.x / V;
     float* out = partial + (size_t)blockIdx.x * S.Jmax * d;

@@ -86,6 +86,7 @@ struct llmcache_bank {
   bool     join_pending = false;
   bool     select_deferred = false;   // large bank: the victim selection runs at commit instead
   bool     bits_dirty = true;    // stored fingerprints changed since the SimHash codes were packed
+  bool     input_stable = false; // llmcache_bank_input_stable: h_in is never the output of the preceding kernel
   // fingerprint-on-write: where the position means of the rows written in a tick go (nullptr: off)
   float*   pool_out = nullptr;
   uint32_t pool_out_ld = 0;

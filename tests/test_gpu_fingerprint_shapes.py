@@ -63,3 +63,31 @@ def test_projected_fingerprint_ragged_shapes(B, n, d, k, use_center, dtype):
     assert bank.status() == L.OK
     U.compare_fingerprints(U.bits(fp2), rq2.cpu().numpy(), want_fp, want_rq)
     bank.close()
+
+
+def test_input_stable_promise_changes_nothing_but_the_start_of_the_pooling_pass():
+    """With llmcache_bank_input_stable the pooling pass streams its input before the preceding kernel of the
+    stream has finished; the fingerprints, decisions and bank state must be bit-identical to the ordinary path."""
+    N, n, d, k, B = 256, 96, 256, 128, 70
+    proj = synth.projection(d, k, 5, DEV)
+    mk = lambda: L.Bank(capacity=N, seq_len=n, d_model=d, fp_dim=k, max_batch=B, hidden_dtype=L.BF16, proj=proj, tau=0.9)
+    ga, gb = mk(), mk()
+    gb.input_stable(True)
+    ba, bb = L.ProbeBuffers(B, k, DEV), L.ProbeBuffers(B, k, DEV)
+    big = torch.empty(64 * 1024 * 1024, dtype=torch.uint8, device=DEV)
+    for step in range(3):
+        h = synth.randn((B, n, d), 40 + step % 2, DEV, torch.bfloat16)       # the third batch repeats the first
+        mo = synth.activations(B, n, d, 50 + step, DEV)
+        for g, b in ((ga, ba), (gb, bb)):
+            big.fill_(step)                                                   # a kernel that is still running when the probe is enqueued
+            g.probe(h, b)
+            g.commit(mo, b)
+        torch.cuda.synchronize()
+        assert torch.equal(ba.fp.view(torch.int16), bb.fp.view(torch.int16))
+        assert torch.equal(ba.rq.view(torch.int32), bb.rq.view(torch.int32))
+        assert torch.equal(ba.hit, bb.hit) and torch.equal(ba.slot, bb.slot)
+    for what in (L.WHAT_FP, L.WHAT_VALID, L.WHAT_LAST_USE, L.WHAT_RATE):
+        assert torch.equal(ga.export(what), gb.export(what))
+    assert int(ba.counts[0]) == B and ga.status() == L.OK and gb.status() == L.OK
+    ga.close()
+    gb.close()
