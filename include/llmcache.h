@@ -237,6 +237,29 @@ int llmcache_probe(llmcache_bank_t* bank, const void* h_in, uint32_t B, float ta
 int llmcache_probe_simhash(llmcache_bank_t* bank, const void* h_in, uint32_t B, float tau,
                            void* h_out, llmcache_probe_io* io, void* stream);
 
+/* A bank split over several objects, one per GPU (the paper's outlook, Sec. VI-E, names sharing one cache between
+ * devices as future work; this is the lookup half of it).  Part p holds the slots [slot_base_p, slot_base_p +
+ * capacity_p) of a bank of n_total slots; every part sees the same batch of query fingerprints.
+ *   1. llmcache_shard_scan on every part: the best (score, slot) of each query over the part's keys is combined
+ *      by a 64-bit maximum into words[b] (device u64 [B]; the caller sets them to zero before the first part's
+ *      scan).  A word is (score in an order-preserving integer form) << 32 | (2^32 - 1 - slot of the whole bank),
+ *      so that the unsigned maximum of two words is the better match, the lower slot on equal scores.
+ *   2. the caller takes the element-wise unsigned maximum of the words over all parts (between GPUs: an
+ *      all-reduce(max); as signed 64-bit integers after flipping the top bit).  This is the one exchange step.
+ *   3. llmcache_shard_decide on every part with its own copy of the combined words: threshold, hit flags, slots of
+ *      the whole bank, scores, ascending index lists and counts -- identical in every part --, the metadata
+ *      refresh of the matched slots the part owns, and, with h_out, the stored outputs of the hits the part owns
+ *      (rows of other parts' hits and of misses are left untouched).  io->fp holds the query fingerprints on entry
+ *      (as for llmcache_probe_fp); io->rq is written.  The words are consumed (set to zero).  Advances the tick
+ *      like a probe and opens a probe: llmcache_commit may follow, with an io that lists this part's share of the
+ *      misses (miss_idx, counts[1], and miss_out rows in that order; fp and rq of the whole batch; the generation
+ *      that llmcache_shard_decide wrote).  How the misses are shared out is the caller's choice.
+ * slot_base + capacity <= n_total <= 2^31. */
+int llmcache_shard_scan(llmcache_bank_t* bank, const void* fp, uint32_t B, uint32_t slot_base, uint64_t* words,
+                        void* stream);
+int llmcache_shard_decide(llmcache_bank_t* bank, uint64_t* words, uint32_t B, float tau, uint32_t slot_base,
+                          uint32_t n_total, void* h_out, llmcache_probe_io* io, void* stream);
+
 /* A promise about the inputs of llmcache_probe / llmcache_fingerprint on this bank: with stable != 0 the caller
  * states that h_in is never written by the kernel that precedes the call in its stream (it was produced earlier,
  * or on another stream that has been waited for).  The pooling pass then starts reading h_in while that

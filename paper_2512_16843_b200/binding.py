@@ -38,6 +38,7 @@ EXPORTS = [
     "llmcache_pool", "llmcache_fingerprint_pooled", "llmcache_probe_pooled", "llmcache_bank_pool_out",
     "llmcache_infer_pooled", "llmcache_fingerprint_static_status", "llmcache_bank_debug_knobs",
     "llmcache_layer_debug_knobs", "llmcache_debug_bounds_build", "llmcache_bank_input_stable",
+    "llmcache_shard_scan", "llmcache_shard_decide",
 ]
 KNOB_PRODUCER_IDLE = 1
 FINGERPRINT_STATIC_MAX_FLOATS = 2 * 1024 * 1024
@@ -146,6 +147,8 @@ def lib():
         L.llmcache_fingerprint_static_status.argtypes = []
         L.llmcache_debug_bounds_build.argtypes = []
         L.llmcache_bank_input_stable.argtypes = [vp, C.c_int]
+        L.llmcache_shard_scan.argtypes = [vp, vp, u32, u32, vp, vp]
+        L.llmcache_shard_decide.argtypes = [vp, vp, u32, C.c_float, u32, u32, vp, C.POINTER(ProbeIO), vp]
         L.llmcache_bank_debug_knobs.argtypes = [vp, C.c_uint64, u32]
         L.llmcache_layer_debug_knobs.argtypes = [vp, C.c_uint64, u32]
         for name in EXPORTS:
@@ -315,6 +318,16 @@ def llmcache_debug_bounds_build() -> bool:
 
 def llmcache_fingerprint_static_status() -> int:
     return int(lib().llmcache_fingerprint_static_status())
+
+
+def llmcache_shard_scan(bank, fp, B, slot_base, words, stream=None) -> None:
+    _check(lib().llmcache_shard_scan(bank, _ptr(fp), B, slot_base, _ptr(words), _stream(stream)), "llmcache_shard_scan")
+
+
+def llmcache_shard_decide(bank, words, B, tau, slot_base, n_total, h_out, io: ProbeIO, stream=None) -> None:
+    tau = float("nan") if tau is None else tau
+    _check(lib().llmcache_shard_decide(bank, _ptr(words), B, tau, slot_base, n_total, _ptr(h_out), C.byref(io),
+                                       _stream(stream)), "llmcache_shard_decide")
 
 
 def llmcache_bank_profile(bank, enable: bool) -> None:

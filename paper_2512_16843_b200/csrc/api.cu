@@ -600,6 +600,59 @@ int llmcache_debug_bounds_build(void) {
 #endif
 }
 
+// ---- a bank split over several objects (or GPUs): scan, exchange of the best words by the caller, decision
+int llmcache_shard_scan(llmcache_bank_t* bk, const void* fp, uint32_t B, uint32_t slot_base, uint64_t* words,
+                        void* stream) {
+  if (!bk || (B && (!fp || !words))) return LLMCACHE_ERR_ARG;
+  if (B > bk->desc.max_batch) return LLMCACHE_ERR_SHAPE;
+  if (!aligned16(fp) || ((uintptr_t)words & 7u)) return LLMCACHE_ERR_ARG;
+  if ((unsigned long long)slot_base + bk->desc.capacity > (1ull << 31)) return LLMCACHE_ERR_SHAPE;
+  DeviceGuard guard(bk->desc.device);
+  if (!guard.ok) return LLMCACHE_ERR_CUDA;
+  cudaError_t e = launch_scan(bk, (const __nv_bfloat16*)fp, B, (cudaStream_t)stream, (unsigned long long*)words, slot_base);
+  return e == cudaSuccess ? LLMCACHE_OK : cuda_fail(e, __func__);
+}
+
+int llmcache_shard_decide(llmcache_bank_t* bk, uint64_t* words, uint32_t B, float tau, uint32_t slot_base,
+                          uint32_t n_total, void* h_out, llmcache_probe_io* io, void* stream) {
+  if (!bk || !io) return LLMCACHE_ERR_ARG;
+  if (B > bk->desc.max_batch) return LLMCACHE_ERR_SHAPE;
+  if ((unsigned long long)slot_base + bk->desc.capacity > n_total || n_total > (1u << 31)) return LLMCACHE_ERR_SHAPE;
+  if (B) {
+    int rc = check_io(io);
+    if (rc != LLMCACHE_OK) return rc;
+    if (!words || ((uintptr_t)words & 7u) || !aligned16(h_out)) return LLMCACHE_ERR_ARG;
+  }
+  if (std::isnan(tau)) tau = bk->desc.tau;
+  if (bk->tick >= 0xFFFFFFFFull) return LLMCACHE_ERR_STATE;
+  DeviceGuard guard(bk->desc.device);
+  if (!guard.ok) return LLMCACHE_ERR_CUDA;
+  cudaStream_t st = (cudaStream_t)stream;
+  bk->tick += 1;
+  bk->generation += 1;
+  bk->n_probes += 1;
+  io->generation = bk->generation;
+  bk->probe_open = true;
+  bk->last_B = B;
+  cudaError_t e = cudaSuccess;
+  if (bk->join_pending) {
+    e = cudaStreamWaitEvent(st, bk->ev_join, 0);
+    bk->join_pending = false;
+  }
+  bk->select_deferred = true;                       // the slots for this part's share of the misses are chosen at commit
+  bk->moved[0] = bk->moved[1] = false;
+  if (B == 0) {
+    if (e == cudaSuccess) e = cudaMemsetAsync(io->counts, 0, 2 * sizeof(uint32_t), st);
+  } else {
+    if (e == cudaSuccess) e = launch_rownorm(bk, (const __nv_bfloat16*)io->fp, B, bk->desc.fp_dim, io->rq, st);
+    if (e == cudaSuccess) e = launch_decide(bk, B, tau, io->rq, io, st, 0, -1, (unsigned long long*)words, slot_base, n_total);
+    if (e == cudaSuccess && h_out && bk->a.act) e = launch_gather(bk, nullptr, h_out, io, B, st, slot_base, n_total);
+  }
+  if (e == cudaSuccess && io->counts_host && io->counts)
+    e = cudaMemcpyAsync(io->counts_host, io->counts, 2 * sizeof(uint32_t), cudaMemcpyDeviceToHost, st);
+  return e == cudaSuccess ? LLMCACHE_OK : cuda_fail(e, __func__);
+}
+
 int llmcache_bank_input_stable(llmcache_bank_t* bk, int stable) {
   if (!bk) return LLMCACHE_ERR_ARG;
   bk->input_stable = stable != 0;

@@ -38,7 +38,12 @@ k_decide_compact(unsigned long long* __restrict__ best, const float* __restrict_
                  unsigned long long* __restrict__ stats,
                  uint32_t* __restrict__ last_use, uint32_t* __restrict__ hits_total, uint32_t* __restrict__ rate,
                  uint32_t* __restrict__ rate_epoch, uint32_t tick, uint32_t epoch,
-                 uint32_t sim_k, int32_t ham_max, uint32_t* __restrict__ status, uint32_t N) {
+                 uint32_t sim_k, int32_t ham_max, uint32_t* __restrict__ status, uint32_t N,
+                 uint32_t slot_base, uint32_t n_total) {
+  // slot_base, n_total: this bank holds the slots [slot_base, slot_base + N) of a bank of n_total slots that is
+  // split over several (0 and N for a whole bank).  The best words carry slot numbers of the whole bank; the
+  // decision, the reported slot and the index lists are the same in every part, the metadata refresh touches
+  // only the slots this part owns.
   griddep_sync();
   __shared__ uint32_t warp_tot[32];
   uint32_t hbase = 0, mbase = 0, ndegen = 0;
@@ -69,14 +74,14 @@ k_decide_compact(unsigned long long* __restrict__ best, const float* __restrict_
           sc = orderable_float((uint32_t)(pk >> 32)) * r;
           is_hit = cmp_ge ? (sc >= tau) : (sc > tau);
         }
-        if (!bounds_ok((uint32_t)sl < N, status, SITE_DECIDE)) is_hit = false;
+        if (!bounds_ok((uint32_t)sl < n_total, status, SITE_DECIDE)) is_hit = false;
       }
       if (!is_hit) sl = -1;
       hit[b] = is_hit ? 1 : 0;
       slot[b] = sl;
       score[b] = sc;
       my_slot = sl;
-      if (is_hit) atomicAdd(hitcnt + sl, 1u);
+      if (is_hit && (uint32_t)sl - slot_base < N) atomicAdd(hitcnt + ((uint32_t)sl - slot_base), 1u);
     }
     uint32_t nh;
     const uint32_t r = block_rank(is_hit, warp_tot, nh);
@@ -97,8 +102,9 @@ k_decide_compact(unsigned long long* __restrict__ best, const float* __restrict_
   for (uint32_t base = 0; base < B; base += DEC_THREADS) {
     const uint32_t b = base + threadIdx.x;
     if (b >= B) continue;
-    const int32_t j = n_chunks == 1 ? my_slot : slot[b];
-    if (j < 0) continue;
+    const int32_t jg = n_chunks == 1 ? my_slot : slot[b];
+    if (jg < 0 || (uint32_t)jg - slot_base >= N) continue;
+    const uint32_t j = (uint32_t)jg - slot_base;
     const uint32_t c = atomicExch(hitcnt + j, 0u);
     const uint32_t old_rate = rate[j], old_epoch = rate_epoch[j], old_hits = hits_total[j];
     if (c == 0) continue;
@@ -137,7 +143,7 @@ __global__ void __launch_bounds__(DEC_THREADS)
 k_decide_flags(unsigned long long* __restrict__ best, const float* __restrict__ rq, uint32_t B, float tau, int cmp_ge,
                uint8_t* __restrict__ hit, int32_t* __restrict__ slot, float* __restrict__ score,
                uint32_t* __restrict__ hitcnt, uint32_t* __restrict__ blk_cnt, uint32_t sim_k, int32_t ham_max,
-               uint32_t* __restrict__ status, uint32_t N) {
+               uint32_t* __restrict__ status, uint32_t N, uint32_t slot_base, uint32_t n_total) {
   griddep_sync();
   __shared__ uint32_t warp_tot[32];
   __shared__ uint32_t sdeg;
@@ -165,13 +171,13 @@ k_decide_flags(unsigned long long* __restrict__ best, const float* __restrict__ 
         sc = orderable_float((uint32_t)(pk >> 32)) * r;
         is_hit = cmp_ge ? (sc >= tau) : (sc > tau);
       }
-      if (!bounds_ok((uint32_t)sl < N, status, SITE_DECIDE)) is_hit = false;
+      if (!bounds_ok((uint32_t)sl < n_total, status, SITE_DECIDE)) is_hit = false;
     }
     if (!is_hit) sl = -1;
     hit[b] = is_hit ? 1 : 0;
     slot[b] = sl;
     score[b] = sc;
-    if (is_hit) atomicAdd(hitcnt + sl, 1u);
+    if (is_hit && (uint32_t)sl - slot_base < N) atomicAdd(hitcnt + ((uint32_t)sl - slot_base), 1u);
   }
   uint32_t nh;
   block_rank(is_hit, warp_tot, nh);
@@ -202,14 +208,15 @@ k_compact_touch(const uint8_t* __restrict__ hit, const int32_t* __restrict__ slo
                 const uint32_t* __restrict__ blk_cnt, int32_t* __restrict__ hit_idx, int32_t* __restrict__ miss_idx,
                 uint32_t* __restrict__ counts, uint32_t* __restrict__ hitcnt, unsigned long long* __restrict__ stats,
                 uint32_t* __restrict__ last_use, uint32_t* __restrict__ hits_total, uint32_t* __restrict__ rate,
-                uint32_t* __restrict__ rate_epoch, uint32_t tick, uint32_t epoch) {
+                uint32_t* __restrict__ rate_epoch, uint32_t tick, uint32_t epoch, uint32_t N, uint32_t slot_base) {
   griddep_sync();
   __shared__ uint32_t warp_tot[32];
   __shared__ uint32_t red[32];
   const uint32_t b = blockIdx.x * DEC_THREADS + threadIdx.x;
   const bool in_range = b < B;
   const bool is_hit = in_range && hit[b] != 0;
-  const int32_t j = is_hit ? slot[b] : -1;
+  const int32_t jg = is_hit ? slot[b] : -1;
+  const int32_t j = (jg >= 0 && (uint32_t)jg - slot_base < N) ? (int32_t)((uint32_t)jg - slot_base) : -1;   // owned: local index
   // hits in the blocks before this one
   uint32_t part = 0;
   for (uint32_t i = threadIdx.x; i < blockIdx.x; i += DEC_THREADS) part += blk_cnt[2 * i];
@@ -249,24 +256,31 @@ k_compact_touch(const uint8_t* __restrict__ hit, const int32_t* __restrict__ slo
   }
 }
 
+// words == nullptr: the bank's own best words; else `words` (of a bank split over several: slot numbers of the
+// whole bank of n_total slots, of which this bank holds [slot_base, slot_base + capacity)).
 cudaError_t launch_decide(llmcache_bank* bk, uint32_t B, float tau, const float* rq,
-                          const llmcache_probe_io* io, cudaStream_t st, uint32_t sim_k, int32_t ham_max) {
+                          const llmcache_probe_io* io, cudaStream_t st, uint32_t sim_k, int32_t ham_max,
+                          unsigned long long* words, uint32_t slot_base, uint32_t n_total) {
   ProfScope prof(bk, LLMCACHE_K_DECIDE, st);
   const uint32_t tick = (uint32_t)bk->tick, epoch = (uint32_t)(bk->tick / bk->pol.half_life);
+  const uint32_t N = bk->desc.capacity;
+  unsigned long long* best = words ? words : bk->a.best;
+  if (!words) { slot_base = 0; n_total = N; }
   if (B <= DEC_SINGLE_BLOCK_MAX)
-    return launch_k(k_decide_compact, dim3(1), dim3(DEC_THREADS), 0, st, bk->a.best, rq, B, tau,
+    return launch_k(k_decide_compact, dim3(1), dim3(DEC_THREADS), 0, st, best, rq, B, tau,
                     (int)(bk->desc.cmp == LLMCACHE_GE), io->hit, io->slot, io->score, io->hit_idx, io->miss_idx,
                     io->counts, bk->a.hitcnt, bk->a.stats, bk->a.last_use, bk->a.hits, bk->a.rate, bk->a.rate_epoch,
-                    tick, epoch, sim_k, ham_max, bk->a.status, bk->desc.capacity);
+                    tick, epoch, sim_k, ham_max, bk->a.status, N, slot_base, n_total);
   const uint32_t nblk = (B + DEC_THREADS - 1) / DEC_THREADS;
-  cudaError_t e = launch_k(k_decide_flags, dim3(nblk), dim3(DEC_THREADS), 0, st, bk->a.best, rq, B, tau,
+  cudaError_t e = launch_k(k_decide_flags, dim3(nblk), dim3(DEC_THREADS), 0, st, best, rq, B, tau,
                            (int)(bk->desc.cmp == LLMCACHE_GE), io->hit, io->slot, io->score, bk->a.hitcnt,
-                           bk->a.blk_cnt, sim_k, ham_max, bk->a.status, bk->desc.capacity);
+                           bk->a.blk_cnt, sim_k, ham_max, bk->a.status, N, slot_base, n_total);
   if (e != cudaSuccess) return e;
   bk->n_launches += 1;
   return launch_k(k_compact_touch, dim3(nblk), dim3(DEC_THREADS), 0, st, (const uint8_t*)io->hit,
                   (const int32_t*)io->slot, B, (const uint32_t*)bk->a.blk_cnt, io->hit_idx, io->miss_idx, io->counts,
-                  bk->a.hitcnt, bk->a.stats, bk->a.last_use, bk->a.hits, bk->a.rate, bk->a.rate_epoch, tick, epoch);
+                  bk->a.hitcnt, bk->a.stats, bk->a.last_use, bk->a.hits, bk->a.rate, bk->a.rate_epoch, tick, epoch,
+                  N, slot_base);
 }
 
 }  // namespace llmc

@@ -138,12 +138,15 @@ cudaError_t launch_pool_finish_moved(llmcache_bank* bk, const llmcache_probe_io*
                                      float* pooled, uint32_t ld, cudaStream_t st);
 cudaError_t launch_pool_finish_plain(llmcache_bank* bk, const PoolPlan& P, uint32_t B, float* pooled, uint32_t ld,
                                      cudaStream_t st);
-cudaError_t launch_scan(llmcache_bank* bk, const __nv_bfloat16* q, uint32_t B, cudaStream_t st);
+cudaError_t launch_scan(llmcache_bank* bk, const __nv_bfloat16* q, uint32_t B, cudaStream_t st,
+                        unsigned long long* words = nullptr, uint32_t slot_base = 0);
 cudaError_t launch_decide(llmcache_bank* bk, uint32_t B, float tau, const float* rq,
-                          const llmcache_probe_io* io, cudaStream_t st, uint32_t sim_k = 0, int32_t ham_max = -1);
+                          const llmcache_probe_io* io, cudaStream_t st, uint32_t sim_k = 0, int32_t ham_max = -1,
+                          unsigned long long* words = nullptr, uint32_t slot_base = 0, uint32_t n_total = 0);
 cudaError_t launch_simhash_scan(llmcache_bank* bk, const __nv_bfloat16* q, uint32_t B, cudaStream_t st);
 cudaError_t launch_gather(llmcache_bank* bk, const void* h_in, void* h_out,
-                          const llmcache_probe_io* io, uint32_t B, cudaStream_t st);
+                          const llmcache_probe_io* io, uint32_t B, cudaStream_t st, uint32_t slot_base = 0,
+                          uint32_t n_total = 0);
 cudaError_t launch_select_victims(llmcache_bank* bk, const llmcache_probe_io* io, uint32_t B, cudaStream_t st);
 cudaError_t setup_select_kernels();
 cudaError_t launch_count_valid(llmcache_bank* bk, uint32_t* count_dev, cudaStream_t st);

@@ -55,7 +55,7 @@ k_gather(const char* __restrict__ act, uint32_t act_rows, char* __restrict__ h_o
          const char* __restrict__ h_in, char* __restrict__ h_miss, size_t in_row_bytes,
          const int32_t* __restrict__ slot, const int32_t* __restrict__ hit_idx,
          const int32_t* __restrict__ miss_idx, const uint32_t* __restrict__ counts,
-         uint32_t* __restrict__ status, uint32_t B, uint32_t N) {
+         uint32_t* __restrict__ status, uint32_t B, uint32_t N, uint32_t slot_base, uint32_t n_total) {
   griddep_sync();
   const uint32_t H = counts[0], M = counts[1];
   const uint32_t upr = (uint32_t)((row_bytes + COPY_UNIT - 1) / COPY_UNIT);
@@ -70,8 +70,10 @@ k_gather(const char* __restrict__ act, uint32_t act_rows, char* __restrict__ h_o
       const unsigned long long left = (u1 < n_hit ? u1 : n_hit) - u;
       const uint32_t w1 = (uint32_t)min((unsigned long long)upr, w0 + left);
       const int32_t b = hit_idx[i];
-      if (bounds_ok(i < B && (uint32_t)b < B && (uint32_t)slot[b] < N, status, SITE_GATHER_HIT)) {
-        const uint32_t row = (uint32_t)slot[b] % act_rows;
+      // a bank that holds the slots [slot_base, slot_base + N) of a larger one copies the rows it owns
+      if (bounds_ok(i < B && (uint32_t)b < B && (uint32_t)slot[b] < n_total, status, SITE_GATHER_HIT) &&
+          (uint32_t)slot[b] - slot_base < N) {
+        const uint32_t row = ((uint32_t)slot[b] - slot_base) % act_rows;
         const size_t off = (size_t)w0 * COPY_UNIT;
         const uint32_t bytes = (uint32_t)(min(row_bytes, (size_t)w1 * COPY_UNIT) - off);
         copy_bytes(act + (size_t)row * row_bytes + off, h_out + (size_t)b * row_bytes + off, nullptr, bytes);
@@ -170,7 +172,7 @@ static uint32_t copy_grid(const llmcache_bank* bk, uint32_t B, size_t row_bytes,
 }
 
 cudaError_t launch_gather(llmcache_bank* bk, const void* h_in, void* h_out,
-                          const llmcache_probe_io* io, uint32_t B, cudaStream_t st) {
+                          const llmcache_probe_io* io, uint32_t B, cudaStream_t st, uint32_t slot_base, uint32_t n_total) {
   if (B == 0) return cudaSuccess;
   const llmcache_bank_desc& D = bk->desc;
   const size_t row_bytes = (size_t)D.seq_len * D.d_model * 2;
@@ -183,7 +185,7 @@ cudaError_t launch_gather(llmcache_bank* bk, const void* h_in, void* h_out,
                   (const char*)(want_hit ? bk->a.act : nullptr), D.act_rows, (char*)(want_hit ? h_out : nullptr), row_bytes,
                   (const char*)(want_miss ? h_in : nullptr), (char*)(want_miss ? io->h_miss : nullptr), in_row_bytes,
                   (const int32_t*)io->slot, (const int32_t*)io->hit_idx, (const int32_t*)io->miss_idx,
-                  (const uint32_t*)io->counts, bk->a.status, B, D.capacity);
+                  (const uint32_t*)io->counts, bk->a.status, B, D.capacity, slot_base, n_total ? n_total : D.capacity);
 }
 
 cudaError_t launch_scatter_insert(llmcache_bank* bk, const void* miss_out, const llmcache_probe_io* io,

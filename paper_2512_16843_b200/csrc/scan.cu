@@ -57,7 +57,8 @@ __global__ void __launch_bounds__(SCAN_THREADS, 1)
 k_scan_tc(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CUtensorMap map_bank,
           const float* __restrict__ rb, const uint8_t* __restrict__ valid,
           unsigned long long* __restrict__ best, uint32_t* __restrict__ status,
-          uint32_t B, uint32_t N, uint32_t KB, uint32_t MB, uint32_t NB, uint32_t chunk_len, uint32_t n_units) {
+          uint32_t B, uint32_t N, uint32_t KB, uint32_t MB, uint32_t NB, uint32_t chunk_len, uint32_t n_units,
+          uint32_t slot_base) {
   griddep_sync();
   extern __shared__ uint8_t smem_raw[];
   const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;
@@ -189,7 +190,8 @@ k_scan_tc(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CUt
         mbar_arrive(tempty_bar(buf));
       }
       const uint32_t b = mb * BM + row_in_tile;
-      if (!stop && b < B && best_j != 0xFFFFFFFFu) atomicMax(best + b, pack_best(best_s, best_j));
+      // slot_base: where this bank's slots start in a bank that is split over several (0 for a whole bank)
+      if (!stop && b < B && best_j != 0xFFFFFFFFu) atomicMax(best + b, pack_best(best_s, best_j + slot_base));
     }
   }
 
@@ -222,7 +224,8 @@ cudaError_t setup_scan_kernels() {
 }
 
 template <int BN>
-static cudaError_t launch_scan_bn(llmcache_bank* bk, const __nv_bfloat16* q, uint32_t B, cudaStream_t st) {
+static cudaError_t launch_scan_bn(llmcache_bank* bk, const __nv_bfloat16* q, uint32_t B, cudaStream_t st,
+                                  unsigned long long* words, uint32_t slot_base) {
   const uint32_t N = bk->desc.capacity, k = bk->desc.fp_dim;
   alignas(64) CUtensorMap map_q, map_bank;
   if (!make_tensor_map_bf16(&map_q, q, B, k, BM) || !make_tensor_map_bf16(&map_bank, bk->a.fp, N, k, BN))
@@ -239,17 +242,20 @@ static cudaError_t launch_scan_bn(llmcache_bank* bk, const __nv_bfloat16* q, uin
   const uint32_t grid = n_units < (uint32_t)bk->sm_count ? n_units : (uint32_t)bk->sm_count;
   ProfScope prof(bk, LLMCACHE_K_SCAN, st);
   return launch_k(k_scan_tc<BN>, dim3(grid), dim3(SCAN_THREADS), ScanSmem<BN>::BYTES, st, map_q, map_bank,
-                  (const float*)bk->a.rb, (const uint8_t*)bk->a.valid, bk->a.best, bk->a.status, B, N, KB, MB, NB,
-                  chunk_len, n_units);
+                  (const float*)bk->a.rb, (const uint8_t*)bk->a.valid, words ? words : bk->a.best, bk->a.status, B, N,
+                  KB, MB, NB, chunk_len, n_units, slot_base);
 }
 
-cudaError_t launch_scan(llmcache_bank* bk, const __nv_bfloat16* q, uint32_t B, cudaStream_t st) {
+// words == nullptr: best words go to the bank's own array; else to `words` (combined by atomicMax with what is
+// there), with slot numbers shifted by slot_base.
+cudaError_t launch_scan(llmcache_bank* bk, const __nv_bfloat16* q, uint32_t B, cudaStream_t st,
+                        unsigned long long* words, uint32_t slot_base) {
   if (B == 0) return cudaSuccess;
   // the widest key tile that still gives every SM a tile; small banks take narrower tiles
   const unsigned long long MB = (B + BM - 1) / BM, N = bk->desc.capacity, sms = (unsigned long long)bk->sm_count;
-  if (MB * ((N + 255) / 256) >= sms) return launch_scan_bn<256>(bk, q, B, st);
-  if (MB * ((N + 127) / 128) >= sms) return launch_scan_bn<128>(bk, q, B, st);
-  return launch_scan_bn<64>(bk, q, B, st);
+  if (MB * ((N + 255) / 256) >= sms) return launch_scan_bn<256>(bk, q, B, st, words, slot_base);
+  if (MB * ((N + 127) / 128) >= sms) return launch_scan_bn<128>(bk, q, B, st, words, slot_base);
+  return launch_scan_bn<64>(bk, q, B, st, words, slot_base);
 }
 
 }  // namespace llmc
