@@ -398,7 +398,8 @@ def test_more_victims_than_the_shared_memory_sort_holds(policy):
     gb.close()
 
 
-@pytest.mark.parametrize("N,B,steps", [(5000, 20000, 3), (40000, 20000, 5), (262144, 65536, 7)])
+@pytest.mark.parametrize("N,B,steps", [(5000, 20000, 3), (40000, 20000, 5), (262144, 65536, 7),
+                                       (4097, 2049, 4), (8193, 8200, 3), (16390, 16385, 3)])
 def test_large_bank_large_batch_commit_lockstep(N, B, steps):
     """Banks and batches for which the decision and the victim selection run as several grids: tens of
     thousands of misses per step take free slots first and then evict by (stale, decayed rate, last use, slot);
