@@ -18,15 +18,19 @@ constexpr int GEMM_THREADS = 192;                   // warp 0: TMA, warp 1: MMA,
 constexpr int GEMM_EPI = 128;
 constexpr uint32_t GA_BYTES = GM * GK * 2, GB_BYTES = GN * GK * 2;
 constexpr uint32_t G_TMEM_COLS = 512;
+constexpr uint32_t G_BOX_BYTES = GM * 32 * 2;       // one 32-column group of a tile: 128 rows of 64 bytes
 struct GemmSmem {
   static constexpr uint32_t A = 0;
   static constexpr uint32_t B = A + GSTAGES * GA_BYTES;
-  static constexpr uint32_t BIAS = B + GSTAGES * GB_BYTES;       // float [2][GN]
-  static constexpr uint32_t BAR = BIAS + 2 * GN * 4;
+  static constexpr uint32_t STG = B + GSTAGES * GB_BYTES;        // two output boxes on their way out
+  static constexpr uint32_t RES = STG + 2 * G_BOX_BYTES;         // two residual boxes on their way in
+  static constexpr uint32_t BIAS = RES + 2 * G_BOX_BYTES;        // float [GN]
+  static constexpr uint32_t BAR = BIAS + GN * 4;
   static constexpr uint32_t MISC = BAR + 16 * 8;
   static constexpr uint32_t TOTAL = MISC + 64;
 };
 constexpr uint32_t GEMM_SMEM_BYTES = GemmSmem::TOTAL + 1024;
+static_assert(GEMM_SMEM_BYTES <= 232448, "shared memory of one block");
 constexpr uint32_t G_IDESC = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(GN >> 3) << 17) | ((uint32_t)(GM >> 4) << 24);
 
 // GELU with the error function, 0.5 x (1 + erf(x / sqrt 2)).  erf by the rational approximation of Abramowitz &
@@ -84,6 +88,7 @@ __device__ __forceinline__ uint32_t pack_bf16(float a, float b) {
 
 __global__ void __launch_bounds__(GEMM_THREADS, 1)
 k_gemm_tc(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_w,
+          const __grid_constant__ CUtensorMap map_out, const __grid_constant__ CUtensorMap map_res,
           const float* __restrict__ bias, const __nv_bfloat16* __restrict__ residual,
           __nv_bfloat16* __restrict__ out, uint32_t* __restrict__ status,
           uint32_t M_max, uint32_t N, uint32_t KB, const uint32_t* __restrict__ m_seq_dev, uint32_t rows_per_seq,
@@ -93,12 +98,14 @@ k_gemm_tc(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUt
   const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;
   uint8_t* gbase = smem_raw + (base - smem_u32(smem_raw));
   const uint32_t sA = base + GemmSmem::A, sB = base + GemmSmem::B;
+  const uint32_t sSTG = base + GemmSmem::STG, sRES = base + GemmSmem::RES;
   float* sbias = reinterpret_cast<float*>(gbase + GemmSmem::BIAS);
   const uint32_t bar0 = base + GemmSmem::BAR;
   auto full_bar = [&](uint32_t s) { return bar0 + 8 * s; };
   auto empty_bar = [&](uint32_t s) { return bar0 + 8 * (GSTAGES + s); };
   auto tfull_bar = [&](uint32_t b) { return bar0 + 8 * (2 * GSTAGES + b); };
   auto tempty_bar = [&](uint32_t b) { return bar0 + 8 * (2 * GSTAGES + 2 + b); };
+  auto res_bar = [&](uint32_t b) { return bar0 + 8 * (2 * GSTAGES + 4 + b); };
   volatile uint32_t* misc = reinterpret_cast<volatile uint32_t*>(gbase + GemmSmem::MISC);
   volatile uint32_t* tmem_slot = misc + 0;
   volatile uint32_t* abort_flag = misc + 1;
@@ -117,7 +124,11 @@ k_gemm_tc(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUt
 
   if (threadIdx.x == 0) {
     for (uint32_t s = 0; s < GSTAGES; ++s) { mbar_init(full_bar(s), 1); mbar_init(empty_bar(s), 1); }
-    for (uint32_t b = 0; b < 2; ++b) { mbar_init(tfull_bar(b), 1); mbar_init(tempty_bar(b), GEMM_EPI); }
+    for (uint32_t b = 0; b < 2; ++b) {
+      mbar_init(tfull_bar(b), 1);
+      mbar_init(tempty_bar(b), GEMM_EPI);
+      mbar_init(res_bar(b), 1);
+    }
     misc[1] = 0; misc[2] = 0; misc[3] = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
@@ -132,7 +143,7 @@ k_gemm_tc(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUt
   tc_fence_after();
   const uint32_t tmem_base = *tmem_slot;
 
-  uint32_t issued = 0;
+  uint32_t issued = 0, r_issued = 0;
   if (warp == 0) {
     if (lane == 0 && !producer_idle(status)) {         // ---- TMA producer
       bool ok = true;
@@ -173,54 +184,112 @@ k_gemm_tc(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUt
       if (!ok) { *abort_flag = 1; atomicExch(status, 1u); }
     }
   } else {
-    // ---- epilogue: bias, activation, residual, bf16 store; thread = one output row of the tile
-    // (eight epilogue warps, two per 32 rows, were measured too: no faster)
+    // ---- epilogue: bias, activation, residual, bf16 output; thread = one output row of the tile, 32 columns at
+    // a time.  Full tiles leave through shared memory: every thread puts its 64 bytes of a 32-column group into
+    // a staging box (64-byte swizzle, so that the 16-byte stores of a warp spread over all banks) and one thread
+    // hands the box to the bulk-copy engine, which writes whole lines; the residual arrives the same way, two
+    // groups ahead.  (With one 16-byte store per thread and row the product ran at 0.6-0.75 of the rate of its own
+    // main loop: a warp's store touched 32 lines, and more epilogue warps changed nothing.)  The last, partial row
+    // block of a device-counted M and the transposed V columns use plain stores.
     const uint32_t et = threadIdx.x - 64, quarter = warp & 3u;
     const uint32_t row_in_tile = quarter * 32 + lane;
+    const uint32_t my_off = row_in_tile * 64u, sw = (row_in_tile >> 1) & 3u;
+    const bool use_res = residual != nullptr;
+    auto tile_full = [&](uint32_t t) { return (t / NB + 1) * GM <= M; };
+    uint32_t r_used = 0, n_staged = 0;
+    uint32_t ct = blockIdx.x, cg = 0;                  // next residual box to request (thread et == 0 only)
+    auto res_issue = [&]() {
+      while (ct < n_tiles && !tile_full(ct)) ct += gridDim.x;
+      if (ct >= n_tiles) return;
+      const uint32_t cmb = ct / NB, cnb = ct % NB, j = r_issued & 1u;
+      mbar_expect_tx(res_bar(j), G_BOX_BYTES);
+      tma_load_2d(sRES + j * G_BOX_BYTES, &map_res, (int)(cnb * GN + cg * 32), (int)(cmb * GM), res_bar(j));
+      ++r_issued;
+      if (++cg == GN / 32 || cnb * GN + cg * 32 >= N) { cg = 0; ct += gridDim.x; }
+    };
+    if (use_res && et == 0) { res_issue(); res_issue(); }
     uint32_t tile = 0;
     for (uint32_t t = blockIdx.x; t < n_tiles; t += gridDim.x, ++tile) {
       const uint32_t mb = t / NB, nb = t % NB;
       const uint32_t buf = tile & 1u, bph = (tile >> 1) & 1u;
-      float* bt = sbias + buf * GN;
       for (uint32_t x = et; x < GN; x += GEMM_EPI) {
         const uint32_t c = nb * GN + x;
-        bt[x] = (bias && c < N) ? bias[c] : 0.f;
+        sbias[x] = (bias && c < N) ? bias[c] : 0.f;
       }
-      if (et == 0) epi_go[buf] = *abort_flag;
+      if (et == 0) *epi_go = *abort_flag;
       asm volatile("bar.sync 1, 128;" ::: "memory");
-      if (epi_go[buf]) break;
+      if (*epi_go) break;
       if (!mbar_wait(tfull_bar(buf), bph, abort_flag, lim)) { *abort_flag = 1; atomicExch(status, 1u); }
       tc_fence_after();
       const uint32_t taddr = tmem_base + buf * GN + ((quarter * 32u) << 16);
       const uint32_t row = mb * GM + row_in_tile;
-      const bool row_ok = row < M;
+      const bool row_ok = row < M, staged = tile_full(t);
 #pragma unroll 1
       for (uint32_t c = 0; c < GN; c += 32) {
+        const uint32_t col0 = nb * GN + c;
+        if (col0 >= N) break;                           // N is a multiple of 64: a 32-column group is all in or all out
         uint32_t v[32];
         tc_ld_32x32(taddr + c, v);
         tc_wait_ld();
-        const uint32_t col0 = nb * GN + c;
-        if (row_ok && col0 < N) {                       // N is a multiple of 64: a 32-column group is all in or all out
-          float f[32];
+        float f[32];
 #pragma unroll
-          for (int i = 0; i < 32; ++i) f[i] = __uint_as_float(v[i]) + bt[c + i];
-          if (act == LAYER_ACT_GELU_ERF) {
+        for (int i = 0; i < 32; ++i) f[i] = __uint_as_float(v[i]) + sbias[c + i];
+        if (act == LAYER_ACT_GELU_ERF) {
 #pragma unroll
-            for (int i = 0; i < 32; i += 2) gelu_erf_pair(f[i], f[i + 1]);
-          } else if (act == LAYER_ACT_GELU_TANH) {
+          for (int i = 0; i < 32; i += 2) gelu_erf_pair(f[i], f[i + 1]);
+        } else if (act == LAYER_ACT_GELU_TANH) {
 #pragma unroll
-            for (int i = 0; i < 32; ++i) f[i] = gelu_tanh_f(f[i]);
-          }
-          if (vt.ptr && col0 >= vt.col0) {
-            // the V third of a q|k|v product goes out transposed per head, for the attention kernel:
-            // vt[((seq * heads + h) * 64 + c) * pitch + pos]; the lanes of a warp are consecutive positions
+          for (int i = 0; i < 32; ++i) f[i] = gelu_tanh_f(f[i]);
+        }
+        if (vt.ptr && col0 >= vt.col0) {
+          // the V third of a q|k|v product goes out transposed per head, for the attention kernel:
+          // vt[((seq * heads + h) * 64 + c) * pitch + pos]; the lanes of a warp are consecutive positions
+          if (row_ok) {
             const uint32_t seq = row / rows_per_seq, pos = row - seq * rows_per_seq;
             const uint32_t hc = col0 - vt.col0;                       // h * 64 + c of the first column
             __nv_bfloat16* dst = vt.ptr + ((size_t)seq * vt.heads * 64 + hc) * vt.pitch + pos;
 #pragma unroll
             for (int i = 0; i < 32; ++i) dst[(size_t)i * vt.pitch] = __float2bfloat16_rn(f[i]);
-            continue;
           }
+          continue;
+        }
+        if (staged) {
+          if (use_res) {
+            const uint32_t j = r_used & 1u;
+            if (!mbar_wait(res_bar(j), (r_used >> 1) & 1u, abort_flag, lim)) { *abort_flag = 1; atomicExch(status, 1u); }
+            ++r_used;
+            const uint8_t* rb = gbase + GemmSmem::RES + j * G_BOX_BYTES + my_off;
+#pragma unroll
+            for (uint32_t q = 0; q < 4; ++q) {
+              const uint4 r = *reinterpret_cast<const uint4*>(rb + ((q ^ sw) << 4));
+              const uint32_t w[4] = {r.x, r.y, r.z, r.w};
+#pragma unroll
+              for (int u = 0; u < 4; ++u) {
+                f[q * 8 + 2 * u]     += __uint_as_float(w[u] << 16);
+                f[q * 8 + 2 * u + 1] += __uint_as_float(w[u] & 0xFFFF0000u);
+              }
+            }
+          }
+          const uint32_t jb = n_staged & 1u;
+          ++n_staged;
+          if (et == 0) bulk_wait_read<1>();             // the box written two groups ago has been read out
+          asm volatile("bar.sync 1, 128;" ::: "memory");
+          if (use_res && et == 0) res_issue();          // everyone has read the residual box: refill it
+          uint8_t* ob = gbase + GemmSmem::STG + jb * G_BOX_BYTES + my_off;
+#pragma unroll
+          for (uint32_t q = 0; q < 4; ++q)
+            *reinterpret_cast<uint4*>(ob + ((q ^ sw) << 4)) =
+                make_uint4(pack_bf16(f[q * 8], f[q * 8 + 1]), pack_bf16(f[q * 8 + 2], f[q * 8 + 3]),
+                           pack_bf16(f[q * 8 + 4], f[q * 8 + 5]), pack_bf16(f[q * 8 + 6], f[q * 8 + 7]));
+          fence_async_smem();
+          asm volatile("bar.sync 1, 128;" ::: "memory");
+          if (et == 0) {
+            tma_store_2d(&map_out, (int)col0, (int)(mb * GM), sSTG + jb * G_BOX_BYTES);
+            bulk_commit();
+          }
+          continue;
+        }
+        if (row_ok) {
           const size_t off = (size_t)row * N + col0;
           if (residual) {
             const uint4* r4 = reinterpret_cast<const uint4*>(residual + off);
@@ -244,6 +313,13 @@ k_gemm_tc(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUt
       }
       tc_fence_before();
       mbar_arrive(tempty_bar(buf));
+      asm volatile("bar.sync 1, 128;" ::: "memory");   // the bias of the next tile overwrites this one's
+    }
+    if (et == 0) {
+      bulk_wait_all();
+      // residual boxes still on their way (only after a wait ran out): they must land before the block ends
+      volatile uint32_t never = 0;
+      for (; r_used < r_issued; ++r_used) mbar_wait(res_bar(r_used & 1u), (r_used >> 1) & 1u, &never, 200000000ull);
     }
   }
 
@@ -276,13 +352,16 @@ cudaError_t launch_gemm(const __nv_bfloat16* a, const __nv_bfloat16* w, const fl
                         uint32_t N, uint32_t K, const uint32_t* m_seq_dev, uint32_t rows_per_seq, uint32_t act,
                         int sm_count, cudaStream_t st, VtOut vt) {
   if (M_max == 0) return cudaSuccess;
-  alignas(64) CUtensorMap map_a, map_w;
-  if (!make_tensor_map_bf16(&map_a, a, M_max, K, GM) || !make_tensor_map_bf16(&map_w, w, N, K, GN))
+  if (residual && vt.ptr) return cudaErrorInvalidValue;      // the transposed columns take no residual
+  alignas(64) CUtensorMap map_a, map_w, map_out, map_res;
+  if (!make_tensor_map_bf16(&map_a, a, M_max, K, GM) || !make_tensor_map_bf16(&map_w, w, N, K, GN) ||
+      !make_tensor_map_bf16_box32(&map_out, out, M_max, N) ||
+      !make_tensor_map_bf16_box32(&map_res, residual ? residual : out, M_max, N))
     return cudaErrorInvalidValue;
   const uint32_t tiles = ((M_max + GM - 1) / GM) * ((N + GN - 1) / GN);
   const uint32_t grid = tiles < (uint32_t)sm_count ? tiles : (uint32_t)sm_count;
-  return launch_k(k_gemm_tc, dim3(grid), dim3(GEMM_THREADS), GEMM_SMEM_BYTES, st, map_a, map_w, bias, residual, out,
-                  status, M_max, N, K / GK, m_seq_dev, rows_per_seq, act, vt);
+  return launch_k(k_gemm_tc, dim3(grid), dim3(GEMM_THREADS), GEMM_SMEM_BYTES, st, map_a, map_w, map_out, map_res, bias,
+                  residual, out, status, M_max, N, K / GK, m_seq_dev, rows_per_seq, act, vt);
 }
 
 }  // namespace llmc

@@ -78,6 +78,25 @@ __device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* map
       "cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];"
       ::"r"(dst), "l"(map), "r"(c0), "r"(c1), "r"(bar) : "memory");
 }
+// asks L2 for a box ahead of time (no shared-memory destination, nothing to wait for)
+__device__ __forceinline__ void tma_prefetch_2d(const CUtensorMap* map, int c0, int c1) {
+  asm volatile("cp.async.bulk.prefetch.tensor.2d.L2.global.tile [%0, {%1, %2}];" ::"l"(map), "r"(c0), "r"(c1) : "memory");
+}
+// shared memory -> global box; completion is tracked by the issuing thread's bulk groups
+__device__ __forceinline__ void tma_store_2d(const CUtensorMap* map, int c0, int c1, uint32_t src) {
+  asm volatile("cp.async.bulk.tensor.2d.global.shared::cta.bulk_group [%0, {%1, %2}], [%3];"
+               ::"l"(map), "r"(c0), "r"(c1), "r"(src) : "memory");
+}
+__device__ __forceinline__ void bulk_commit() { asm volatile("cp.async.bulk.commit_group;" ::: "memory"); }
+// returns once at most PENDING of this thread's bulk groups still read their shared-memory source
+template <int PENDING>
+__device__ __forceinline__ void bulk_wait_read() {
+  asm volatile("cp.async.bulk.wait_group.read %0;" ::"n"(PENDING) : "memory");
+}
+// returns once all of this thread's bulk groups are complete (their writes performed)
+__device__ __forceinline__ void bulk_wait_all() { asm volatile("cp.async.bulk.wait_group 0;" ::: "memory"); }
+// makes this thread's shared-memory writes visible to the bulk-copy engine
+__device__ __forceinline__ void fence_async_smem() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
 __device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
 __device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
 __device__ __forceinline__ void tc_commit(uint32_t bar) {
@@ -147,5 +166,8 @@ bool make_tensor_map_bf16(CUtensorMap* map, const void* ptr, uint64_t rows, uint
 // of the matrix (a box that reaches them is filled with zeros there)
 bool make_tensor_map_bf16_pitch(CUtensorMap* map, const void* ptr, uint64_t rows, uint64_t k, uint64_t pitch,
                                 uint32_t box_rows);
+// boxes of 32 columns x 128 rows (64 bytes per row, 64-byte swizzle) of a dense [rows, cols] bf16 matrix: the
+// pieces in which the dense layers' epilogue stores its output and fetches the residual
+bool make_tensor_map_bf16_box32(CUtensorMap* map, const void* ptr, uint64_t rows, uint64_t cols);
 
 }  // namespace llmc
