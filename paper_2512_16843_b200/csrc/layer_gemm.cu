@@ -14,16 +14,16 @@ namespace llmc {
 
 namespace {
 constexpr int GM = 128, GN = 256, GK = 64, GSTAGES = 4, G_UMMA_K = 16;
-constexpr int GEMM_THREADS = 192;                   // warp 0: TMA, warp 1: MMA, warps 2..5: epilogue
-constexpr int GEMM_EPI = 128;
+constexpr int GEMM_THREADS = 320;                   // warp 0: TMA, warp 1: MMA, warps 2..9: epilogue (two sets of four)
+constexpr int GEMM_EPI = 256;
 constexpr uint32_t GA_BYTES = GM * GK * 2, GB_BYTES = GN * GK * 2;
 constexpr uint32_t G_TMEM_COLS = 512;
 constexpr uint32_t G_BOX_BYTES = GM * 32 * 2;       // one 32-column group of a tile: 128 rows of 64 bytes
 struct GemmSmem {
   static constexpr uint32_t A = 0;
   static constexpr uint32_t B = A + GSTAGES * GA_BYTES;
-  static constexpr uint32_t STG = B + GSTAGES * GB_BYTES;        // two output boxes on their way out
-  static constexpr uint32_t RES = STG + 2 * G_BOX_BYTES;         // two residual boxes on their way in
+  static constexpr uint32_t STG = B + GSTAGES * GB_BYTES;        // one output box per epilogue set on its way out
+  static constexpr uint32_t RES = STG + 2 * G_BOX_BYTES;         // one residual box per epilogue set on its way in
   static constexpr uint32_t BIAS = RES + 2 * G_BOX_BYTES;        // float [GN]
   static constexpr uint32_t BAR = BIAS + GN * 4;
   static constexpr uint32_t MISC = BAR + 16 * 8;
@@ -33,49 +33,38 @@ constexpr uint32_t GEMM_SMEM_BYTES = GemmSmem::TOTAL + 1024;
 static_assert(GEMM_SMEM_BYTES <= 232448, "shared memory of one block");
 constexpr uint32_t G_IDESC = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(GN >> 3) << 17) | ((uint32_t)(GM >> 4) << 24);
 
-// GELU with the error function, 0.5 x (1 + erf(x / sqrt 2)).  erf by the rational approximation of Abramowitz &
-// Stegun 7.1.26 (absolute error below 1.5e-7, far under the bf16 rounding of the result): one reciprocal, one
-// exponential and a degree-5 polynomial, without the branches of the library routine.
-__device__ __forceinline__ float rcp_approx(float x) {
-  float y;
-  asm("rcp.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
-  return y;
-}
-__device__ __forceinline__ float ex2_approx(float x) {
-  float y;
-  asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
-  return y;
-}
-__device__ __forceinline__ float gelu_erf_f(float x) {
-  const float z = fabsf(x) * 0.70710678118654752f;
-  const float t = rcp_approx(fmaf(0.3275911f, z, 1.0f));
-  float p = fmaf(1.061405429f, t, -1.453152027f);
-  p = fmaf(p, t, 1.421413741f);
-  p = fmaf(p, t, -0.284496736f);
-  p = fmaf(p, t, 0.254829592f);
-  const float e = ex2_approx(-1.4426950408889634f * z * z);
-  const float erf_abs = fmaf(-p * t, e, 1.0f);                      // erf(|x| / sqrt 2)
-  return 0.5f * x + 0.5f * fabsf(x) * erf_abs;                     // x (1 + sign(x) erf) / 2
-}
-// the same for two values at once, with packed fp32 arithmetic
-__device__ __forceinline__ void gelu_erf_pair(float& x0, float& x1) {
-  const float a0 = fabsf(x0), a1 = fabsf(x1);
-  const unsigned long long a = f2_pack(a0, a1);
-  const unsigned long long z = f2_mul(a, f2_pack(0.70710678118654752f, 0.70710678118654752f));
-  const unsigned long long den = f2_fma(f2_pack(0.3275911f, 0.3275911f), z, f2_pack(1.0f, 1.0f));
-  const unsigned long long t = f2_pack(rcp_approx(f2_lo(den)), rcp_approx(f2_hi(den)));
-  unsigned long long p = f2_fma(f2_pack(1.061405429f, 1.061405429f), t, f2_pack(-1.453152027f, -1.453152027f));
-  p = f2_fma(p, t, f2_pack(1.421413741f, 1.421413741f));
-  p = f2_fma(p, t, f2_pack(-0.284496736f, -0.284496736f));
-  p = f2_fma(p, t, f2_pack(0.254829592f, 0.254829592f));
-  const unsigned long long arg = f2_mul(f2_mul(z, z), f2_pack(-1.4426950408889634f, -1.4426950408889634f));
-  const unsigned long long e = f2_pack(ex2_approx(f2_lo(arg)), ex2_approx(f2_hi(arg)));
-  // erf(|x| / sqrt 2) = 1 - p t e;  gelu = x / 2 + |x| erf / 2
-  const unsigned long long erf_abs = f2_fma(f2_mul(p, t), f2_mul(e, f2_pack(-1.0f, -1.0f)), f2_pack(1.0f, 1.0f));
-  const unsigned long long half = f2_pack(0.5f, 0.5f);
-  const unsigned long long g = f2_fma(f2_mul(a, half), erf_abs, f2_mul(f2_pack(x0, x1), half));
-  x0 = f2_lo(g);
-  x1 = f2_hi(g);
+// GELU with the error function, x/2 + |x|/2 x erf(|x| / sqrt 2), for two values at once with packed fp32
+// arithmetic and no special-function instruction: on u = min(|x|, 3.3 sqrt 2) an odd polynomial u Q(u^2) with nine
+// coefficients stands for erf(u / sqrt 2) (beyond the clamp erf is within 3.1e-6 of its value there).  The
+// coefficients minimise the largest error of GELU itself (gelu_erf_fit.py, beside this file): 8.2e-5 absolute
+// with the float32 evaluation included, below the bf16 rounding of the result.  (The rational approximation with
+// a reciprocal and an exponential used before cost two special-function instructions per element, and those
+// bounded the epilogue of the first feed-forward product.)
+__device__ __forceinline__ unsigned long long f2_dup(float x) { return f2_pack(x, x); }
+// eight pairs at a time, stage by stage: the nine-term Horner chain of one pair is serial, eight of them side by
+// side keep the pipeline fed with two epilogue warps per scheduler
+__device__ __forceinline__ void gelu_erf2_x8(unsigned long long (&y)[8]) {
+  unsigned long long u[8], s[8], q[8];
+#pragma unroll
+  for (int j = 0; j < 8; ++j) {
+    u[j] = f2_pack(fminf(fabsf(f2_lo(y[j])), 4.666905f), fminf(fabsf(f2_hi(y[j])), 4.666905f));
+    s[j] = f2_mul(u[j], u[j]);
+  }
+#pragma unroll
+  for (int j = 0; j < 8; ++j) q[j] = f2_fma(f2_dup(4.615854921e-11f), s[j], f2_dup(-5.357377653e-09f));
+  const float k[7] = {2.722534873e-07f, -8.016299034e-06f, 1.529819274e-04f, -2.011742676e-03f,
+                      1.894705929e-02f, -1.315938234e-01f, 7.972128987e-01f};
+#pragma unroll
+  for (int t = 0; t < 7; ++t) {
+#pragma unroll
+    for (int j = 0; j < 8; ++j) q[j] = f2_fma(q[j], s[j], f2_dup(k[t]));
+  }
+#pragma unroll
+  for (int j = 0; j < 8; ++j) {
+    const unsigned long long erf_abs = f2_mul(u[j], q[j]);
+    const unsigned long long h = f2_pack(0.5f * fabsf(f2_lo(y[j])), 0.5f * fabsf(f2_hi(y[j])));
+    y[j] = f2_fma(h, erf_abs, f2_mul(y[j], f2_dup(0.5f)));
+  }
 }
 __device__ __forceinline__ float gelu_tanh_f(float x) {
   return 0.5f * x * (1.0f + tanhf(0.7978845608028654f * (x + 0.044715f * x * x * x)));
@@ -188,26 +177,31 @@ k_gemm_tc(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUt
     // a time.  Full tiles leave through shared memory: every thread puts its 64 bytes of a 32-column group into
     // a staging box (64-byte swizzle, so that the 16-byte stores of a warp spread over all banks) and one thread
     // hands the box to the bulk-copy engine, which writes whole lines; the residual arrives the same way, two
-    // groups ahead.  (With one 16-byte store per thread and row the product ran at 0.6-0.75 of the rate of its own
+    // one group ahead.  (With one 16-byte store per thread and row the product ran at 0.6-0.75 of the rate of its own
     // main loop: a warp's store touched 32 lines, and more epilogue warps changed nothing.)  The last, partial row
     // block of a device-counted M and the transposed V columns use plain stores.
-    const uint32_t et = threadIdx.x - 64, quarter = warp & 3u;
+    // Two sets of four warps share a tile: set 0 takes the even groups, set 1 the odd ones, each with its own
+    // staging box, residual box, named barrier and issuing thread, so that one set's arithmetic (the GELU is
+    // ~15 dependent instructions per element) covers the other's waits.
+    const uint32_t et = threadIdx.x - 64, set = et >> 7, st = et & 127u, quarter = warp & 3u;
+    const uint32_t set_bar = 2u + set;
     const uint32_t row_in_tile = quarter * 32 + lane;
     const uint32_t my_off = row_in_tile * 64u, sw = (row_in_tile >> 1) & 3u;
     const bool use_res = residual != nullptr;
     auto tile_full = [&](uint32_t t) { return (t / NB + 1) * GM <= M; };
-    uint32_t r_used = 0, n_staged = 0;
-    uint32_t ct = blockIdx.x, cg = 0;                  // next residual box to request (thread et == 0 only)
+    uint32_t r_used = 0;
+    uint32_t ct = blockIdx.x, cg = set;                // next residual box to request (thread st == 0 of the set only)
     auto res_issue = [&]() {
       while (ct < n_tiles && !tile_full(ct)) ct += gridDim.x;
       if (ct >= n_tiles) return;
-      const uint32_t cmb = ct / NB, cnb = ct % NB, j = r_issued & 1u;
-      mbar_expect_tx(res_bar(j), G_BOX_BYTES);
-      tma_load_2d(sRES + j * G_BOX_BYTES, &map_res, (int)(cnb * GN + cg * 32), (int)(cmb * GM), res_bar(j));
+      const uint32_t cmb = ct / NB, cnb = ct % NB;
+      mbar_expect_tx(res_bar(set), G_BOX_BYTES);
+      tma_load_2d(sRES + set * G_BOX_BYTES, &map_res, (int)(cnb * GN + cg * 32), (int)(cmb * GM), res_bar(set));
       ++r_issued;
-      if (++cg == GN / 32 || cnb * GN + cg * 32 >= N) { cg = 0; ct += gridDim.x; }
+      cg += 2;
+      if (cg >= GN / 32 || cnb * GN + cg * 32 >= N) { cg = set; ct += gridDim.x; }
     };
-    if (use_res && et == 0) { res_issue(); res_issue(); }
+    if (use_res && st == 0) res_issue();
     uint32_t tile = 0;
     for (uint32_t t = blockIdx.x; t < n_tiles; t += gridDim.x, ++tile) {
       const uint32_t mb = t / NB, nb = t % NB;
@@ -217,7 +211,7 @@ k_gemm_tc(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUt
         sbias[x] = (bias && c < N) ? bias[c] : 0.f;
       }
       if (et == 0) *epi_go = *abort_flag;
-      asm volatile("bar.sync 1, 128;" ::: "memory");
+      asm volatile("bar.sync 1, 256;" ::: "memory");
       if (*epi_go) break;
       if (!mbar_wait(tfull_bar(buf), bph, abort_flag, lim)) { *abort_flag = 1; atomicExch(status, 1u); }
       tc_fence_after();
@@ -225,7 +219,7 @@ k_gemm_tc(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUt
       const uint32_t row = mb * GM + row_in_tile;
       const bool row_ok = row < M, staged = tile_full(t);
 #pragma unroll 1
-      for (uint32_t c = 0; c < GN; c += 32) {
+      for (uint32_t c = set * 32; c < GN; c += 64) {
         const uint32_t col0 = nb * GN + c;
         if (col0 >= N) break;                           // N is a multiple of 64: a 32-column group is all in or all out
         uint32_t v[32];
@@ -233,11 +227,23 @@ k_gemm_tc(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUt
         tc_wait_ld();
         float f[32];
 #pragma unroll
-        for (int i = 0; i < 32; ++i) f[i] = __uint_as_float(v[i]) + sbias[c + i];
-        if (act == LAYER_ACT_GELU_ERF) {
+        for (int half = 0; half < 2; ++half) {
+          const float2* b2 = reinterpret_cast<const float2*>(sbias + c) + half * 8;
+          unsigned long long y[8];
 #pragma unroll
-          for (int i = 0; i < 32; i += 2) gelu_erf_pair(f[i], f[i + 1]);
-        } else if (act == LAYER_ACT_GELU_TANH) {
+          for (int j = 0; j < 8; ++j) {
+            const float2 b = b2[j];
+            y[j] = f2_add(f2_pack(__uint_as_float(v[half * 16 + 2 * j]), __uint_as_float(v[half * 16 + 2 * j + 1])),
+                          f2_pack(b.x, b.y));
+          }
+          if (act == LAYER_ACT_GELU_ERF) gelu_erf2_x8(y);
+#pragma unroll
+          for (int j = 0; j < 8; ++j) {
+            f[half * 16 + 2 * j] = f2_lo(y[j]);
+            f[half * 16 + 2 * j + 1] = f2_hi(y[j]);
+          }
+        }
+        if (act == LAYER_ACT_GELU_TANH) {
 #pragma unroll
           for (int i = 0; i < 32; ++i) f[i] = gelu_tanh_f(f[i]);
         }
@@ -255,10 +261,9 @@ k_gemm_tc(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUt
         }
         if (staged) {
           if (use_res) {
-            const uint32_t j = r_used & 1u;
-            if (!mbar_wait(res_bar(j), (r_used >> 1) & 1u, abort_flag, lim)) { *abort_flag = 1; atomicExch(status, 1u); }
+            if (!mbar_wait(res_bar(set), r_used & 1u, abort_flag, lim)) { *abort_flag = 1; atomicExch(status, 1u); }
             ++r_used;
-            const uint8_t* rb = gbase + GemmSmem::RES + j * G_BOX_BYTES + my_off;
+            const uint8_t* rb = gbase + GemmSmem::RES + set * G_BOX_BYTES + my_off;
 #pragma unroll
             for (uint32_t q = 0; q < 4; ++q) {
               const uint4 r = *reinterpret_cast<const uint4*>(rb + ((q ^ sw) << 4));
@@ -270,21 +275,19 @@ k_gemm_tc(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUt
               }
             }
           }
-          const uint32_t jb = n_staged & 1u;
-          ++n_staged;
-          if (et == 0) bulk_wait_read<1>();             // the box written two groups ago has been read out
-          asm volatile("bar.sync 1, 128;" ::: "memory");
-          if (use_res && et == 0) res_issue();          // everyone has read the residual box: refill it
-          uint8_t* ob = gbase + GemmSmem::STG + jb * G_BOX_BYTES + my_off;
+          if (st == 0) bulk_wait_read<0>();             // the set's previous box has been read out
+          asm volatile("bar.sync %0, 128;" ::"r"(set_bar) : "memory");
+          if (use_res && st == 0) res_issue();          // the whole set has read the residual box: refill it
+          uint8_t* ob = gbase + GemmSmem::STG + set * G_BOX_BYTES + my_off;
 #pragma unroll
           for (uint32_t q = 0; q < 4; ++q)
             *reinterpret_cast<uint4*>(ob + ((q ^ sw) << 4)) =
                 make_uint4(pack_bf16(f[q * 8], f[q * 8 + 1]), pack_bf16(f[q * 8 + 2], f[q * 8 + 3]),
                            pack_bf16(f[q * 8 + 4], f[q * 8 + 5]), pack_bf16(f[q * 8 + 6], f[q * 8 + 7]));
           fence_async_smem();
-          asm volatile("bar.sync 1, 128;" ::: "memory");
-          if (et == 0) {
-            tma_store_2d(&map_out, (int)col0, (int)(mb * GM), sSTG + jb * G_BOX_BYTES);
+          asm volatile("bar.sync %0, 128;" ::"r"(set_bar) : "memory");
+          if (st == 0) {
+            tma_store_2d(&map_out, (int)col0, (int)(mb * GM), sSTG + set * G_BOX_BYTES);
             bulk_commit();
           }
           continue;
@@ -313,13 +316,13 @@ k_gemm_tc(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUt
       }
       tc_fence_before();
       mbar_arrive(tempty_bar(buf));
-      asm volatile("bar.sync 1, 128;" ::: "memory");   // the bias of the next tile overwrites this one's
+      asm volatile("bar.sync 1, 256;" ::: "memory");   // the bias of the next tile overwrites this one's
     }
-    if (et == 0) {
+    if (st == 0) {
       bulk_wait_all();
       // residual boxes still on their way (only after a wait ran out): they must land before the block ends
       volatile uint32_t never = 0;
-      for (; r_used < r_issued; ++r_used) mbar_wait(res_bar(r_used & 1u), (r_used >> 1) & 1u, &never, 200000000ull);
+      for (; r_used < r_issued; ++r_used) mbar_wait(res_bar(set), r_used & 1u, &never, 200000000ull);
     }
   }
 
