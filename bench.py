@@ -150,9 +150,9 @@ def make_inputs(cfg, seed, dev):
 NCU_TRAFFIC = {
     # two-layer case of the same workload (same launch shapes, same hit fraction: no scaling needed)
     "bert_large_churn": {
-        "pool": {"file": "fp_phases.cuh", "sha": "3b5339583ee2", "bytes_per_launch": 539716000},
-        "gather": {"file": "rows.cu", "sha": "0cbeb35c5bf2", "bytes_per_launch": 712760000},
-        "scatter": {"file": "rows.cu", "sha": "0cbeb35c5bf2", "bytes_per_launch": 350839000},
+        "pool": {"file": "fp_phases.cuh", "sha": "8c6604ef24f0", "bytes_per_launch": 538869000},
+        "gather": {"file": "rows.cu", "sha": "d5888d0fc059", "bytes_per_launch": 712128000},
+        "scatter": {"file": "rows.cu", "sha": "d5888d0fc059", "bytes_per_launch": 353201000},
     },
 }
 
