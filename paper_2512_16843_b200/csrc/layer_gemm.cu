@@ -1,9 +1,10 @@
 // Dense layer of the miss path: C[M, N] = act(A[M, K] . W[N, K]^T + bias) (+ residual), bf16 in and
 // out, fp32 accumulation.  The transformer layer f_l that runs on the misses (Algorithm 1,
 // "h_l <- f_l(h_{l-1})") is made of four of these.  Same machinery as the bank scan: TMA (128-byte
-// swizzle) into a 4-stage ring, tcgen05.mma 128 x 256 x 16 into two TMEM accumulators, epilogue warps
-// that drain one accumulator while the next tile's MMAs run.  The number of valid rows may come from
-// device memory (the miss count of the probe that precedes it), so no host sync is needed.
+// swizzle) into a 4-stage ring, tcgen05.mma 128 x 256 x 16 into two TMEM accumulators, eight epilogue warps
+// that drain one accumulator while the next tile's MMAs run and hand their output to the bulk-copy engine
+// through shared memory.  The number of valid rows may come from device memory (the miss count of the probe
+// that precedes it), so no host sync is needed.
 // All mbarrier waits are bounded (status word, see scan.cu).
 #include <cuda.h>
 #include "llmcache_internal.cuh"
@@ -224,6 +225,19 @@ k_gemm_tc(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUt
         if (col0 >= N) break;                           // N is a multiple of 64: a 32-column group is all in or all out
         uint32_t v[32];
         tc_ld_32x32(taddr + c, v);
+        // the residual of this group goes to registers first and its box is refilled at once, so that the next
+        // group's residual has this whole group's time to arrive
+        uint4 rr[4];
+        const bool res_here = staged && use_res;
+        if (res_here) {
+          if (!mbar_wait(res_bar(set), r_used & 1u, abort_flag, lim)) { *abort_flag = 1; atomicExch(status, 1u); }
+          ++r_used;
+          const uint8_t* rb = gbase + GemmSmem::RES + set * G_BOX_BYTES + my_off;
+#pragma unroll
+          for (uint32_t q = 0; q < 4; ++q) rr[q] = *reinterpret_cast<const uint4*>(rb + ((q ^ sw) << 4));
+          asm volatile("bar.sync %0, 128;" ::"r"(set_bar) : "memory");
+          if (st == 0) res_issue();
+        }
         tc_wait_ld();
         float f[32];
 #pragma unroll
@@ -261,13 +275,9 @@ k_gemm_tc(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUt
         }
         if (staged) {
           if (use_res) {
-            if (!mbar_wait(res_bar(set), r_used & 1u, abort_flag, lim)) { *abort_flag = 1; atomicExch(status, 1u); }
-            ++r_used;
-            const uint8_t* rb = gbase + GemmSmem::RES + set * G_BOX_BYTES + my_off;
 #pragma unroll
             for (uint32_t q = 0; q < 4; ++q) {
-              const uint4 r = *reinterpret_cast<const uint4*>(rb + ((q ^ sw) << 4));
-              const uint32_t w[4] = {r.x, r.y, r.z, r.w};
+              const uint32_t w[4] = {rr[q].x, rr[q].y, rr[q].z, rr[q].w};
 #pragma unroll
               for (int u = 0; u < 4; ++u) {
                 f[q * 8 + 2 * u]     += __uint_as_float(w[u] << 16);
@@ -277,7 +287,6 @@ k_gemm_tc(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUt
           }
           if (st == 0) bulk_wait_read<0>();             // the set's previous box has been read out
           asm volatile("bar.sync %0, 128;" ::"r"(set_bar) : "memory");
-          if (use_res && st == 0) res_issue();          // the whole set has read the residual box: refill it
           uint8_t* ob = gbase + GemmSmem::STG + set * G_BOX_BYTES + my_off;
 #pragma unroll
           for (uint32_t q = 0; q < 4; ++q)
