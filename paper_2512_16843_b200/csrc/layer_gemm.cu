@@ -23,11 +23,11 @@ constexpr uint32_t G_BOX_BYTES = GM * 32 * 2;       // one 32-column group of a 
 struct GemmSmem {
   static constexpr uint32_t A = 0;
   static constexpr uint32_t B = A + GSTAGES * GA_BYTES;
-  static constexpr uint32_t STG = B + GSTAGES * GB_BYTES;        // one output box per epilogue set on its way out
-  static constexpr uint32_t RES = STG + 2 * G_BOX_BYTES;         // one residual box per epilogue set on its way in
+  static constexpr uint32_t STG = B + GSTAGES * GB_BYTES;        // per epilogue set one box (four warps x 32 rows) on its way out
+  static constexpr uint32_t RES = STG + 2 * G_BOX_BYTES;         // the same for the residual on its way in
   static constexpr uint32_t BIAS = RES + 2 * G_BOX_BYTES;        // float [GN]
   static constexpr uint32_t BAR = BIAS + GN * 4;
-  static constexpr uint32_t MISC = BAR + 16 * 8;
+  static constexpr uint32_t MISC = BAR + 24 * 8;
   static constexpr uint32_t TOTAL = MISC + 64;
 };
 constexpr uint32_t GEMM_SMEM_BYTES = GemmSmem::TOTAL + 1024;
@@ -95,7 +95,7 @@ k_gemm_tc(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUt
   auto empty_bar = [&](uint32_t s) { return bar0 + 8 * (GSTAGES + s); };
   auto tfull_bar = [&](uint32_t b) { return bar0 + 8 * (2 * GSTAGES + b); };
   auto tempty_bar = [&](uint32_t b) { return bar0 + 8 * (2 * GSTAGES + 2 + b); };
-  auto res_bar = [&](uint32_t b) { return bar0 + 8 * (2 * GSTAGES + 4 + b); };
+  auto res_bar = [&](uint32_t w) { return bar0 + 8 * (2 * GSTAGES + 4 + w); };      // one per epilogue warp
   volatile uint32_t* misc = reinterpret_cast<volatile uint32_t*>(gbase + GemmSmem::MISC);
   volatile uint32_t* tmem_slot = misc + 0;
   volatile uint32_t* abort_flag = misc + 1;
@@ -117,8 +117,8 @@ k_gemm_tc(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUt
     for (uint32_t b = 0; b < 2; ++b) {
       mbar_init(tfull_bar(b), 1);
       mbar_init(tempty_bar(b), GEMM_EPI);
-      mbar_init(res_bar(b), 1);
     }
+    for (uint32_t w = 0; w < GEMM_EPI / 32; ++w) mbar_init(res_bar(w), 1);
     misc[1] = 0; misc[2] = 0; misc[3] = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
@@ -176,33 +176,34 @@ k_gemm_tc(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUt
   } else {
     // ---- epilogue: bias, activation, residual, bf16 output; thread = one output row of the tile, 32 columns at
     // a time.  Full tiles leave through shared memory: every thread puts its 64 bytes of a 32-column group into
-    // a staging box (64-byte swizzle, so that the 16-byte stores of a warp spread over all banks) and one thread
-    // hands the box to the bulk-copy engine, which writes whole lines; the residual arrives the same way, two
-    // one group ahead.  (With one 16-byte store per thread and row the product ran at 0.6-0.75 of the rate of its own
-    // main loop: a warp's store touched 32 lines, and more epilogue warps changed nothing.)  The last, partial row
-    // block of a device-counted M and the transposed V columns use plain stores.
-    // Two sets of four warps share a tile: set 0 takes the even groups, set 1 the odd ones, each with its own
-    // staging box, residual box, named barrier and issuing thread, so that one set's arithmetic (the GELU is
-    // ~15 dependent instructions per element) covers the other's waits.
-    const uint32_t et = threadIdx.x - 64, set = et >> 7, st = et & 127u, quarter = warp & 3u;
-    const uint32_t set_bar = 2u + set;
+    // its warp's 32-row staging box (64-byte swizzle, so that the 16-byte stores of a warp spread over all banks)
+    // and lane 0 hands the box to the bulk-copy engine, which writes whole lines; the residual rows arrive the same
+    // way, one group ahead.  (With one 16-byte store per thread and row the product ran at 0.6-0.75 of the rate of
+    // its own main loop: a warp's store touched 32 lines, and more epilogue warps changed nothing.)  The last,
+    // partial row block of a device-counted M and the transposed V columns use plain stores.
+    // Two sets of four warps share a tile: set 0 takes the even groups, set 1 the odd ones.  Every warp has its own
+    // boxes, residual barrier and bulk groups and meets the others only at the tile's ends, so that one warp's
+    // arithmetic (the GELU is a chain of dependent instructions) covers another's waits.
+    const uint32_t et = threadIdx.x - 64, set = et >> 7, quarter = warp & 3u;
+    const uint32_t ew = et >> 5;                        // epilogue warp 0..7
+    const uint32_t sub = set * G_BOX_BYTES + quarter * (G_BOX_BYTES / 4);     // this warp's 32 rows of its set's box
     const uint32_t row_in_tile = quarter * 32 + lane;
     const uint32_t my_off = row_in_tile * 64u, sw = (row_in_tile >> 1) & 3u;
     const bool use_res = residual != nullptr;
     auto tile_full = [&](uint32_t t) { return (t / NB + 1) * GM <= M; };
     uint32_t r_used = 0;
-    uint32_t ct = blockIdx.x, cg = set;                // next residual box to request (thread st == 0 of the set only)
+    uint32_t ct = blockIdx.x, cg = set;                // next residual rows to request (lane 0 of every warp)
     auto res_issue = [&]() {
       while (ct < n_tiles && !tile_full(ct)) ct += gridDim.x;
       if (ct >= n_tiles) return;
       const uint32_t cmb = ct / NB, cnb = ct % NB;
-      mbar_expect_tx(res_bar(set), G_BOX_BYTES);
-      tma_load_2d(sRES + set * G_BOX_BYTES, &map_res, (int)(cnb * GN + cg * 32), (int)(cmb * GM), res_bar(set));
+      mbar_expect_tx(res_bar(ew), G_BOX_BYTES / 4);
+      tma_load_2d(sRES + sub, &map_res, (int)(cnb * GN + cg * 32), (int)(cmb * GM + quarter * 32), res_bar(ew));
       ++r_issued;
       cg += 2;
       if (cg >= GN / 32 || cnb * GN + cg * 32 >= N) { cg = set; ct += gridDim.x; }
     };
-    if (use_res && st == 0) res_issue();
+    if (use_res && lane == 0) res_issue();
     uint32_t tile = 0;
     for (uint32_t t = blockIdx.x; t < n_tiles; t += gridDim.x, ++tile) {
       const uint32_t mb = t / NB, nb = t % NB;
@@ -230,13 +231,13 @@ k_gemm_tc(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUt
         uint4 rr[4];
         const bool res_here = staged && use_res;
         if (res_here) {
-          if (!mbar_wait(res_bar(set), r_used & 1u, abort_flag, lim)) { *abort_flag = 1; atomicExch(status, 1u); }
+          if (!mbar_wait(res_bar(ew), r_used & 1u, abort_flag, lim)) { *abort_flag = 1; atomicExch(status, 1u); }
           ++r_used;
           const uint8_t* rb = gbase + GemmSmem::RES + set * G_BOX_BYTES + my_off;
 #pragma unroll
           for (uint32_t q = 0; q < 4; ++q) rr[q] = *reinterpret_cast<const uint4*>(rb + ((q ^ sw) << 4));
-          asm volatile("bar.sync %0, 128;" ::"r"(set_bar) : "memory");
-          if (st == 0) res_issue();
+          __syncwarp();
+          if (lane == 0) res_issue();
         }
         tc_wait_ld();
         float f[32];
@@ -285,8 +286,8 @@ k_gemm_tc(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUt
               }
             }
           }
-          if (st == 0) bulk_wait_read<0>();             // the set's previous box has been read out
-          asm volatile("bar.sync %0, 128;" ::"r"(set_bar) : "memory");
+          if (lane == 0) bulk_wait_read<0>();           // the warp's previous rows have been read out
+          __syncwarp();
           uint8_t* ob = gbase + GemmSmem::STG + set * G_BOX_BYTES + my_off;
 #pragma unroll
           for (uint32_t q = 0; q < 4; ++q)
@@ -294,9 +295,9 @@ k_gemm_tc(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUt
                 make_uint4(pack_bf16(f[q * 8], f[q * 8 + 1]), pack_bf16(f[q * 8 + 2], f[q * 8 + 3]),
                            pack_bf16(f[q * 8 + 4], f[q * 8 + 5]), pack_bf16(f[q * 8 + 6], f[q * 8 + 7]));
           fence_async_smem();
-          asm volatile("bar.sync %0, 128;" ::"r"(set_bar) : "memory");
-          if (st == 0) {
-            tma_store_2d(&map_out, (int)col0, (int)(mb * GM), sSTG + set * G_BOX_BYTES);
+          __syncwarp();
+          if (lane == 0) {
+            tma_store_2d(&map_out, (int)col0, (int)(mb * GM + quarter * 32), sSTG + sub);
             bulk_commit();
           }
           continue;
@@ -327,11 +328,11 @@ k_gemm_tc(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUt
       mbar_arrive(tempty_bar(buf));
       asm volatile("bar.sync 1, 256;" ::: "memory");   // the bias of the next tile overwrites this one's
     }
-    if (st == 0) {
+    if (lane == 0) {
       bulk_wait_all();
       // residual boxes still on their way (only after a wait ran out): they must land before the block ends
       volatile uint32_t never = 0;
-      for (; r_used < r_issued; ++r_used) mbar_wait(res_bar(set), r_used & 1u, &never, 200000000ull);
+      for (; r_used < r_issued; ++r_used) mbar_wait(res_bar(ew), r_used & 1u, &never, 200000000ull);
     }
   }
 

@@ -166,8 +166,8 @@ bool make_tensor_map_bf16(CUtensorMap* map, const void* ptr, uint64_t rows, uint
 // of the matrix (a box that reaches them is filled with zeros there)
 bool make_tensor_map_bf16_pitch(CUtensorMap* map, const void* ptr, uint64_t rows, uint64_t k, uint64_t pitch,
                                 uint32_t box_rows);
-// boxes of 32 columns x 128 rows (64 bytes per row, 64-byte swizzle) of a dense [rows, cols] bf16 matrix: the
-// pieces in which the dense layers' epilogue stores its output and fetches the residual
+// boxes of 32 columns x 32 rows (64 bytes per row, 64-byte swizzle) of a dense [rows, cols] bf16 matrix: the
+// pieces in which a warp of the dense layers' epilogue stores its output and fetches the residual
 bool make_tensor_map_bf16_box32(CUtensorMap* map, const void* ptr, uint64_t rows, uint64_t cols);
 
 }  // namespace llmc
