@@ -44,6 +44,7 @@ def check_layer_output(got_bits, x_bits, ow, heads, **kw):
     (130, 192, 3, 320, 2, True, True, True),         # two query tiles, causal, odd tile counts
     (128, 768, 12, 3072, 2, False, False, False),    # BERT-base layer
     (256, 768, 12, 3072, 1, True, True, True),       # GPT-2-small layer
+    (200, 1024, 16, 4096, 3, False, False, False),   # BERT-large layer; 600 rows: four full row blocks and a partial one
 ])
 def test_layer_forward_matches_oracle(n, d, heads, ffn, S, pre_ln, causal, tanh):
     w = synth.layer_weights(d, ffn, 100 + d + n, DEV)
