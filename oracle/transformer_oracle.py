@@ -11,6 +11,8 @@ What it computes:
   two-layer feed-forward network with GELU, residual, layer normalisation.  Two arrangements:
     post-norm, bidirectional, GELU with erf          (BERT-style encoder layer)
     pre-norm,  causal mask,  GELU with tanh formula  (GPT-2-style decoder layer)
+* `embed`: h_0 = E(X), the hidden states that enter layer 1 in Algorithm 1: token embedding plus position
+  embedding, followed (BERT-style embeddings) by a layer normalisation; the paper does not spell E out either.
 * `infer`: Algorithm 1 (LLMCache-Infer) for a batch: for l = 1..L, probe bank l with the layer's input; hits
   take the stored output, misses run the layer and are inserted.
 
@@ -22,7 +24,9 @@ tight; with False nothing is rounded.
 
 Pins (tests/test_oracle_transformer.py): torch.nn.TransformerEncoderLayer in float64 (both arrangements),
 torch.nn.functional.layer_norm / gelu, hand-worked softmax rows, the causal mask (a future token cannot
-change an earlier output), permutation equivariance of the bidirectional layer, and for `infer` the chain
+change an earlier output), permutation equivariance of the bidirectional layer, for `embed` a hand-worked row,
+torch.nn.functional.embedding + layer_norm in float64, a table of zeros that leaves the position rows, and
+an id outside the table; and for `infer` the chain
 property of Algorithm 1 (a repeated input is served from the banks at every layer and returns the same bits).
 """
 from __future__ import annotations
@@ -72,6 +76,40 @@ def layer_norm(x: np.ndarray, g: np.ndarray, b: np.ndarray, eps: float = 1e-5) -
     mu = x.mean(axis=-1, keepdims=True)
     var = ((x - mu) ** 2).mean(axis=-1, keepdims=True)
     return (x - mu) / np.sqrt(var + eps) * g + b
+
+
+def embed_f64(tokens: np.ndarray, tok_emb_bits: np.ndarray, pos_emb_bits: Optional[np.ndarray],
+              layer_normed: bool = True, gain=None, bias=None, eps: float = 1e-5) -> np.ndarray:
+    """h_0 = E(X) (Algorithm 1, the assignment before the loop) in float64, not rounded.
+
+    tokens: int [S, n]; tok_emb_bits: bf16 bits [vocab, d]; pos_emb_bits: bf16 bits [n, d] or None.
+    h_0[s, i] = E_tok[tokens[s, i]] + E_pos[i], then layer_norm over d if layer_normed (gain, bias: float32 [d],
+    None = 1 and 0).  A token id outside the table gives a row of zeros.
+    """
+    tokens = np.asarray(tokens)
+    S, n = tokens.shape
+    E = _w(tok_emb_bits)
+    vocab, d = E.shape
+    out = np.zeros((S, n, d), dtype=np.float64)
+    for s in range(S):
+        for i in range(n):
+            t = int(tokens[s, i])
+            if t < 0 or t >= vocab:
+                continue
+            x = E[t].copy()
+            if pos_emb_bits is not None:
+                x = x + _w(pos_emb_bits[i])
+            if layer_normed:
+                g = np.ones(d) if gain is None else _v(gain)
+                b = np.zeros(d) if bias is None else _v(bias)
+                x = layer_norm(x, g, b, eps)
+            out[s, i] = x
+    return out
+
+
+def embed(tokens, tok_emb_bits, pos_emb_bits, layer_normed=True, gain=None, bias=None, eps=1e-5) -> np.ndarray:
+    """`embed_f64` stored as bf16 (round to nearest even): bit patterns [S, n, d]."""
+    return O.bf16_round(embed_f64(tokens, tok_emb_bits, pos_emb_bits, layer_normed, gain, bias, eps).astype(np.float32))
 
 
 _erf = np.vectorize(math.erf, otypes=[np.float64])

@@ -139,3 +139,47 @@ def test_divergence_monitor_flags_only_entries_whose_stored_output_drifted():
     pr = O.probe(bank, h, "bf16")
     checked, dropped = T.divergence_check(bank, w, h, pr, heads, stride=3, bound=0.05)
     assert [b for b, _, _ in checked] == [int(pr.hit_idx[i]) for i in range(0, len(pr.hit_idx), 3)] and dropped == 0
+
+
+def test_embed_hand_worked_library_and_degenerate_cases():
+    """h_0 = E(X) of Algorithm 1.  (a) one row by hand: [1, 3] has mean 2 and variance 1, so with eps = 0 the
+    normalised row is [-1, 1], and with gain [2, 1], bias [0.5, 0] it is [-1.5, 1]; (b) the library's
+    embedding lookup + layer_norm in float64; (c) a token table of zeros leaves the position rows, row i at
+    position i (an index mix-up between position and sequence would show); (d) an id outside the table gives a
+    zero row; (e) the stored form is the bf16 rounding of the exact one."""
+    f2b = lambda a: O.bf16_round(np.asarray(a, dtype=np.float32))
+    E = f2b([[1.0, 3.0], [2.0, 2.0]])
+    P0 = f2b([[0.0, 0.0]])
+    got = T.embed_f64(np.array([[0]]), E, P0, True, None, None, 0.0)
+    assert np.allclose(got, [[[-1.0, 1.0]]], atol=1e-15)
+    got = T.embed_f64(np.array([[0]]), E, P0, True, np.float32([2, 1]), np.float32([0.5, 0]), 0.0)
+    assert np.allclose(got, [[[-1.5, 1.0]]], atol=1e-15)
+    assert np.array_equal(T.embed_f64(np.array([[1]]), E, f2b([[0.5, -0.25]]), False), [[[2.5, 1.75]]])
+
+    rng = np.random.default_rng(3)
+    vocab, n, d, S = 50, 7, 24, 5
+    Eb, Pb = f2b(rng.standard_normal((vocab, d))), f2b(rng.standard_normal((n, d)))
+    g, b = rng.standard_normal(d).astype(np.float32), rng.standard_normal(d).astype(np.float32)
+    tok = rng.integers(0, vocab, (S, n))
+    te = torch.from_numpy(O.bf16_to_f32(Eb).astype(np.float64))
+    tp = torch.from_numpy(O.bf16_to_f32(Pb).astype(np.float64))
+    x = torch.nn.functional.embedding(torch.from_numpy(tok), te) + tp[None]
+    ref = torch.nn.functional.layer_norm(x, (d,), torch.from_numpy(g.astype(np.float64)),
+                                         torch.from_numpy(b.astype(np.float64)), 1e-5).numpy()
+    got = T.embed_f64(tok, Eb, Pb, True, g, b, 1e-5)
+    assert np.abs(got - ref).max() < 1e-12
+    assert np.abs(T.embed_f64(tok, Eb, Pb, False) - x.numpy()).max() == 0.0
+    assert np.abs(T.embed_f64(tok, Eb, None, False) - te.numpy()[tok]).max() == 0.0
+
+    zeros = np.zeros((vocab, d), dtype=np.uint16)
+    got = T.embed_f64(tok, zeros, Pb, False)
+    for s in range(S):
+        assert np.array_equal(got[s], O.bf16_to_f32(Pb).astype(np.float64))
+
+    bad = tok.copy()
+    bad[2, 3], bad[4, 0] = vocab, -1
+    got = T.embed_f64(bad, Eb, Pb, True, g, b, 1e-5)
+    assert not got[2, 3].any() and not got[4, 0].any() and got[2, 2].any()
+
+    bits = T.embed(tok, Eb, Pb, True, g, b, 1e-5)
+    assert bits.dtype == np.uint16 and np.array_equal(bits, O.bf16_round(ref.astype(np.float32)))
