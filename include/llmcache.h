@@ -392,6 +392,21 @@ int llmcache_layer_status(llmcache_layer_t* layer);
 /* As llmcache_bank_debug_knobs, for the layer's kernels. */
 int llmcache_layer_debug_knobs(llmcache_layer_t* layer, uint64_t wait_limit_ns, uint32_t flags);
 
+
+/* Input embeddings, "h_0 <- E(X)" of Algorithm 1: the hidden states that enter layer 1.
+ *   h0[s, i, :] = E_tok[tokens[s, i], :] + E_pos[i, :]                      (layer_norm == 0)
+ *   h0[s, i, :] = LayerNorm(that sum) * ln_gain + ln_bias over d_model      (layer_norm != 0; fp32, biased variance)
+ * tokens: device int64 [n_seqs, seq_len]; tok_emb: device bf16 [vocab, d_model]; pos_emb: device bf16
+ * [seq_len, d_model] or NULL (no position term); ln_gain, ln_bias: device f32 [d_model], each may be NULL (1 and
+ * 0); h0: device bf16 [n_seqs, seq_len, d_model], written once, rounded to nearest even.  The caller owns every
+ * buffer; nothing is allocated and the call does not synchronise.  d_model: a multiple of 8, at most 16,384
+ * (else LLMCACHE_ERR_SHAPE); tables and h0 16-byte aligned, tokens 8-byte aligned (else LLMCACHE_ERR_ARG).
+ * A token id outside [0, vocab) cannot be checked on the host: its row of h0 is written as zeros and, if bad_ids
+ * (device u32, caller-zeroed) is not NULL, counted there.  n_seqs == 0 is valid and does nothing (the pointers are then not looked at). */
+int llmcache_embed(const int64_t* tokens, uint64_t n_seqs, uint32_t seq_len, uint32_t d_model, int64_t vocab,
+                   const void* tok_emb, const void* pos_emb, int32_t layer_norm, const float* ln_gain,
+                   const float* ln_bias, float ln_eps, void* h0, uint32_t* bad_ids, void* stream);
+
 /* Algorithm 1 (LLMCache-Infer) for a batch of B sequences, without any host sync: for l = 1..n_layers,
  * probe banks[l] with the current hidden states (hits take the stored output), run layers[l] on the
  * compacted misses, commit (write back + insert).  banks == NULL runs every layer in full (no caching).

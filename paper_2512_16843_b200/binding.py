@@ -38,7 +38,7 @@ EXPORTS = [
     "llmcache_pool", "llmcache_fingerprint_pooled", "llmcache_probe_pooled", "llmcache_bank_pool_out",
     "llmcache_infer_pooled", "llmcache_fingerprint_static_status", "llmcache_bank_debug_knobs",
     "llmcache_layer_debug_knobs", "llmcache_debug_bounds_build", "llmcache_bank_input_stable",
-    "llmcache_shard_scan", "llmcache_shard_decide",
+    "llmcache_shard_scan", "llmcache_shard_decide", "llmcache_embed",
 ]
 KNOB_PRODUCER_IDLE = 1
 FINGERPRINT_STATIC_MAX_FLOATS = 2 * 1024 * 1024
@@ -112,6 +112,7 @@ def lib():
         L.llmcache_strerror.argtypes = [C.c_int]
         L.llmcache_last_cuda_error.restype = C.c_char_p
         L.llmcache_last_cuda_error.argtypes = []
+        L.llmcache_embed.argtypes = [vp, C.c_uint64, u32, u32, C.c_int64, vp, vp, C.c_int32, vp, vp, C.c_float, vp, vp, vp]
         L.llmcache_bank_bytes.argtypes = [C.POINTER(BankDesc), C.POINTER(C.c_size_t)]
         L.llmcache_bank_create.argtypes = [C.POINTER(BankDesc), C.POINTER(vp)]
         L.llmcache_bank_destroy.argtypes = [vp]
@@ -506,6 +507,17 @@ def llmcache_layer_forward(layer, x, n_seqs, n_seqs_dev, out, stream=None) -> No
 
 def llmcache_layer_status(layer) -> int:
     return int(lib().llmcache_layer_status(layer))
+
+
+def llmcache_embed(tokens, tok_emb, pos_emb, h0, *, layer_norm=True, ln_gain=None, ln_bias=None, eps=1e-5,
+                   bad_ids=None, stream=None) -> None:
+    """h0 = E(X) of Algorithm 1: token + position embeddings, optionally layer-normed.  tokens: int64 [S, n] on the
+    device; tok_emb bf16 [vocab, d]; pos_emb bf16 [n, d] or None; h0 bf16 [S, n, d]."""
+    S, n = tokens.shape
+    vocab, d = tok_emb.shape
+    _check(lib().llmcache_embed(_ptr(tokens), S, n, d, vocab, _ptr(tok_emb), _ptr(pos_emb), int(layer_norm),
+                                _ptr(ln_gain), _ptr(ln_bias), eps, _ptr(h0), _ptr(bad_ids), _stream(stream)),
+           "llmcache_embed")
 
 
 def llmcache_infer(banks, layers, h0, B, tau, buf_a, buf_b, h_miss, miss_out, io, stream=None) -> int:

@@ -19,6 +19,11 @@ cudaError_t launch_gemm(const __nv_bfloat16* a, const __nv_bfloat16* w, const fl
 cudaError_t launch_layernorm(const __nv_bfloat16* x, const float* g, const float* b, __nv_bfloat16* y, uint32_t M_max,
                              uint32_t d, const uint32_t* m_seq_dev, uint32_t rows_per_seq, float eps, int sm_count,
                              cudaStream_t st);
+// h0 = token embeddings + position embeddings (pos_emb may be null), optionally layer-normed (gain, bias may be null)
+cudaError_t launch_embed(const long long* tokens, const __nv_bfloat16* tok_emb, const __nv_bfloat16* pos_emb,
+                         const float* gain, const float* bias, __nv_bfloat16* h0, uint32_t* bad_ids,
+                         unsigned long long rows, uint32_t n, uint32_t d, long long vocab, int layer_norm, float eps,
+                         int sm_count, cudaStream_t st);
 // Attention on the tcgen05 tensor cores; vt: scratch for the per-head transposes of V,
 // seq_max * heads * 64 rows of attention_vt_pitch(n) elements.
 cudaError_t setup_attention_kernel();

@@ -244,3 +244,54 @@ def test_divergence_monitor_matches_oracle():
     assert np.array_equal(bank.export(L.WHAT_VALID).numpy(), ob.valid)
     assert bank.status() == L.OK and layer.status() == L.OK
     layer.close(); bank.close()
+
+
+@pytest.mark.parametrize("S,n,d,vocab,ln,affine,pos", [
+    (3, 40, 128, 1000, True, True, True),          # ragged: 4 chunks of a lane's 4 hold data on half the lanes
+    (2, 128, 768, 30522, True, False, True),       # BERT-base embeddings (the workload generator's recipe)
+    (2, 64, 768, 50257, False, False, True),       # GPT-2-style: no layer norm
+    (1, 33, 1024, 777, True, True, False),         # no position term
+    (2, 17, 2048, 512, True, True, True),          # eight chunks per lane
+    (1, 9, 4096, 64, True, True, True),            # any width: the sum is formed three times
+])
+def test_embed_matches_oracle(S, n, d, vocab, ln, affine, pos):
+    """h_0 = E(X): every element within one bf16 step of the float64 oracle (the sum of two bf16 numbers is exact
+    in fp32; the layer norm's fp32 mean and variance differ from float64 by ~1e-7 relative, which can flip a
+    rounding), and at most 1 % of them different at all."""
+    E = synth.randn((vocab, d), 11, DEV, torch.bfloat16, scale=0.5)
+    P = synth.randn((n, d), 12, DEV, torch.bfloat16, scale=0.5) if pos else None
+    g = (1 + 0.1 * synth.randn((d,), 13, DEV, torch.float32)) if affine else None
+    b = (0.1 * synth.randn((d,), 14, DEV, torch.float32)) if affine else None
+    tok = torch.randint(0, vocab, (S, n), generator=torch.Generator(device="cpu").manual_seed(15)).to(DEV)
+    tok[0, 1] = vocab + 5                           # not a token of the table
+    tok[S - 1, n - 1] = -3
+    h0 = torch.full((S, n, d), 7.0, dtype=torch.bfloat16, device=DEV)
+    bad = torch.zeros(1, dtype=torch.int32, device=DEV)
+    L.llmcache_embed(tok, E, P, h0, layer_norm=ln, ln_gain=g, ln_bias=b, eps=1e-5, bad_ids=bad)
+    torch.cuda.synchronize()
+    assert int(bad[0]) == 2
+    exact = T.embed_f64(tok.cpu().numpy(), synth.bf16_bits(E), synth.bf16_bits(P) if pos else None, ln,
+                        None if g is None else g.cpu().numpy(), None if b is None else b.cpu().numpy(), 1e-5)
+    want = O.bf16_round(exact.astype(np.float32))
+    got = synth.bf16_bits(h0)
+    assert not got[0, 1].any() and not got[S - 1, n - 1].any()
+    gf, wf = O.bf16_to_f32(got).astype(np.float64), O.bf16_to_f32(want).astype(np.float64)
+    step = np.maximum(np.abs(wf), 2.0 ** -126) * 2.0 ** -7         # one bf16 step at that magnitude, at most
+    assert np.all(np.abs(gf - wf) <= step)
+    assert np.mean(got != want) <= 0.01
+    if not ln:
+        assert np.array_equal(got, want)            # a sum of two bf16 numbers, rounded once: the same bits
+
+
+def test_embed_argument_errors_and_empty_batch():
+    E = synth.randn((10, 64), 1, DEV, torch.bfloat16)
+    tok = torch.zeros((2, 4), dtype=torch.int64, device=DEV)
+    h0 = torch.zeros((2, 4, 64), dtype=torch.bfloat16, device=DEV)
+    L.llmcache_embed(tok[:0], E, None, h0[:0])      # nothing to do
+    with pytest.raises(L.LLMCacheError) as e:
+        L.llmcache_embed(tok, synth.randn((10, 60), 1, DEV, torch.bfloat16), None,
+                         torch.zeros((2, 4, 60), dtype=torch.bfloat16, device=DEV))
+    assert e.value.status == L.ERR_SHAPE
+    with pytest.raises(L.LLMCacheError) as e:
+        L.llmcache_embed(tok, E, None, h0.view(-1)[1:])          # two bytes past a 16-byte boundary
+    assert e.value.status == L.ERR_ARG
