@@ -158,6 +158,18 @@ NCU_TRAFFIC = {
 
 SUB_WORKLOADS = ["bert_base", "gpt2_small", "single_layer_fp32"]
 
+# Shapes of the random-init models of the end-to-end workload (the families the paper evaluates on, Sec. V-A):
+# post-norm / bidirectional / erf-GELU encoders with layer-normed embeddings, and a pre-norm / causal / tanh-GELU
+# decoder without an embedding layer norm.
+E2E_MODELS = {
+    "bert_base": dict(name="BERT-base", layers=12, d_model=768, heads=12, ffn=3072, seq_len=384, batch=256, vocab=30522,
+                      bank=2048, pre_ln=False, causal=False, tanh_gelu=False, embed_ln=True),
+    "bert_large": dict(name="BERT-large", layers=24, d_model=1024, heads=16, ffn=4096, seq_len=512, batch=512,
+                       vocab=30522, bank=1024, pre_ln=False, causal=False, tanh_gelu=False, embed_ln=True),
+    "gpt2_small": dict(name="GPT-2-small", layers=12, d_model=768, heads=12, ffn=3072, seq_len=1024, batch=32,
+                       vocab=50257, bank=1024, pre_ln=True, causal=True, tanh_gelu=True, embed_ln=False),
+}
+
 
 def parse():
     ap = argparse.ArgumentParser()
@@ -173,8 +185,10 @@ def parse():
     ap.add_argument("--bank", type=int, default=65536, help="scan_stress: number of bank entries")
     ap.add_argument("--queries", type=int, default=65536, help="scan_stress: queries per batch (gather_stress: 8192 per probe)")
     ap.add_argument("--act-rows", type=int, default=16384, help="gather_stress: rows of the activation store (1 MiB each)")
-    ap.add_argument("--batch", type=int, default=0, help="e2e_bert_base: sequences per batch (default 256)")
-    ap.add_argument("--seq-len", type=int, default=0, help="e2e_bert_base: sequence length (default 384)")
+    ap.add_argument("--batch", type=int, default=0, help="e2e_bert_base: sequences per batch (default: the model's)")
+    ap.add_argument("--seq-len", type=int, default=0, help="e2e_bert_base: sequence length (default: the model's)")
+    ap.add_argument("--model", default="bert_base", choices=list(E2E_MODELS),
+                    help="e2e_bert_base: the shape of the random-init model (default bert_base)")
     ap.add_argument("--layers", type=int, default=0, help="number of per-layer banks (default: the workload's; fewer only for profiler captures)")
     ap.add_argument("--input-stable", type=int, default=1,
                     help="1: tell the banks that the probe inputs are resident buffers that no kernel of the run writes "
@@ -289,6 +303,21 @@ def build_batches(wl, seeds_tok, count, seed, device, B=None):
         fr = wl.tokens(B - n_edit, seed + 10 * i + 2)
         tok = torch.cat([ed, fr])[synth.shuffled(B, seed + 10 * i + 3, device)]
         out.append(wl.hidden(tok))
+    return out
+
+
+def build_token_batches(wl, seeds_tok, count, seed, device, B):
+    """The token ids of build_batches' batches (60% edits of the seeds, 40% fresh, shuffled), not embedded."""
+    from paper_2512_16843_b200 import synth
+    n_edit = int(round(B * CFG["edit_fraction"]))
+    g = torch.Generator().manual_seed(seed + 77)
+    out = []
+    for i in range(count):
+        if B < 8:
+            n_edit = int((torch.rand(B, generator=g) < CFG["edit_fraction"]).sum())
+        ed, _ = wl.edited(seeds_tok, n_edit, CFG["edit_positions"], seed + 10 * i + 1)
+        fr = wl.tokens(B - n_edit, seed + 10 * i + 2)
+        out.append(torch.cat([ed, fr])[synth.shuffled(B, seed + 10 * i + 3, device)].contiguous())
     return out
 
 
@@ -713,36 +742,46 @@ def run_gather_stress(args, steps=None, warmup=None):
 
 
 def run_e2e(args):
-    """End-to-end Algorithm 1 on a BERT-base-shaped random-init encoder: the same batches with and without
-    the per-layer banks (the paper's NoCache vs LLMCache comparison, Table I, on synthetic data)."""
+    """End-to-end Algorithm 1 on a random-init model of one of the shapes the paper evaluates on: token ids in,
+    h_L out (embedding step, then the layer-wise caching loop), the same batches with and without the per-layer
+    banks (the paper's NoCache vs LLMCache comparison, Table I, on synthetic data)."""
     from paper_2512_16843_b200 import binding as L
     from paper_2512_16843_b200 import synth
     L.lib()
     if not torch.cuda.is_available():
         raise SystemExit("bench.py needs a CUDA device (there is no CPU fallback)")
     dev = torch.device("cuda", 0)
-    Lyr = args.layers or CFG["layers"]
-    d, n, B, N, k = (CFG[x] for x in ("d_model", "seq_len", "batch", "bank", "fp_dim"))
+    MD = E2E_MODELS[args.model]
+    Lyr = args.layers or MD["layers"]
+    d, n, B, N, k = MD["d_model"], MD["seq_len"], MD["batch"], MD["bank"], CFG["fp_dim"]
     B, n = args.batch or B, args.seq_len or n          # e.g. --batch 1 --seq-len 128: the setting the paper measures in
-    heads, ffn = 12, 3072
+    heads, ffn = MD["heads"], MD["ffn"]
+    arch = dict(pre_ln=MD["pre_ln"], causal=MD["causal"], tanh_gelu=MD["tanh_gelu"])
     seed = synth.BASE_SEED + 6000
-    wl = synth.TokenWorkload(CFG["vocab"], n, d, seed, dev)
+    wl = synth.TokenWorkload(MD["vocab"], n, d, seed, dev)
     seeds_tok = wl.tokens(CFG["n_seeds"], seed + 5)
     proj = synth.projection(d, k, seed + 6, dev)
     ws = [synth.layer_weights(d, ffn, seed + 100 * (l + 1), dev) for l in range(Lyr)]
     CAL = 64                                           # sequences of the calibration batch
-    probe = L.Layer(ws[0], heads=heads, seq_len=n, max_seqs=max(B, CAL))
+    probe = L.Layer(ws[0], heads=heads, seq_len=n, max_seqs=max(B, CAL), **arch)
     need = L.llmcache_layer_bytes(probe.desc)
     probe.close()
     workspace = torch.empty(need + 256, dtype=torch.uint8, device=dev)
     off = (-workspace.data_ptr()) % 256
-    layers = [L.Layer(w, heads=heads, seq_len=n, max_seqs=max(B, CAL), workspace=workspace[off:]) for w in ws]
+    layers = [L.Layer(w, heads=heads, seq_len=n, max_seqs=max(B, CAL), workspace=workspace[off:], **arch) for w in ws]
     mk = lambda: torch.empty((max(B, CAL), n, d), dtype=torch.bfloat16, device=dev)
-    buf_a, buf_b, h_miss, miss_out = mk(), mk(), mk(), mk()
+    buf_a, buf_b, h_miss, miss_out, h0_buf = mk(), mk(), mk(), mk(), mk()
+    bad_ids = torch.zeros(1, dtype=torch.int32, device=dev)
+
+    def embed(tok):
+        """h_0 = E(X) through the library's kernel, into a resident buffer."""
+        L.llmcache_embed(tok, wl.E, wl.P, h0_buf, layer_norm=MD["embed_ln"], bad_ids=bad_ids)
+        return h0_buf
+
     # centring vectors (an input of the library): mean pooled layer input of a seeded calibration batch;
     # without them the pooled outputs of random-init layers are all alike and every sequence would match
     tau = 0.85
-    centers, h = [], wl.hidden(wl.tokens(CAL, seed + 9))
+    centers, h = [], embed(wl.tokens(CAL, seed + 9))[:CAL].clone()
     for l in range(Lyr):
         centers.append(h.float().mean(dim=(0, 1)).contiguous())
         layers[l].forward(h, buf_a[:CAL])
@@ -756,13 +795,14 @@ def run_e2e(args):
     hb, hbf, hl = [b.handle for b in banks], [b.handle for b in banks_f], [l.handle for l in layers]
     # enough distinct batches that none comes round again within an arm (a repeated batch would hit in full)
     P = args.pool_batches or min(160, args.warmup + args.steps + 10)
-    pool = build_batches(wl, seeds_tok, P, seed + 1000, dev, B)
+    pool = build_token_batches(wl, seeds_tok, P, seed + 1000, dev, B)
     # the banks are filled with fresh sequences and then the seeds (so that these are not the first to be evicted),
     # B at a time
     warm_tok = torch.cat([wl.tokens(N - CFG["n_seeds"], seed + 7), seeds_tok])
-    warm = [wl.hidden(warm_tok[i:i + B]) for i in range(0, N - B + 1, B)]
+    warm = [warm_tok[i:i + B].contiguous() for i in range(0, N - B + 1, B)]
 
-    def infer(h, cached):
+    def infer(tok, cached):
+        h = embed(tok)
         if cached == 2:
             return L.llmcache_infer_pooled(hbf, hl, h, B, None, buf_a, buf_b, h_miss, miss_out, bufs.io, pooled)
         return L.llmcache_infer(hb if cached else None, hl, h, B, None, buf_a, buf_b, h_miss, miss_out, bufs.io)
@@ -808,15 +848,22 @@ def run_e2e(args):
     F = torch.nn.functional
     w0 = ws[0]
 
-    def torch_layer(x):
-        qkv = F.linear(x, w0["w_qkv"], w0["b_qkv"].to(torch.bfloat16))
-        q, kk, v = (t.view(B, n, heads, 64).transpose(1, 2) for t in qkv.chunk(3, dim=-1))
-        a = F.scaled_dot_product_attention(q, kk, v).transpose(1, 2).reshape(B, n, d)
-        y = F.layer_norm(F.linear(a, w0["w_o"], w0["b_o"].to(torch.bfloat16)) + x, (d,), w0["ln1_g"].to(torch.bfloat16), w0["ln1_b"].to(torch.bfloat16))
-        f = F.gelu(F.linear(y, w0["w_1"], w0["b_1"].to(torch.bfloat16)))
-        return F.layer_norm(F.linear(f, w0["w_2"], w0["b_2"].to(torch.bfloat16)) + y, (d,), w0["ln2_g"].to(torch.bfloat16), w0["ln2_b"].to(torch.bfloat16))
+    bf = lambda t: t.to(torch.bfloat16)
+    ln = lambda t, g_, b_: F.layer_norm(t, (d,), bf(w0[g_]), bf(w0[b_]))
+    act = (lambda t: F.gelu(t, approximate="tanh")) if MD["tanh_gelu"] else F.gelu
 
-    x = pool[0]
+    def torch_layer(x):
+        a_in = ln(x, "ln1_g", "ln1_b") if MD["pre_ln"] else x
+        qkv = F.linear(a_in, w0["w_qkv"], bf(w0["b_qkv"]))
+        q, kk, v = (t.view(B, n, heads, 64).transpose(1, 2) for t in qkv.chunk(3, dim=-1))
+        a = F.scaled_dot_product_attention(q, kk, v, is_causal=MD["causal"]).transpose(1, 2).reshape(B, n, d)
+        y = F.linear(a, w0["w_o"], bf(w0["b_o"])) + x
+        if MD["pre_ln"]:
+            return F.linear(act(F.linear(ln(y, "ln2_g", "ln2_b"), w0["w_1"], bf(w0["b_1"]))), w0["w_2"], bf(w0["b_2"])) + y
+        y = ln(y, "ln1_g", "ln1_b")
+        return ln(F.linear(act(F.linear(y, w0["w_1"], bf(w0["b_1"]))), w0["w_2"], bf(w0["b_2"])) + y, "ln2_g", "ln2_b")
+
+    x = embed(pool[0])[:B]
     for _ in range(2):
         torch_layer(x)
     torch.cuda.synchronize()
@@ -838,11 +885,14 @@ def run_e2e(args):
            "hit_fraction_mean": res["llmcache_hits"], "hit_fraction_per_layer": per_layer_hits,
            "nocache_torch_library_ms": torch_ms, "speedup_vs_torch_library": torch_ms / res["llmcache"], "n_gpus": 1, "steps": args.steps, "warmup": args.warmup,
            "higher_is_better": False, "dtype": "bf16", "data": "synthetic",
-           "config": {"workload": f"BERT-base-shaped random-init encoder, {Lyr} layers, d_model 768, 12 heads, FFN 3072, "
-                                  f"batch {B} x seq_len {n}, 60% token-level edits of 64 seeds, per-layer banks of {N}, "
+           "config": {"workload": f"{MD['name']}-shaped random-init model ({'pre' if MD['pre_ln'] else 'post'}-norm, "
+                                  f"{'causal' if MD['causal'] else 'bidirectional'}), {Lyr} layers, d_model {d}, {heads} heads, "
+                                  f"FFN {ffn}, batch {B} x seq_len {n} token ids in (embedding step inside the timed "
+                                  f"region), 60% token-level edits of 64 seeds, per-layer banks of {N}, "
                                   f"fp_dim {k} (centred), tau {tau}",
                       "context": "the paper reports 2.4x for BERT-base on an A100 at batch 1 / seq 128 with real data "
                                  "(Table I); different hardware, data and batch: context only"}}
+    assert int(bad_ids[0]) == 0
     print(json.dumps(out))
     for o in layers + banks + banks_f:
         o.close()
