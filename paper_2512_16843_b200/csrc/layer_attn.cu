@@ -232,21 +232,26 @@ k_attention_tc(const __grid_constant__ CUtensorMap map_qkv, const __grid_constan
       tc_fence_after();
       // pass 1: maximum of the raw products over this thread's 64 columns (the scale is positive)
       float mx = -INFINITY;
-      {
-        uint32_t v0[32], v1[32];
-        tc_ld_32x32(acc, v0);
-        tc_ld_32x32(acc + 32, v1);
+#pragma unroll 1
+      for (uint32_t c = 0; c < 64; c += 32) {
+        uint32_t v[32];
+        tc_ld_32x32(acc + c, v);
         tc_wait_ld();
         if (masked) {
 #pragma unroll
           for (uint32_t i = 0; i < 32; ++i) {
-            const uint32_t ka = k0 + i, kb = ka + 32;
-            if (ka < n && (!causal || ka <= qrow)) mx = fmaxf(mx, __uint_as_float(v0[i]));
-            if (kb < n && (!causal || kb <= qrow)) mx = fmaxf(mx, __uint_as_float(v1[i]));
+            const uint32_t key = k0 + c + i;
+            if (key < n && (!causal || key <= qrow)) mx = fmaxf(mx, __uint_as_float(v[i]));
           }
         } else {
+          // four independent chains, joined at the end
+          float m4[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};
 #pragma unroll
-          for (uint32_t i = 0; i < 32; ++i) mx = fmaxf(mx, fmaxf(__uint_as_float(v0[i]), __uint_as_float(v1[i])));
+          for (uint32_t i = 0; i < 32; i += 4) {
+#pragma unroll
+            for (uint32_t u = 0; u < 4; ++u) m4[u] = fmaxf(m4[u], __uint_as_float(v[i + u]));
+          }
+          mx = fmaxf(mx, fmaxf(fmaxf(m4[0], m4[1]), fmaxf(m4[2], m4[3])));
         }
       }
       float* xm = xch + (j & 1u) * 256;
