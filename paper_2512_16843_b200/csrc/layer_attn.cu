@@ -16,6 +16,7 @@
 // output.  Two accumulators of 128 columns alternate between key tiles, so that the S of the next tile is computed
 // while the softmax works on the current one.  Every wait is bounded (status word, as in scan.cu).
 #include <cuda.h>
+#include <type_traits>
 #include "llmcache_internal.cuh"
 #include "ptx.cuh"
 #include "layer.cuh"
@@ -266,31 +267,36 @@ k_attention_tc(const __grid_constant__ CUtensorMap map_qkv, const __grid_constan
       // pass 2: exponentials, their sum, P as bf16 into shared memory (16-byte chunk c of row r at chunk c ^ (r % 8))
       unsigned long long ps2 = 0ull;
       const uint32_t sub = sP + hf * AT_TILE + r * 128u;
+      // two copies of the loop: only the tile that holds the sequence's end or the diagonal tests every key
+      auto pass2 = [&](auto with_mask) {
+        constexpr bool MASKED = decltype(with_mask)::value;
 #pragma unroll 1
-      for (uint32_t c = 0; c < 64; c += 32) {
-        uint32_t v[32];
-        tc_ld_32x32(acc + c, v);
-        tc_wait_ld();
+        for (uint32_t c = 0; c < 64; c += 32) {
+          uint32_t v[32];
+          tc_ld_32x32(acc + c, v);
+          tc_wait_ld();
 #pragma unroll
-        for (uint32_t q4 = 0; q4 < 4; ++q4) {
-          uint32_t pk[4];
+          for (uint32_t q4 = 0; q4 < 4; ++q4) {
+            uint32_t pk[4];
 #pragma unroll
-          for (uint32_t e = 0; e < 4; ++e) {
-            const uint32_t i = q4 * 8 + 2 * e;
-            const unsigned long long t2 = f2_fma(f2_pack(__uint_as_float(v[i]), __uint_as_float(v[i + 1])), sc2, nm2);
-            float pa = ex2f(f2_lo(t2)), pb = ex2f(f2_hi(t2));
-            if (masked) {
-              const uint32_t key = k0 + c + i;
-              if (dead || !(key < n && (!causal || key <= qrow))) pa = 0.f;
-              if (dead || !(key + 1 < n && (!causal || key + 1 <= qrow))) pb = 0.f;
+            for (uint32_t e = 0; e < 4; ++e) {
+              const uint32_t i = q4 * 8 + 2 * e;
+              const unsigned long long t2 = f2_fma(f2_pack(__uint_as_float(v[i]), __uint_as_float(v[i + 1])), sc2, nm2);
+              float pa = ex2f(f2_lo(t2)), pb = ex2f(f2_hi(t2));
+              if constexpr (MASKED) {
+                const uint32_t key = k0 + c + i;
+                if (dead || !(key < n && (!causal || key <= qrow))) pa = 0.f;
+                if (dead || !(key + 1 < n && (!causal || key + 1 <= qrow))) pb = 0.f;
+              }
+              ps2 = f2_add(ps2, f2_pack(pa, pb));
+              pk[e] = pack2(pa, pb);
             }
-            ps2 = f2_add(ps2, f2_pack(pa, pb));
-            pk[e] = pack2(pa, pb);
+            const uint32_t chunk = (c >> 3) + q4;
+            sts16(sub + ((chunk ^ (r & 7u)) << 4), pk[0], pk[1], pk[2], pk[3]);
           }
-          const uint32_t chunk = (c >> 3) + q4;
-          sts16(sub + ((chunk ^ (r & 7u)) << 4), pk[0], pk[1], pk[2], pk[3]);
         }
-      }
+      };
+      if (masked) pass2(std::true_type{}); else pass2(std::false_type{});
       tc_fence_before();                                              // S_j has been read ...
       asm volatile("fence.proxy.async.shared::cta;" ::: "memory");    // ... and P_j is visible to the tensor cores
       mbar_arrive(p_full);
