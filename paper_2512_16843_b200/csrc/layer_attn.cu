@@ -265,7 +265,7 @@ k_attention_tc(const __grid_constant__ CUtensorMap map_qkv, const __grid_constan
       const float corr = dead ? 1.f : ex2f(m_run - m_new);
       const unsigned long long sc2 = f2_pack(sc, sc), nm2 = f2_pack(dead ? 0.f : -m_new, dead ? 0.f : -m_new);
       // pass 2: exponentials, their sum, P as bf16 into shared memory (16-byte chunk c of row r at chunk c ^ (r % 8))
-      unsigned long long ps2 = 0ull;
+      float psa = 0.f, psb = 0.f;                        // two running sums (even and odd columns)
       const uint32_t sub = sP + hf * AT_TILE + r * 128u;
       // two copies of the loop: only the tile that holds the sequence's end or the diagonal tests every key
       auto pass2 = [&](auto with_mask) {
@@ -288,7 +288,8 @@ k_attention_tc(const __grid_constant__ CUtensorMap map_qkv, const __grid_constan
                 if (dead || !(key < n && (!causal || key <= qrow))) pa = 0.f;
                 if (dead || !(key + 1 < n && (!causal || key + 1 <= qrow))) pb = 0.f;
               }
-              ps2 = f2_add(ps2, f2_pack(pa, pb));
+              psa += pa;
+              psb += pb;
               pk[e] = pack2(pa, pb);
             }
             const uint32_t chunk = (c >> 3) + q4;
@@ -300,7 +301,7 @@ k_attention_tc(const __grid_constant__ CUtensorMap map_qkv, const __grid_constan
       tc_fence_before();                                              // S_j has been read ...
       asm volatile("fence.proxy.async.shared::cta;" ::: "memory");    // ... and P_j is visible to the tensor cores
       mbar_arrive(p_full);
-      l_run = l_run * corr + (f2_lo(ps2) + f2_hi(ps2));
+      l_run = l_run * corr + (psa + psb);
       m_run = m_new;
       corr_prev = corr;
     }
