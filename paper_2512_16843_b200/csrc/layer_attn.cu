@@ -49,6 +49,11 @@ __device__ __forceinline__ float ex2f(float x) {
   asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
   return y;
 }
+__device__ __forceinline__ float max3f(float a, float b, float c) {       // one instruction on this architecture
+  float y;
+  asm("max.f32 %0, %1, %2, %3;" : "=f"(y) : "f"(a), "f"(b), "f"(c));
+  return y;
+}
 __device__ __forceinline__ uint32_t pack2(float a, float b) {
   const __nv_bfloat162 v = __floats2bfloat162_rn(a, b);
   return *reinterpret_cast<const uint32_t*>(&v);
@@ -248,11 +253,12 @@ k_attention_tc(const __grid_constant__ CUtensorMap map_qkv, const __grid_constan
           // four independent chains, joined at the end
           float m4[4] = {-INFINITY, -INFINITY, -INFINITY, -INFINITY};
 #pragma unroll
-          for (uint32_t i = 0; i < 32; i += 4) {
+          for (uint32_t i = 0; i < 32; i += 8) {
 #pragma unroll
-            for (uint32_t u = 0; u < 4; ++u) m4[u] = fmaxf(m4[u], __uint_as_float(v[i + u]));
+            for (uint32_t u = 0; u < 4; ++u)
+              m4[u] = max3f(m4[u], __uint_as_float(v[i + 2 * u]), __uint_as_float(v[i + 2 * u + 1]));
           }
-          mx = fmaxf(mx, fmaxf(fmaxf(m4[0], m4[1]), fmaxf(m4[2], m4[3])));
+          mx = fmaxf(max3f(mx, m4[0], m4[1]), fmaxf(m4[2], m4[3]));
         }
       }
       float* xm = xch + (j & 1u) * 256;
