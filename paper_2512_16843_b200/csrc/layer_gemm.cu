@@ -76,13 +76,17 @@ __device__ __forceinline__ uint32_t pack_bf16(float a, float b) {
 }
 }  // namespace
 
+// ACT, RES, VT: the activation, whether a residual is added and whether the V columns go out transposed are fixed
+// per instantiation, so that each epilogue carries only its own code
+template <uint32_t ACT, bool RES, bool VT>
 __global__ void __launch_bounds__(GEMM_THREADS, 1)
 k_gemm_tc(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_w,
           const __grid_constant__ CUtensorMap map_out, const __grid_constant__ CUtensorMap map_res,
           const float* __restrict__ bias, const __nv_bfloat16* __restrict__ residual,
           __nv_bfloat16* __restrict__ out, uint32_t* __restrict__ status,
           uint32_t M_max, uint32_t N, uint32_t KB, const uint32_t* __restrict__ m_seq_dev, uint32_t rows_per_seq,
-          uint32_t act, VtOut vt) {
+          VtOut vt) {
+  constexpr uint32_t act = ACT;
   griddep_sync();
   extern __shared__ uint8_t smem_raw[];
   const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;
@@ -189,7 +193,7 @@ k_gemm_tc(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUt
     const uint32_t sub = set * G_BOX_BYTES + quarter * (G_BOX_BYTES / 4);     // this warp's 32 rows of its set's box
     const uint32_t row_in_tile = quarter * 32 + lane;
     const uint32_t my_off = row_in_tile * 64u, sw = (row_in_tile >> 1) & 3u;
-    const bool use_res = residual != nullptr;
+    constexpr bool use_res = RES;
     auto tile_full = [&](uint32_t t) { return (t / NB + 1) * GM <= M; };
     uint32_t r_used = 0;
     uint32_t ct = blockIdx.x, cg = set;                // next residual rows to request (lane 0 of every warp)
@@ -262,7 +266,7 @@ k_gemm_tc(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUt
 #pragma unroll
           for (int i = 0; i < 32; ++i) f[i] = gelu_tanh_f(f[i]);
         }
-        if (vt.ptr && col0 >= vt.col0) {
+        if (VT && col0 >= vt.col0) {
           // the V third of a q|k|v product goes out transposed per head, for the attention kernel:
           // vt[((seq * heads + h) * 64 + c) * pitch + pos]; the lanes of a warp are consecutive positions
           if (row_ok) {
@@ -304,7 +308,7 @@ k_gemm_tc(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUt
         }
         if (row_ok) {
           const size_t off = (size_t)row * N + col0;
-          if (residual) {
+          if (RES) {
             const uint4* r4 = reinterpret_cast<const uint4*>(residual + off);
 #pragma unroll
             for (int q = 0; q < 4; ++q) {
@@ -353,10 +357,33 @@ k_gemm_tc(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUt
   }
 }
 
+namespace {
+// the instantiation for (act, residual, transposed V columns), or null
+using GemmKernel = void (*)(const CUtensorMap, const CUtensorMap, const CUtensorMap, const CUtensorMap, const float*,
+                            const __nv_bfloat16*, __nv_bfloat16*, uint32_t*, uint32_t, uint32_t, uint32_t, const uint32_t*,
+                            uint32_t, VtOut);
+GemmKernel gemm_kernel(uint32_t act, bool res, bool vt) {
+  if (vt) return (!res && act == LAYER_ACT_NONE) ? k_gemm_tc<LAYER_ACT_NONE, false, true> : nullptr;
+  switch (act) {
+    case LAYER_ACT_NONE: return res ? k_gemm_tc<LAYER_ACT_NONE, true, false> : k_gemm_tc<LAYER_ACT_NONE, false, false>;
+    case LAYER_ACT_GELU_ERF: return res ? k_gemm_tc<LAYER_ACT_GELU_ERF, true, false> : k_gemm_tc<LAYER_ACT_GELU_ERF, false, false>;
+    case LAYER_ACT_GELU_TANH: return res ? k_gemm_tc<LAYER_ACT_GELU_TANH, true, false> : k_gemm_tc<LAYER_ACT_GELU_TANH, false, false>;
+    default: return nullptr;
+  }
+}
+}  // namespace
+
 cudaError_t setup_gemm_kernel() {
   cudaError_t e = tensor_map_setup();
   if (e != cudaSuccess) return e;
-  return cudaFuncSetAttribute(k_gemm_tc, cudaFuncAttributeMaxDynamicSharedMemorySize, GEMM_SMEM_BYTES);
+  const uint32_t acts[3] = {LAYER_ACT_NONE, LAYER_ACT_GELU_ERF, LAYER_ACT_GELU_TANH};
+  for (uint32_t act : acts)
+    for (int res = 0; res < 2; ++res) {
+      e = cudaFuncSetAttribute(gemm_kernel(act, res != 0, false), cudaFuncAttributeMaxDynamicSharedMemorySize, GEMM_SMEM_BYTES);
+      if (e != cudaSuccess) return e;
+    }
+  return cudaFuncSetAttribute(gemm_kernel(LAYER_ACT_NONE, false, true), cudaFuncAttributeMaxDynamicSharedMemorySize,
+                              GEMM_SMEM_BYTES);
 }
 
 // out[M, N] = act(a[M, K] . w[N, K]^T + bias) (+ residual).  K, N multiples of 64.
@@ -365,7 +392,8 @@ cudaError_t launch_gemm(const __nv_bfloat16* a, const __nv_bfloat16* w, const fl
                         uint32_t N, uint32_t K, const uint32_t* m_seq_dev, uint32_t rows_per_seq, uint32_t act,
                         int sm_count, cudaStream_t st, VtOut vt) {
   if (M_max == 0) return cudaSuccess;
-  if (residual && vt.ptr) return cudaErrorInvalidValue;      // the transposed columns take no residual
+  const GemmKernel kern = gemm_kernel(act, residual != nullptr, vt.ptr != nullptr);
+  if (!kern) return cudaErrorInvalidValue;                   // e.g. the transposed columns take no residual or activation
   alignas(64) CUtensorMap map_a, map_w, map_out, map_res;
   if (!make_tensor_map_bf16(&map_a, a, M_max, K, GM) || !make_tensor_map_bf16(&map_w, w, N, K, GN) ||
       !make_tensor_map_bf16_box32(&map_out, out, M_max, N) ||
@@ -373,8 +401,8 @@ cudaError_t launch_gemm(const __nv_bfloat16* a, const __nv_bfloat16* w, const fl
     return cudaErrorInvalidValue;
   const uint32_t tiles = ((M_max + GM - 1) / GM) * ((N + GN - 1) / GN);
   const uint32_t grid = tiles < (uint32_t)sm_count ? tiles : (uint32_t)sm_count;
-  return launch_k(k_gemm_tc, dim3(grid), dim3(GEMM_THREADS), GEMM_SMEM_BYTES, st, map_a, map_w, map_out, map_res, bias,
-                  residual, out, status, M_max, N, K / GK, m_seq_dev, rows_per_seq, act, vt);
+  return launch_k(kern, dim3(grid), dim3(GEMM_THREADS), GEMM_SMEM_BYTES, st, map_a, map_w, map_out, map_res, bias,
+                  residual, out, status, M_max, N, K / GK, m_seq_dev, rows_per_seq, vt);
 }
 
 }  // namespace llmc
