@@ -574,7 +574,10 @@ def run_ours(args):
             out["sub_workloads"][sub] = brief(rec)
         # the layer-wise caching loop end to end (token ids in, h_L out) on the BERT-base shape: the miss-path
         # layers are timed here, apart from the probe
-        out["algorithm1"] = run_e2e(args, steps=5, warmup=3)
+        try:
+            out["algorithm1"] = run_e2e(args, steps=5, warmup=3)
+        except Exception as exc:                      # the probe's figures above stand on their own
+            out["algorithm1"] = {"error": repr(exc)}
     if rank == 0:
         print(json.dumps(out))
     if dist is not None:
